@@ -1,0 +1,397 @@
+"""Pins for the CPU oracle against things other than itself.
+
+Hand-worked values for the formats the paper names, invariants, brute force
+over all codes, exact decimal arithmetic from the standard library, and
+double-precision library convolutions / matrix products (exact for these
+magnitudes).  None of these re-use the oracle's own formulae.
+"""
+import os
+from decimal import ROUND_HALF_UP, Decimal
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import reference as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_rows(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as fh:
+        for line in fh:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+# ---------------------------------------------------------------- quantizer (Sec. 2)
+def test_handworked_qmf_values():
+    for n, f, x, q, sat in _read_rows("qmf_handworked.txt"):
+        n, f, q, sat = int(n), int(f), int(q), int(sat)
+        got, cnt = orc.quantize(np.array([float(x)], dtype=np.float32), n, f)
+        assert int(got[0]) == q, (n, f, x, int(got[0]), q)
+        assert cnt.sat_pos == (1 if sat > 0 else 0), (n, f, x)
+        assert cnt.sat_neg == (1 if sat < 0 else 0), (n, f, x)
+        assert cnt.zeros == (1 if q == 0 else 0)
+
+
+def _nearest_code_bruteforce(x: float, n: int, f: int) -> int:
+    """Nearest representable value by exhaustive search over all 2^n codes, in exact
+    rational arithmetic; ties go to the larger magnitude; outside the range the nearest
+    code is the end of the range."""
+    xv = Fraction(x)
+    best, best_d = None, None
+    for q in range(-(1 << (n - 1)), 1 << (n - 1)):
+        d = abs(xv - Fraction(q, 1 << f))
+        if best is None or d < best_d or (d == best_d and abs(q) > abs(best)):
+            best, best_d = q, d
+    return best
+
+
+def test_quantizer_is_nearest_code_bruteforce_n4():
+    # every fp32 value on a fine grid across and beyond the range of Q1.3 ... Q4.0
+    for f in range(0, 4):
+        step = 2.0 ** -(f + 3)
+        xs = np.arange(-80, 81, dtype=np.float64) * step * (2.0 ** f) / 4 + 0.0
+        xs = np.concatenate([xs, np.arange(-80, 81) * step]).astype(np.float32)
+        got, _ = orc.quantize(xs, 4, f)
+        for x, g in zip(xs, got):
+            assert int(g) == _nearest_code_bruteforce(float(x), 4, f), (f, float(x))
+
+
+def test_quantizer_against_decimal_half_up_random():
+    rng = np.random.default_rng(1)
+    for n, f in [(16, 15), (16, 8), (16, 2), (12, 9), (8, 4), (5, 0)]:
+        xs = (rng.standard_normal(4000) * 2.0 ** (n - 1 - f) * 0.6).astype(np.float32)
+        # add exact ties
+        ties = ((rng.integers(-(1 << (n - 1)), 1 << (n - 1), 200) + 0.5) * 2.0 ** -f).astype(np.float32)
+        xs = np.concatenate([xs, ties])
+        got, cnt = orc.quantize(xs, n, f)
+        lo, hi = -(1 << (n - 1)), (1 << (n - 1)) - 1
+        sp = sn = z = 0
+        for x, g in zip(xs, got):
+            r = int((Decimal(float(x)) * (1 << f)).quantize(Decimal(1), rounding=ROUND_HALF_UP))
+            sp += r > hi
+            sn += r < lo
+            r = min(max(r, lo), hi)
+            z += r == 0
+            assert int(g) == r, (n, f, float(x))
+        assert (cnt.sat_pos, cnt.sat_neg, cnt.zeros) == (sp, sn, z)
+
+
+def test_quantizer_invariants_exhaustive_16bit():
+    n = 16
+    for f in (15, 8, 0):
+        q_all = np.arange(-32768, 32768, dtype=np.int64)
+        x = (q_all * 2.0 ** -f).astype(np.float32)          # exact: 16-bit integers scaled
+        q, cnt = orc.quantize(x, n, f)
+        assert np.array_equal(q.astype(np.int64), q_all)    # idempotence on representable values
+        assert cnt.sat_pos == 0 and cnt.sat_neg == 0 and cnt.zeros == 1
+        assert np.array_equal(orc.dequantize(q, f), q_all * 2.0 ** -f)
+
+
+def test_quantizer_monotone_bounded_symmetric_error():
+    rng = np.random.default_rng(2)
+    n, f = 12, 7
+    xs = np.sort((rng.standard_normal(20000) * 12).astype(np.float32))
+    q, _ = orc.quantize(xs, n, f)
+    qi = q.astype(np.int64)
+    assert np.all(np.diff(qi) >= 0)
+    assert qi.min() >= -(1 << (n - 1)) and qi.max() <= (1 << (n - 1)) - 1
+    inside = (xs.astype(np.float64) * 2 ** f < (1 << (n - 1)) - 0.5) & (xs.astype(np.float64) * 2 ** f > -(1 << (n - 1)) - 0.5)
+    err = np.abs(orc.dequantize(q, f) - xs.astype(np.float64))
+    assert np.all(err[inside] <= 2.0 ** -(f + 1))
+    # odd symmetry away from the asymmetric end of the range
+    qn, _ = orc.quantize(-xs, n, f)
+    keep = np.abs(qi) < (1 << (n - 1)) - 1
+    assert np.array_equal(qn.astype(np.int64)[keep], -qi[keep])
+
+
+def test_quantizer_special_values():
+    x = np.array([np.nan, np.inf, -np.inf, -0.0, 1e-45, -1e-45, 3e38, -3e38], dtype=np.float32)
+    q, cnt = orc.quantize(x, 16, 8)
+    assert q.tolist() == [0, 32767, -32768, 0, 0, 0, 32767, -32768]
+    assert (cnt.sat_pos, cnt.sat_neg, cnt.zeros) == (2, 2, 4)
+
+
+def test_relu_commutes_with_quantizer():
+    rng = np.random.default_rng(3)
+    xs = (rng.standard_normal(5000) * 3).astype(np.float32)
+    a, ca = orc.quantize(xs, 16, 10, relu=True)
+    b, _ = orc.quantize(xs, 16, 10, relu=False)
+    assert np.array_equal(a, np.maximum(b, 0))
+    assert ca.zeros == int(np.sum(np.maximum(b, 0) == 0))
+    c, _ = orc.quantize(np.maximum(xs, 0), 16, 10)
+    assert np.array_equal(a, c)
+
+
+def test_coarser_format_creates_zeros():
+    # Sec. 3.1: quantization raises the number of zero activations
+    rng = np.random.default_rng(4)
+    xs = np.abs(rng.standard_normal(10000)).astype(np.float32)
+    zeros = [orc.quantize(xs, 16, f)[1].zeros for f in (14, 8, 4, 2, 0)]
+    assert zeros == sorted(zeros) and zeros[-1] > zeros[0]
+    assert orc.quantize(np.array([0.1], np.float32), 16, 2)[0][0] == 0
+
+
+# ---------------------------------------------------------------- planes
+def test_plane_split_handworked_and_exhaustive():
+    q = np.array([-1, -32768, 32767, -255, 300, 0, 255, 256, -256, -257], dtype=np.int16)
+    hi, lo = orc.split_planes(q)
+    assert hi.tolist() == [-1, -128, 127, -1, 1, 0, 0, 1, -1, -2]
+    assert lo.tolist() == [255, 0, 255, 1, 44, 0, 255, 0, 0, 255]
+    q_all = np.arange(-32768, 32768, dtype=np.int16)
+    hi, lo = orc.split_planes(q_all)
+    assert np.array_equal(256 * hi.astype(np.int64) + lo.astype(np.int64), q_all.astype(np.int64))
+
+
+# ---------------------------------------------------------------- range rule (Sec. 2.3)
+@pytest.mark.parametrize("M,n,m", [(0.0, 16, 0), (0.99, 16, 0), (1.0, 16, 1), (1.5, 16, 1),
+                                   (2.0, 16, 2), (127.9, 16, 7), (128.0, 16, 8), (300.0, 8, 7),
+                                   (1e-30, 16, 0), (float("inf"), 16, 15), (40000.0, 16, 15),
+                                   (16383.9, 16, 14), (16384.0, 16, 15), (3.0, 1, 0)])
+def test_range_rule_handworked(M, n, m):
+    assert orc.int_bits_from_max(M, n) == m
+
+
+def test_range_from_tensor_and_paper_formats():
+    # Sec. 3.1: weights "very small and centered around zero" fit with 1-2 integer bits
+    x = np.array([0.02, -0.6, 0.3, np.nan], dtype=np.float32)
+    M, m, f = orc.measure_range(x, 16)
+    assert abs(M - 0.6) < 1e-7 and (m, f) == (0, 15)        # Q1.15
+    M, m, f = orc.measure_range(np.array([1.7, -0.2], np.float32), 16)
+    assert (m, f) == (1, 14)                                  # Q2.14
+    M, m, f = orc.measure_range(np.array([-5000.0, 20.0], np.float32), 16)
+    assert (m, f) == (13, 2)                                  # Q14.2
+    M, m, f = orc.measure_range(np.array([100.0], np.float32), 16)
+    assert (m, f) == (7, 8)                                   # Q8.8
+
+
+def test_range_rule_guarantees_representable_up_to_one_lsb():
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        n = int(rng.integers(2, 17))
+        x = (rng.standard_normal(64) * 10.0 ** rng.uniform(-3, 3)).astype(np.float32)
+        M, m, f = orc.measure_range(x, n)
+        q, cnt = orc.quantize(x, n, f)
+        if m < n - 1 or M < 2.0 ** (n - 1):
+            assert cnt.sat_neg == 0
+            assert np.all(np.abs(orc.dequantize(q, f) - x.astype(np.float64)) <= 2.0 ** -f)
+            if m > 0:
+                assert M >= 2.0 ** (m - 1)                    # m is the smallest that fits
+
+
+def test_range_accumulator_form_matches_float_form():
+    for F in (0, 5, 20, 29):
+        for A in [0, 1, (1 << F) - 1, 1 << F, (1 << F) + 1, 3 << F, (1 << (F + 6)) - 1, 1 << (F + 6),
+                  1 << (F + 20)]:
+            want = orc.int_bits_from_max(float(Fraction(A, 1 << F)), 16) if A < (1 << 52) else None
+            got = orc.int_bits_from_acc(A, F, 16)
+            exact = 0
+            while exact < 15 and not (Fraction(A, 1 << F) < (1 << exact)):
+                exact += 1
+            assert got == exact
+            if want is not None and A < (1 << 24):
+                assert got == want
+
+
+# ---------------------------------------------------------------- accumulation (Sec. 2)
+def test_handworked_dot_product():
+    kv, shifts = {}, []
+    for row in _read_rows("dot_product_handworked.txt"):
+        if row[0] == "shift":
+            shifts.append(tuple(int(t) for t in row[1:]))
+        else:
+            kv[row[0]] = [int(t) for t in row[1:]]
+    xq, _ = orc.quantize(np.array([[0.5, 0.25]], np.float32), 16, 15)
+    wq, _ = orc.quantize(np.array([[1.0, -0.5]], np.float32), 16, 14)
+    bq, _ = orc.quantize(np.array([0.1], np.float32), 16, 14)
+    assert xq.ravel().tolist() == kv["x_q"] and wq.ravel().tolist() == kv["w_q"]
+    assert bq.tolist() == kv["bias_q"]
+    acc = orc.ip_acc(xq, wq)
+    assert acc.ravel().tolist() == kv["acc"]
+    y, _ = orc.epilogue(acc, bq, 14, 29, False, 16, 15)
+    assert y.ravel().tolist() == kv["y_q"]
+    assert orc.epilogue_range(acc, bq, 14, 29, False) == kv["v"][0]
+    assert orc.epilogue_range(acc, None, 0, 29, False) == kv["acc"][0]
+    for v, s, r in shifts:
+        assert orc.shift_round(v, s) == r
+
+
+def _torch_conv_double(xq, fx, wq, fw, pad, stride):
+    """Library convolution (double) of the dequantized operands; exact because every product
+    is < 2^30 and every sum < 2^53."""
+    x = torch.from_numpy(xq.astype(np.float64) * 2.0 ** -fx).permute(0, 3, 1, 2)
+    w = torch.from_numpy(wq.astype(np.float64) * 2.0 ** -fw).permute(0, 3, 1, 2)
+    y = torch.nn.functional.conv2d(x, w, None, stride=stride, padding=pad)
+    return y.permute(0, 2, 3, 1).numpy()
+
+
+@pytest.mark.parametrize("shape", [
+    # N, H, W, C, K, R, S, pad, stride
+    (2, 7, 6, 5, 4, 3, 3, 1, 1), (1, 9, 9, 3, 7, 5, 5, 0, 1), (2, 8, 10, 4, 3, 3, 3, 1, 2),
+    (1, 5, 5, 2, 2, 1, 1, 0, 1), (3, 6, 6, 1, 5, 3, 2, 0, 1), (1, 11, 7, 6, 2, 3, 3, 2, 2),
+])
+def test_conv_equals_double_precision_library_conv(shape):
+    N, H, W, C, K, R, S, pad, stride = shape
+    rng = np.random.default_rng(sum(shape))
+    xq = rng.integers(-32768, 32768, (N, H, W, C)).astype(np.int16)
+    wq = rng.integers(-32768, 32768, (K, R, S, C)).astype(np.int16)
+    fx, fw = 9, 14
+    acc = orc.conv_acc(xq, wq, (pad, pad), (stride, stride))
+    ref = _torch_conv_double(xq, fx, wq, fw, pad, stride) * 2.0 ** (fx + fw)
+    assert acc.shape == ref.shape
+    assert np.array_equal(acc.astype(np.float64), ref)
+    # spot-check entry point
+    n, oh, ow, k = N - 1, acc.shape[1] // 2, acc.shape[2] - 1, K - 1
+    assert orc.conv_acc_at(xq, wq, (pad, pad), (stride, stride), n, oh, ow, k) == acc[n, oh, ow, k]
+
+
+def test_ip_equals_integer_matmul():
+    rng = np.random.default_rng(7)
+    xq = rng.integers(-32768, 32768, (5, 37)).astype(np.int16)
+    wq = rng.integers(-32768, 32768, (11, 37)).astype(np.int16)
+    acc = orc.ip_acc(xq, wq)
+    assert np.array_equal(acc, xq.astype(np.int64) @ wq.astype(np.int64).T)
+
+
+def test_structural_special_cases():
+    rng = np.random.default_rng(8)
+    xq = rng.integers(-2000, 2000, (2, 6, 5, 4)).astype(np.int16)
+    # 1x1 convolution is an inner product over pixels
+    w1 = rng.integers(-300, 300, (3, 1, 1, 4)).astype(np.int16)
+    a = orc.conv_acc(xq, w1)
+    b = orc.ip_acc(xq.reshape(-1, 4), w1.reshape(3, 4)).reshape(2, 6, 5, 3)
+    assert np.array_equal(a, b)
+    # inner product is a convolution over a 1x1 image
+    c = orc.conv_acc(xq.reshape(2, 1, 1, -1), rng.integers(-9, 9, (7, 1, 1, 120)).astype(np.int16))
+    assert c.shape == (2, 1, 1, 7)
+    # centre-tap delta kernel reproduces the input channel
+    wd = np.zeros((4, 3, 3, 4), dtype=np.int16)
+    for k in range(4):
+        wd[k, 1, 1, k] = 1
+    assert np.array_equal(orc.conv_acc(xq, wd, (1, 1)), xq.astype(np.int64))
+    # off-centre delta shifts: tap (r=0, s=1) reads the pixel one row above (cross-correlation)
+    ws = np.zeros((1, 3, 3, 4), dtype=np.int16)
+    ws[0, 0, 1, 2] = 1
+    sh = orc.conv_acc(xq, ws, (1, 1))[..., 0]
+    assert np.array_equal(sh[:, 1:, :], xq[:, :-1, :, 2]) and np.all(sh[:, 0, :] == 0)
+    # all-ones kernel on an all-ones image counts the taps inside the image: 4 / 6 / 9
+    ones = np.ones((1, 5, 5, 1), dtype=np.int16)
+    box = orc.conv_acc(ones, np.ones((1, 3, 3, 1), dtype=np.int16), (1, 1))[0, :, :, 0]
+    assert box[0, 0] == 4 and box[0, 2] == 6 and box[2, 2] == 9 and box[4, 4] == 4
+    # batch independence, linearity in x, output-channel permutation
+    w = rng.integers(-500, 500, (6, 3, 3, 4)).astype(np.int16)
+    full = orc.conv_acc(xq, w, (1, 1))
+    assert np.array_equal(full[1:], orc.conv_acc(xq[1:], w, (1, 1)))
+    assert np.array_equal(orc.conv_acc((2 * xq).astype(np.int16), w, (1, 1)), 2 * full)
+    perm = np.array([3, 0, 5, 1, 2, 4])
+    assert np.array_equal(orc.conv_acc(xq, w[perm], (1, 1)), full[..., perm])
+
+
+# ---------------------------------------------------------------- epilogue (Sec. 2.1)
+def test_epilogue_against_decimal_arithmetic():
+    rng = np.random.default_rng(9)
+    acc = rng.integers(-(1 << 40), 1 << 40, (50, 6)).astype(np.int64)
+    acc[0, :] = [0, 1 << 13, -(1 << 13), (1 << 13) - 1, 3 << 13, -(3 << 13)]   # exact ties at s = 14
+    bq = rng.integers(-32768, 32768, 6).astype(np.int16)
+    for relu in (False, True):
+        for (F, fb, n_out, f_out) in [(29, 14, 16, 15), (29, 14, 16, 3), (20, 20, 8, 2), (10, 4, 16, 12),
+                                      (30, 15, 4, 0)]:
+            y, cnt = orc.epilogue(acc, bq, fb, F, relu, n_out, f_out)
+            lo, hi = -(1 << (n_out - 1)), (1 << (n_out - 1)) - 1
+            sp = sn = z = 0
+            vmax = 0
+            for i in range(acc.shape[0]):
+                for c in range(6):
+                    v = int(acc[i, c]) + int(bq[c]) * (1 << (F - fb))
+                    if relu:
+                        v = max(v, 0)
+                    vmax = max(vmax, abs(v))
+                    r = int((Decimal(v) / Decimal(2) ** (F - f_out)).quantize(Decimal(1), rounding=ROUND_HALF_UP))
+                    sp += r > hi
+                    sn += r < lo
+                    r = min(max(r, lo), hi)
+                    z += r == 0
+                    assert int(y[i, c]) == r
+            assert (cnt.sat_pos, cnt.sat_neg, cnt.zeros) == (sp, sn, z)
+            assert orc.epilogue_range(acc, bq, fb, F, relu) == vmax
+
+
+def test_layer_equals_float_layer_then_quantize():
+    """Brute-force float-vs-fixed: the fixed-point layer output equals the quantizer applied to
+    the real-valued (double) layer on the dequantized operands, and so stays within half an
+    output LSB of it."""
+    rng = np.random.default_rng(10)
+    x = np.maximum(rng.standard_normal((2, 6, 6, 8)), 0).astype(np.float32)
+    w = (rng.standard_normal((5, 3, 3, 8)) * 0.15).astype(np.float32)
+    b = (rng.standard_normal(5) * 0.01).astype(np.float32)
+    fx = orc.measure_range(x, 16)[2]
+    xq, _ = orc.quantize(x, 16, fx)
+    wq, fw = orc.quantize_param(w, 16)
+    bq, _ = orc.quantize(b, 16, fw)
+    acc = orc.conv_acc(xq, wq, (1, 1))
+    res = orc.lp_layer(acc, fx, fw, bq, fw, True, 16)
+    real = _torch_conv_double(xq, fx, wq, fw, 1, 1) + bq.astype(np.float64) * 2.0 ** -fw
+    real = np.maximum(real, 0)
+    assert real.max() < 2.0 ** (15 - res.frac_bits)
+    if res.frac_bits < 15:
+        assert real.max() >= 2.0 ** (14 - res.frac_bits)     # decimal point as far left as the range allows
+    yq, _ = orc.quantize(real.astype(np.float32), 16, res.frac_bits)
+    # real is not an fp32 number in general: compare through exact decimal rounding instead
+    for v, got in zip(real.ravel(), res.y.ravel()):
+        r = int((Decimal(float(v)) * (1 << res.frac_bits)).quantize(Decimal(1), rounding=ROUND_HALF_UP))
+        assert int(got) == min(r, 32767)
+    assert np.all(np.abs(orc.dequantize(res.y, res.frac_bits) - real) <= 2.0 ** -res.frac_bits)
+    del yq
+
+
+def test_requantize_format_change():
+    q = np.array([5, -5, 6, -6, 3, 4, -4, 32767, -32768, 0], dtype=np.int16)
+    y, cnt = orc.requantize(q, 10, False, 16, 9)          # one bit coarser
+    assert y.tolist() == [3, -3, 3, -3, 2, 2, -2, 16384, -16384, 0]
+    y, cnt = orc.requantize(q, 10, True, 16, 12)          # two bits finer: saturates the ends
+    assert y.tolist() == [20, 0, 24, 0, 12, 16, 0, 32767, 0, 0]
+    assert (cnt.sat_pos, cnt.sat_neg, cnt.zeros) == (1, 0, 5)
+    y, _ = orc.requantize(q, 10, False, 8, 3)
+    assert y.tolist()[:7] == [0, 0, 0, 0, 0, 0, 0] and y.tolist()[7:9] == [127, -128]
+
+
+# ---------------------------------------------------------------- pooling
+def test_maxpool_commutes_with_quantizer():
+    rng = np.random.default_rng(11)
+    x = (rng.standard_normal((2, 6, 8, 3)) * 2).astype(np.float32)
+    q, _ = orc.quantize(x, 16, 9)
+    pooled_real = x.reshape(2, 3, 2, 4, 2, 3).max(axis=(2, 4))
+    want, _ = orc.quantize(pooled_real, 16, 9)
+    assert np.array_equal(orc.maxpool2x2(q), want)
+    # negative-only window: maximum is the least negative value, not zero
+    neg = -np.arange(1, 17, dtype=np.int16).reshape(1, 4, 4, 1)
+    assert orc.maxpool2x2(neg).ravel().tolist() == [-1, -3, -9, -11]
+
+
+# ---------------------------------------------------------------- network driver
+def test_network_driver_lenet_shapes_and_formats():
+    from paper_1711_04713_b200 import workloads as wl
+    specs = wl.lenet_specs()
+    params = wl.make_params(specs, seed=0)
+    x = wl.lenet_input(2, seed=0)
+    rec = orc.run_network(params, x, (16, 15), 16)
+    shapes = [r["y"].shape for r in rec]
+    assert shapes == [(2, 28, 28, 1), (2, 24, 24, 20), (2, 12, 12, 20), (2, 8, 8, 50), (2, 4, 4, 50),
+                      (2, 500), (2, 10)]
+    for r in rec:
+        if r["type"] in ("conv", "ip"):
+            assert 0 <= r["frac_bits"] <= 15
+            assert r["counters"].sat_neg == 0
+            # the decimal point chosen from the batch range leaves at most the one-LSB edge case
+            assert r["counters"].sat_pos <= 1
+    # running again with the formats fixed reproduces the calibrated run
+    fixed = [r["frac_bits"] for r in rec if r["type"] in ("conv", "ip")]
+    rec2 = orc.run_network(params, x, (16, 15), 16, fixed_formats=fixed)
+    for a, b in zip(rec, rec2):
+        assert np.array_equal(a["y"], b["y"])
