@@ -1,0 +1,162 @@
+/*
+ * adaption.h - C ABI of the B200 (sm_100a) forward path of the low-precision layers of
+ * ADaPTION (arXiv 1711.04713): LPConvolution, LPInnerProduct, LPAct, the quantizer they
+ * share and the dynamic-range measurement that fixes each layer's decimal point.
+ *
+ * Fixed point (Sec. 2 of the paper, "QBD.AD"): a value is stored as a signed integer q of
+ * n_bits = BD + AD bits (BD counts the sign bit) and stands for q * 2^-frac_bits,
+ * frac_bits = AD.  q lies in [-2^(n_bits-1), 2^(n_bits-1)-1].  1 <= n_bits <= 16 and
+ * 0 <= frac_bits <= n_bits-1.
+ *
+ * Storage of a fixed-point tensor in device memory ("planes"): rows of `inner` elements with
+ * a pitch of c_stride elements (c_stride >= inner, a multiple of 16; the padding holds zeros).
+ *   n_bits >  8 : two byte planes, hi = q >> 8 (signed) and lo = q & 255 (unsigned),
+ *                 so that q = 256*hi + lo;
+ *   n_bits <= 8 : one plane, `lo`, holding q itself as a signed byte; hi is NULL.
+ * An optional int16 copy q16 (same pitch) can be requested on outputs.
+ * Activations are NHWC (rows = pixels, inner = channels); convolution weights are
+ * [K][R][S][C] (rows = K*R*S, inner = C); inner-product operands are [B][K] and [O][K].
+ *
+ * General rules.  Every pointer is a DEVICE pointer unless its name starts with h_.  The
+ * caller owns every buffer; the library allocates nothing.  All work is enqueued on the
+ * given CUDA stream (a cudaStream_t passed as void*; NULL = default stream) and returns
+ * without synchronising.  Every function returns an ADAPTION_* status; argument errors are
+ * found on the host before anything is launched.  Plane and workspace pointers must be
+ * 16-byte aligned.  Counters in adaption_stats accumulate: the caller zeroes them.
+ */
+#ifndef ADAPTION_H
+#define ADAPTION_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* exported symbols of the shared library */
+#if defined(__GNUC__)
+#define ADAPTION_API __attribute__((visibility("default")))
+#else
+#define ADAPTION_API
+#endif
+
+enum {
+  ADAPTION_OK = 0,
+  ADAPTION_ERR_INVALID_ARG = 1,
+  ADAPTION_ERR_UNSUPPORTED = 2,
+  ADAPTION_ERR_ALIGNMENT = 3,
+  ADAPTION_ERR_WORKSPACE = 4,
+  ADAPTION_ERR_K_TOO_LARGE = 5,
+  ADAPTION_ERR_CUDA = 6,
+  ADAPTION_ERR_TIMEOUT = 7
+};
+
+/* rounding_scheme of the paper (Sec. 2, Sec. 2.4).  Deterministic = round to nearest, ties
+ * away from zero.  Stochastic rounding is not implemented: ADAPTION_ERR_UNSUPPORTED. */
+enum { ADAPTION_ROUND_DETERMINISTIC = 0, ADAPTION_ROUND_STOCHASTIC = 1 };
+
+/* What a layer call does with its pre-activation values v (accumulator + bias, after ReLU if
+ * asked): REQUANT rounds them to the output format and stores them; RANGE only records
+ * max|v| in stats.max_abs_acc (the per-layer range measurement of Sec. 2.1 / 2.3). */
+enum { ADAPTION_MODE_REQUANT = 0, ADAPTION_MODE_RANGE = 1 };
+
+/* Kernel choice for the layer calls.  AUTO takes the tensor-core path whenever the shape
+ * allows it; DIRECT forces the plain integer kernel, TENSOR fails with
+ * ADAPTION_ERR_UNSUPPORTED where the tensor-core path cannot run. */
+enum { ADAPTION_ALGO_AUTO = 0, ADAPTION_ALGO_TENSOR = 1, ADAPTION_ALGO_DIRECT = 2 };
+
+typedef struct adaption_qfmt {
+  int32_t n_bits;    /* BD + AD */
+  int32_t frac_bits; /* AD */
+} adaption_qfmt;
+
+typedef struct adaption_qtensor {
+  void* hi;          /* int8 plane q >> 8, NULL when n_bits <= 8 */
+  void* lo;          /* uint8 plane q & 255 (n_bits > 8) or int8 plane q (n_bits <= 8) */
+  int16_t* q16;      /* optional int16 copy (outputs only), may be NULL */
+  adaption_qfmt fmt;
+  int64_t c_stride;  /* row pitch in elements, multiple of 16, >= inner extent */
+} adaption_qtensor;
+
+typedef struct adaption_stats {
+  uint64_t zeros;       /* stored outputs equal to 0 (Sec. 3.1: sparsity = zeros / total) */
+  uint64_t sat_pos;     /* values clipped at the top of the output range */
+  uint64_t sat_neg;     /* values clipped at the bottom */
+  int64_t max_abs_acc;  /* RANGE mode: max |v| in units of 2^-(f_x + f_w) */
+  int32_t status;       /* 0, or ADAPTION_ERR_TIMEOUT if a device-side wait gave up */
+  int32_t reserved;
+} adaption_stats;
+
+typedef struct adaption_conv_shape {
+  int32_t N, H, W, C; /* input NHWC */
+  int32_t K;          /* output channels */
+  int32_t R, S;       /* filter height, width */
+  int32_t pad_h, pad_w;
+  int32_t stride_h, stride_w;
+} adaption_conv_shape;
+
+/* Sec. 2.1 / 2.3 (dynamic range -> decimal point).  Folds max|x| of x[0..numel) into
+ * *d_max_abs (the caller sets it to 0 before the first tensor of a group; NaN is ignored),
+ * then writes to *d_fmt_out the format with n_bits total bits whose integer part is the
+ * smallest that holds the maximum: m = min{m in [0, n_bits-1] : max < 2^m},
+ * frac_bits = n_bits-1-m.  d_fmt_out may be NULL.  numel may be 0. */
+ADAPTION_API int adaption_measure_range(const float* d_x, size_t numel, int32_t n_bits, float* d_max_abs,
+                           adaption_qfmt* d_fmt_out, void* stream);
+
+/* Sec. 2 (the quantizer of the LP layers).  x is fp32 [outer][inner] dense; out receives
+ * q = saturate(round(x * 2^frac_bits)).  If d_fmt is not NULL the fractional bits are read
+ * on the device from d_fmt->frac_bits (as written by adaption_measure_range) instead of
+ * out.fmt.frac_bits; n_bits always comes from out.fmt.  NaN -> 0, +-Inf saturate.
+ * d_stats (may be NULL) accumulates zeros and saturations over the outer*inner real elements. */
+ADAPTION_API int adaption_quantize(const float* d_x, size_t outer, size_t inner, adaption_qtensor out,
+                      const adaption_qfmt* d_fmt, int32_t rounding, adaption_stats* d_stats,
+                      void* stream);
+
+/* Sec. 2.1 (LPAct: the activation quantizer, followed by ReLU when relu != 0).  Exactly one
+ * of d_x_f32 (fp32 [outer][inner]) and h_x_q (host pointer to the descriptor of a fixed-point
+ * tensor, whose format is converted) is given.  Otherwise as adaption_quantize. */
+ADAPTION_API int adaption_lp_act(const float* d_x_f32, const adaption_qtensor* h_x_q, size_t outer,
+                    size_t inner, int32_t relu, adaption_qtensor out, const adaption_qfmt* d_fmt,
+                    int32_t rounding, adaption_stats* d_stats, void* stream);
+
+/* Sec. 2 (LPConvolution forward).  y[n,oh,ow,k] = requant(relu(sum_{r,s,c} x[n, oh*stride_h
+ * + r - pad_h, ow*stride_w + s - pad_w, c] * w[k,r,s,c] + bias[k])), taps outside the image
+ * contribute 0, the sum is exact.  x and w must share c_stride.  bias_q (int16 [K], may be
+ * NULL) has bias_frac_bits <= x.fmt.frac_bits + w.fmt.frac_bits.  In RANGE mode y is ignored.
+ * The workspace query returns the bytes the call needs (possibly 0); the workspace contents
+ * need no initialisation.  d_stats must not be NULL. */
+ADAPTION_API size_t adaption_lp_conv_workspace_bytes(const adaption_conv_shape* h_shape, adaption_qfmt fx,
+                                        adaption_qfmt fw, int64_t c_stride, int32_t algo);
+ADAPTION_API int adaption_lp_conv_fwd(const adaption_conv_shape* h_shape, adaption_qtensor x,
+                         adaption_qtensor w, const int16_t* d_bias_q, int32_t bias_frac_bits,
+                         int32_t relu, int32_t mode, int32_t algo, adaption_qtensor y,
+                         adaption_stats* d_stats, void* d_workspace, size_t workspace_bytes,
+                         void* stream);
+
+/* Sec. 2 (LPInnerProduct forward).  y[b,o] = requant(relu(sum_k x[b,k] * w[o,k] + bias[o])).
+ * x is [B][K], w is [O][K], y is [B][O]. */
+ADAPTION_API size_t adaption_lp_ip_workspace_bytes(int64_t B, int64_t K, int64_t O, adaption_qfmt fx,
+                                      adaption_qfmt fw, int32_t algo);
+ADAPTION_API int adaption_lp_ip_fwd(int64_t B, int64_t K, int64_t O, adaption_qtensor x, adaption_qtensor w,
+                       const int16_t* d_bias_q, int32_t bias_frac_bits, int32_t relu,
+                       int32_t mode, int32_t algo, adaption_qtensor y, adaption_stats* d_stats,
+                       void* d_workspace, size_t workspace_bytes, void* stream);
+
+/* The 2x2, stride-2 max pooling that sits between the low-precision layers of the networks
+ * the paper studies (VGG16; Table 1, "Pooling").  Works on the stored integers, same format
+ * in and out; H and W even.  x is [N][H][W][C], y is [N][H/2][W/2][C]. */
+ADAPTION_API int adaption_maxpool2x2(adaption_qtensor x, int32_t N, int32_t H, int32_t W, int32_t C,
+                        adaption_qtensor y, void* stream);
+
+/* Host helper for RANGE mode (Sec. 2.3): the format with n_bits whose integer part is the
+ * smallest that holds max_abs_acc * 2^-acc_frac_bits. */
+ADAPTION_API int adaption_choose_frac_bits_from_acc(int64_t max_abs_acc, int32_t acc_frac_bits,
+                                       int32_t n_bits, adaption_qfmt* h_out);
+
+ADAPTION_API const char* adaption_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAPTION_H */

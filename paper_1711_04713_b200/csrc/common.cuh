@@ -1,0 +1,143 @@
+// Shared device/host helpers of the CUDA path (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "adaption.h"
+
+namespace adaption {
+
+// Parameters of the requantizer applied to a pre-activation value v given in units of
+// 2^-F (paper Sec. 2.1: the activation is quantized to the layer's format, ReLU follows;
+// rounding is to nearest with ties away from zero, then saturation).
+struct RequantParams {
+  int32_t shift;     // F - f_out; > 0: rounding right shift, <= 0: exact left shift by -shift
+  int32_t relu;      // clamp negatives to zero first
+  int32_t qmin;      // -2^(n_out-1)
+  int32_t qmax;      //  2^(n_out-1)-1
+  int32_t out_planes;  // 2: hi/lo byte planes (n_out > 8), 1: single signed byte plane
+};
+
+struct Counts {
+  uint32_t zeros = 0, sat_pos = 0, sat_neg = 0;
+};
+
+// v / 2^shift rounded half away from zero, saturated.  For shift > 0 and negative v the
+// identity -((-v + h) >> s) == (v + h - 1) >> s (h = 2^(s-1), arithmetic shift) is used.
+__device__ __forceinline__ int32_t requant_value(int64_t v, const RequantParams& rq, bool counted,
+                                                 Counts& c) {
+  if (rq.relu && v < 0) v = 0;
+  int64_t r;
+  if (rq.shift > 0) {
+    const int64_t half = (int64_t)1 << (rq.shift - 1);
+    r = (v + half + (v >> 63)) >> rq.shift;
+  } else {
+    r = v * ((int64_t)1 << (-rq.shift));
+  }
+  if (r > (int64_t)rq.qmax) {
+    r = rq.qmax;
+    c.sat_pos += counted;
+  } else if (r < (int64_t)rq.qmin) {
+    r = rq.qmin;
+    c.sat_neg += counted;
+  }
+  c.zeros += (counted && r == 0);
+  return (int32_t)r;
+}
+
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ int64_t warp_max_i64(int64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    int64_t t = __shfl_xor_sync(0xffffffffu, v, o);
+    v = t > v ? t : v;
+  }
+  return v;
+}
+
+// One atomic per warp and counter; lanes must all call.
+__device__ __forceinline__ void flush_counts_warp(const Counts& c, adaption_stats* stats) {
+  uint32_t z = warp_sum(c.zeros), p = warp_sum(c.sat_pos), n = warp_sum(c.sat_neg);
+  if ((threadIdx.x & 31) == 0 && stats != nullptr) {
+    if (z) atomicAdd((unsigned long long*)&stats->zeros, (unsigned long long)z);
+    if (p) atomicAdd((unsigned long long*)&stats->sat_pos, (unsigned long long)p);
+    if (n) atomicAdd((unsigned long long*)&stats->sat_neg, (unsigned long long)n);
+  }
+}
+
+__device__ __forceinline__ void flush_max_warp(int64_t m, adaption_stats* stats) {
+  m = warp_max_i64(m);
+  if ((threadIdx.x & 31) == 0 && m > 0) atomicMax((long long*)&stats->max_abs_acc, (long long)m);
+}
+
+// canonical integer of element i from the stored planes
+__device__ __forceinline__ int32_t load_q(const int8_t* hi, const uint8_t* lo, size_t i) {
+  if (hi != nullptr) return ((int32_t)hi[i]) * 256 + (int32_t)lo[i];
+  return (int32_t)((const int8_t*)lo)[i];
+}
+
+__device__ __forceinline__ void store_q(int8_t* hi, uint8_t* lo, int16_t* q16, size_t i, int32_t q) {
+  if (hi != nullptr) {
+    hi[i] = (int8_t)(q >> 8);
+    lo[i] = (uint8_t)(q & 255);
+  } else {
+    lo[i] = (uint8_t)(q & 255);
+  }
+  if (q16 != nullptr) q16[i] = (int16_t)q;
+}
+
+inline RequantParams make_requant(int32_t acc_frac_bits, adaption_qfmt out, int32_t relu) {
+  RequantParams rq;
+  rq.shift = acc_frac_bits - out.frac_bits;
+  rq.relu = relu ? 1 : 0;
+  rq.qmin = -(1 << (out.n_bits - 1));
+  rq.qmax = (1 << (out.n_bits - 1)) - 1;
+  rq.out_planes = out.n_bits > 8 ? 2 : 1;
+  return rq;
+}
+
+inline bool fmt_ok(adaption_qfmt f) {
+  return f.n_bits >= 1 && f.n_bits <= 16 && f.frac_bits >= 0 && f.frac_bits <= f.n_bits - 1;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// a fixed-point tensor as an input operand: planes present and aligned
+int check_qtensor_in(const adaption_qtensor& t, int64_t inner);
+// ... as an output: planes (or at least q16) present
+int check_qtensor_out(const adaption_qtensor& t, int64_t inner);
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? ADAPTION_OK : ADAPTION_ERR_CUDA; }
+
+// ---- launches implemented in the other translation units ---------------------------------
+struct GemmProblem {
+  // logical GEMM: rows M (pixels or batch), columns N (output channels), reduction over K
+  int64_t M = 0, N = 0, K = 0;   // K: real reduction length (no padding)
+  bool is_conv = false;
+  adaption_conv_shape cs{};      // valid when is_conv
+  int32_t OH = 0, OW = 0;
+  adaption_qtensor x{}, w{}, y{};
+  const int16_t* bias = nullptr;
+  int32_t bias_shift = 0;        // F - bias_frac_bits
+  int32_t acc_frac_bits = 0;     // F = f_x + f_w
+  int32_t relu = 0, mode = 0;
+  adaption_stats* stats = nullptr;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  cudaStream_t stream = nullptr;
+};
+
+int launch_direct(const GemmProblem& p);
+bool tensor_path_supported(const GemmProblem& p);
+size_t tensor_path_workspace(const GemmProblem& p);
+int launch_tensor(const GemmProblem& p);
+// bias/ReLU/requantize (or range) of an int64 accumulator matrix acc[M][ld] -> y
+int launch_finalize(const int64_t* acc, int64_t ld, const GemmProblem& p);
+
+}  // namespace adaption

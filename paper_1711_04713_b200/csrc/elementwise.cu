@@ -1,0 +1,439 @@
+// HBM-bound kernels: dynamic-range measurement, the fp32 -> fixed-point quantizer (LPAct with an
+// fp32 input is the same kernel with the ReLU flag), fixed-point format conversion, 2x2 max-pool.
+// All of them are coalesced streaming kernels sized to a multiple of the SM count.
+#include "common.cuh"
+
+namespace adaption {
+
+static int g_num_sms = 0;
+
+int num_sms() {
+  if (g_num_sms == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+    g_num_sms = n;
+  }
+  return g_num_sms;
+}
+
+static inline int stream_grid(size_t work_items, int threads, int blocks_per_sm) {
+  size_t want = (work_items + threads - 1) / threads;
+  size_t cap = (size_t)num_sms() * blocks_per_sm;
+  if (want < 1) want = 1;
+  return (int)(want < cap ? want : cap);
+}
+
+// ------------------------------------------------------------------------------------------
+// Dynamic range (paper Sec. 2.1, Sec. 2.3): max |x|, NaN ignored.  Non-negative floats order
+// like their bit patterns, so the cross-block reduction is an integer atomicMax.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) range_max_abs_kernel(const float* __restrict__ x, size_t numel,
+                                                            size_t head, size_t n4,
+                                                            float* __restrict__ d_max_abs) {
+  float m = 0.0f;
+  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  // unaligned head and tail as scalars
+  if (tid < head) m = fmaxf(m, fabsf(x[tid]));
+  const size_t tail_begin = head + n4 * 4;
+  if (tail_begin + tid < numel) m = fmaxf(m, fabsf(x[tail_begin + tid]));
+  const float4* __restrict__ x4 = reinterpret_cast<const float4*>(x + head);
+  size_t i = tid;
+  for (; i + 3 * nthreads < n4; i += 4 * nthreads) {
+    float4 a = __ldg(x4 + i), b = __ldg(x4 + i + nthreads), c = __ldg(x4 + i + 2 * nthreads),
+           d = __ldg(x4 + i + 3 * nthreads);
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(b.x), fabsf(b.y)), fmaxf(fabsf(b.z), fabsf(b.w))));
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(c.x), fabsf(c.y)), fmaxf(fabsf(c.z), fabsf(c.w))));
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(d.x), fabsf(d.y)), fmaxf(fabsf(d.z), fabsf(d.w))));
+  }
+  for (; i < n4; i += nthreads) {
+    float4 a = __ldg(x4 + i);
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  __shared__ float wmax[8];
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float b = wmax[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) b = fmaxf(b, wmax[w]);
+    if (b > 0.0f) atomicMax(reinterpret_cast<int*>(d_max_abs), __float_as_int(b));
+  }
+}
+
+// Decimal point from the maximum (Sec. 2.3): smallest m in [0, n-1] with max < 2^m.  For
+// max >= 1 with binary exponent e (max in [2^e, 2^(e+1))) that is e+1; Inf has e = 128.
+__global__ void choose_fmt_kernel(const float* __restrict__ d_max_abs, int32_t n_bits,
+                                  adaption_qfmt* __restrict__ d_fmt) {
+  const int bits = __float_as_int(*d_max_abs) & 0x7fffffff;
+  const int e = (bits >> 23) - 127;
+  int m = e >= 0 ? e + 1 : 0;
+  if (m > n_bits - 1) m = n_bits - 1;
+  d_fmt->n_bits = n_bits;
+  d_fmt->frac_bits = n_bits - 1 - m;
+}
+
+// ------------------------------------------------------------------------------------------
+// Quantizer (paper Sec. 2): q = saturate(round_half_away(x * 2^f)).  x * 2^f is exact in fp32;
+// the tie rule is applied on the exact fractional part (trunc + exact remainder), never on a
+// rounded sum.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int32_t quantize_f32(float x, float scale, int relu, int32_t qmin,
+                                                int32_t qmax, bool counted, Counts& c) {
+  float y = x * scale;
+  int32_t r;
+  if (y != y) {
+    r = 0;  // NaN
+  } else {
+    if (relu && y < 0.0f) y = 0.0f;
+    y = fminf(fmaxf(y, -131072.0f), 131072.0f);  // keeps every in-range value, saturates the rest
+    const float t = truncf(y);
+    const float frac = y - t;  // exact
+    r = (int32_t)t;
+    if (fabsf(frac) >= 0.5f) r += (y > 0.0f) ? 1 : -1;
+  }
+  if (r > qmax) {
+    r = qmax;
+    c.sat_pos += counted;
+  } else if (r < qmin) {
+    r = qmin;
+    c.sat_neg += counted;
+  }
+  c.zeros += (counted && r == 0);
+  return r;
+}
+
+__device__ __forceinline__ float scale_of(int32_t frac_bits) {
+  return __int_as_float((127 + frac_bits) << 23);
+}
+
+struct QuantOut {
+  uint32_t* hi;   // words of 4 bytes
+  uint32_t* lo;
+  uint2* q16;     // 4 int16
+  int32_t planes;
+};
+
+__device__ __forceinline__ void store4(const QuantOut& o, size_t word, int32_t q0, int32_t q1,
+                                       int32_t q2, int32_t q3) {
+  const uint32_t lo = (uint32_t)(q0 & 255) | ((uint32_t)(q1 & 255) << 8) |
+                      ((uint32_t)(q2 & 255) << 16) | ((uint32_t)(q3 & 255) << 24);
+  o.lo[word] = lo;
+  if (o.planes == 2) {
+    const uint32_t hi = (uint32_t)((q0 >> 8) & 255) | ((uint32_t)((q1 >> 8) & 255) << 8) |
+                        ((uint32_t)((q2 >> 8) & 255) << 16) | ((uint32_t)((q3 >> 8) & 255) << 24);
+    o.hi[word] = hi;
+  }
+  if (o.q16 != nullptr) {
+    uint2 v;
+    v.x = (uint32_t)(q0 & 0xffff) | ((uint32_t)(q1 & 0xffff) << 16);
+    v.y = (uint32_t)(q2 & 0xffff) | ((uint32_t)(q3 & 0xffff) << 16);
+    o.q16[word] = v;
+  }
+}
+
+// Dense rows (inner == c_stride): the tensor is one flat array; one float4 in, one 4-byte word
+// per plane out, four independent groups in flight per thread.
+__global__ void __launch_bounds__(256) quantize_flat_kernel(const float4* __restrict__ x, size_t n4,
+                                                            QuantOut out, int32_t frac_bits,
+                                                            const adaption_qfmt* __restrict__ d_fmt,
+                                                            int relu, int32_t qmin, int32_t qmax,
+                                                            adaption_stats* __restrict__ stats) {
+  if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
+  const float scale = scale_of(frac_bits);
+  Counts c;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * nthreads < n4; i += 4 * nthreads) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = __ldcs(x + i + u * nthreads);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      store4(out, i + u * nthreads, quantize_f32(v[u].x, scale, relu, qmin, qmax, true, c),
+             quantize_f32(v[u].y, scale, relu, qmin, qmax, true, c),
+             quantize_f32(v[u].z, scale, relu, qmin, qmax, true, c),
+             quantize_f32(v[u].w, scale, relu, qmin, qmax, true, c));
+    }
+  }
+  for (; i < n4; i += nthreads) {
+    const float4 v = __ldcs(x + i);
+    store4(out, i, quantize_f32(v.x, scale, relu, qmin, qmax, true, c),
+           quantize_f32(v.y, scale, relu, qmin, qmax, true, c),
+           quantize_f32(v.z, scale, relu, qmin, qmax, true, c),
+           quantize_f32(v.w, scale, relu, qmin, qmax, true, c));
+  }
+  if (stats != nullptr) flush_counts_warp(c, stats);
+}
+
+// Rows with channel padding (inner < c_stride) or unaligned input: one thread per group of four
+// stored channels; padding channels receive zeros and are not counted.
+__global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restrict__ x, size_t outer,
+                                                            int64_t inner, int64_t c_stride,
+                                                            QuantOut out, int32_t frac_bits,
+                                                            const adaption_qfmt* __restrict__ d_fmt,
+                                                            int relu, int32_t qmin, int32_t qmax,
+                                                            adaption_stats* __restrict__ stats) {
+  if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
+  const float scale = scale_of(frac_bits);
+  Counts c;
+  const int64_t groups_per_row = c_stride / 4;
+  const size_t total = outer * (size_t)groups_per_row;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += nthreads) {
+    const size_t row = g / groups_per_row;
+    const int64_t c0 = (int64_t)(g - row * groups_per_row) * 4;
+    int32_t q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const bool real = c0 + u < inner;
+      const float v = real ? __ldg(x + row * inner + c0 + u) : 0.0f;
+      q[u] = quantize_f32(v, scale, relu, qmin, qmax, real, c);
+    }
+    store4(out, g, q[0], q[1], q[2], q[3]);
+  }
+  if (stats != nullptr) flush_counts_warp(c, stats);
+}
+
+// Format conversion of a stored fixed-point tensor (LPAct on quantized values): optional ReLU,
+// rounding shift from f_in to f_out, saturation to the output width.
+__global__ void __launch_bounds__(256) requant_rows_kernel(const uint32_t* __restrict__ in_hi,
+                                                           const uint32_t* __restrict__ in_lo,
+                                                           int64_t in_stride, size_t outer,
+                                                           int64_t inner, int64_t c_stride, QuantOut out,
+                                                           int32_t in_frac_bits, int32_t out_frac_bits,
+                                                           const adaption_qfmt* __restrict__ d_fmt,
+                                                           RequantParams rq,
+                                                           adaption_stats* __restrict__ stats) {
+  if (d_fmt != nullptr) out_frac_bits = d_fmt->frac_bits;
+  rq.shift = in_frac_bits - out_frac_bits;
+  Counts c;
+  const int64_t groups_per_row = c_stride / 4;
+  const size_t total = outer * (size_t)groups_per_row;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += nthreads) {
+    const size_t row = g / groups_per_row;
+    const int64_t c0 = (int64_t)(g - row * groups_per_row) * 4;
+    uint32_t wlo = 0, whi = 0;
+    if (c0 < in_stride) {
+      const size_t word = (row * (size_t)in_stride + (size_t)c0) / 4;
+      wlo = __ldg(in_lo + word);
+      if (in_hi != nullptr) whi = __ldg(in_hi + word);
+    }
+    int32_t q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int32_t l = (wlo >> (8 * u)) & 255;
+      int32_t v;
+      if (in_hi != nullptr)
+        v = ((int32_t)(int8_t)((whi >> (8 * u)) & 255)) * 256 + l;
+      else
+        v = (int32_t)(int8_t)l;
+      const bool real = c0 + u < inner;
+      q[u] = requant_value(real ? (int64_t)v : 0, rq, real, c);
+    }
+    store4(out, g, q[0], q[1], q[2], q[3]);
+  }
+  if (stats != nullptr) flush_counts_warp(c, stats);
+}
+
+// ------------------------------------------------------------------------------------------
+// 2x2 / stride 2 max-pool on stored integers; 16 channels (one 16-byte vector per plane) per
+// thread.  Exact on the quantized values because the quantizer is monotone.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void max16(uint4& bh, uint4& bl, const uint4& h, const uint4& l, bool two) {
+  uint32_t* ph = reinterpret_cast<uint32_t*>(&bh);
+  uint32_t* pl = reinterpret_cast<uint32_t*>(&bl);
+  const uint32_t* qh = reinterpret_cast<const uint32_t*>(&h);
+  const uint32_t* ql = reinterpret_cast<const uint32_t*>(&l);
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    uint32_t oh = 0, ol = 0;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      int32_t cur, cand;
+      if (two) {
+        cur = ((int32_t)(int8_t)((ph[w] >> (8 * b)) & 255)) * 256 + (int32_t)((pl[w] >> (8 * b)) & 255);
+        cand = ((int32_t)(int8_t)((qh[w] >> (8 * b)) & 255)) * 256 + (int32_t)((ql[w] >> (8 * b)) & 255);
+      } else {
+        cur = (int32_t)(int8_t)((pl[w] >> (8 * b)) & 255);
+        cand = (int32_t)(int8_t)((ql[w] >> (8 * b)) & 255);
+      }
+      const int32_t m = cand > cur ? cand : cur;
+      ol |= (uint32_t)(m & 255) << (8 * b);
+      oh |= (uint32_t)((m >> 8) & 255) << (8 * b);
+    }
+    ph[w] = oh;
+    pl[w] = ol;
+  }
+}
+
+__global__ void __launch_bounds__(256) maxpool2x2_kernel(const uint4* __restrict__ in_hi,
+                                                         const uint4* __restrict__ in_lo,
+                                                         uint4* __restrict__ out_hi,
+                                                         uint4* __restrict__ out_lo,
+                                                         int16_t* __restrict__ out_q16, int N, int H,
+                                                         int W, int64_t in_vecs, int64_t out_vecs) {
+  // in_vecs / out_vecs: 16-byte vectors per pixel (c_stride / 16)
+  const int OH = H / 2, OW = W / 2;
+  const int64_t vecs = in_vecs < out_vecs ? in_vecs : out_vecs;
+  const size_t total = (size_t)N * OH * OW * (size_t)out_vecs;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  const bool two = in_hi != nullptr;
+  for (size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += nthreads) {
+    const int64_t v = (int64_t)(t % (size_t)out_vecs);
+    size_t pix = t / (size_t)out_vecs;
+    const int ow = (int)(pix % OW);
+    pix /= OW;
+    const int oh = (int)(pix % OH);
+    const int n = (int)(pix / OH);
+    uint4 bh = make_uint4(0, 0, 0, 0), bl = make_uint4(0, 0, 0, 0);
+    if (v < vecs) {
+      const size_t p00 = (((size_t)n * H + 2 * oh) * W + 2 * ow) * (size_t)in_vecs + (size_t)v;
+      const size_t offs[4] = {p00, p00 + (size_t)in_vecs, p00 + (size_t)W * in_vecs,
+                              p00 + (size_t)W * in_vecs + (size_t)in_vecs};
+      uint4 h[4], l[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        l[k] = __ldg(in_lo + offs[k]);
+        h[k] = two ? __ldg(in_hi + offs[k]) : make_uint4(0, 0, 0, 0);
+      }
+      bh = h[0];
+      bl = l[0];
+#pragma unroll
+      for (int k = 1; k < 4; ++k) max16(bh, bl, h[k], l[k], two);
+    }
+    out_lo[t] = bl;
+    if (two) out_hi[t] = bh;
+    if (out_q16 != nullptr) {
+      const uint32_t* ph = reinterpret_cast<const uint32_t*>(&bh);
+      const uint32_t* pl = reinterpret_cast<const uint32_t*>(&bl);
+      int16_t* dst = out_q16 + t * 16;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const int32_t l8 = (pl[e / 4] >> (8 * (e % 4))) & 255;
+        dst[e] = two ? (int16_t)(((int32_t)(int8_t)((ph[e / 4] >> (8 * (e % 4))) & 255)) * 256 + l8)
+                     : (int16_t)(int8_t)l8;
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+int check_qtensor_in(const adaption_qtensor& t, int64_t inner) {
+  if (!fmt_ok(t.fmt)) return ADAPTION_ERR_INVALID_ARG;
+  if (t.lo == nullptr) return ADAPTION_ERR_INVALID_ARG;
+  if (t.fmt.n_bits > 8 && t.hi == nullptr) return ADAPTION_ERR_INVALID_ARG;
+  if (t.c_stride < inner || (t.c_stride % 16) != 0) return ADAPTION_ERR_INVALID_ARG;
+  if (!aligned16(t.lo) || !aligned16(t.hi)) return ADAPTION_ERR_ALIGNMENT;
+  return ADAPTION_OK;
+}
+
+int check_qtensor_out(const adaption_qtensor& t, int64_t inner) {
+  int rc = check_qtensor_in(t, inner);
+  if (rc != ADAPTION_OK) return rc;
+  if (t.q16 != nullptr && !aligned16(t.q16)) return ADAPTION_ERR_ALIGNMENT;
+  return ADAPTION_OK;
+}
+
+static QuantOut quant_out_of(const adaption_qtensor& t) {
+  QuantOut o;
+  o.planes = t.fmt.n_bits > 8 ? 2 : 1;
+  o.hi = o.planes == 2 ? reinterpret_cast<uint32_t*>(t.hi) : nullptr;
+  o.lo = reinterpret_cast<uint32_t*>(t.lo);
+  o.q16 = reinterpret_cast<uint2*>(t.q16);
+  return o;
+}
+
+int quantize_impl(const float* d_x, size_t outer, size_t inner, const adaption_qtensor& out,
+                  const adaption_qfmt* d_fmt, int32_t relu, int32_t rounding, adaption_stats* d_stats,
+                  cudaStream_t stream) {
+  if (rounding == ADAPTION_ROUND_STOCHASTIC) return ADAPTION_ERR_UNSUPPORTED;
+  if (rounding != ADAPTION_ROUND_DETERMINISTIC) return ADAPTION_ERR_INVALID_ARG;
+  int rc = check_qtensor_out(out, (int64_t)inner);
+  if (rc != ADAPTION_OK) return rc;
+  if (outer == 0 || inner == 0) return ADAPTION_OK;
+  if (d_x == nullptr) return ADAPTION_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_x) & 3u) != 0) return ADAPTION_ERR_ALIGNMENT;
+  const int32_t qmin = -(1 << (out.fmt.n_bits - 1)), qmax = (1 << (out.fmt.n_bits - 1)) - 1;
+  const QuantOut qo = quant_out_of(out);
+  if ((int64_t)inner == out.c_stride && aligned16(d_x)) {
+    const size_t n4 = outer * inner / 4;
+    const int grid = stream_grid((n4 + 3) / 4, 256, 8);
+    quantize_flat_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const float4*>(d_x), n4, qo,
+                                                   out.fmt.frac_bits, d_fmt, relu, qmin, qmax, d_stats);
+  } else {
+    const size_t groups = outer * (size_t)(out.c_stride / 4);
+    const int grid = stream_grid(groups, 256, 8);
+    quantize_rows_kernel<<<grid, 256, 0, stream>>>(d_x, outer, (int64_t)inner, out.c_stride, qo,
+                                                   out.fmt.frac_bits, d_fmt, relu, qmin, qmax, d_stats);
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+int requant_impl(const adaption_qtensor& in, size_t outer, size_t inner, int32_t relu,
+                 const adaption_qtensor& out, const adaption_qfmt* d_fmt, int32_t rounding,
+                 adaption_stats* d_stats, cudaStream_t stream) {
+  if (rounding == ADAPTION_ROUND_STOCHASTIC) return ADAPTION_ERR_UNSUPPORTED;
+  if (rounding != ADAPTION_ROUND_DETERMINISTIC) return ADAPTION_ERR_INVALID_ARG;
+  int rc = check_qtensor_in(in, (int64_t)inner);
+  if (rc != ADAPTION_OK) return rc;
+  rc = check_qtensor_out(out, (int64_t)inner);
+  if (rc != ADAPTION_OK) return rc;
+  if (outer == 0 || inner == 0) return ADAPTION_OK;
+  RequantParams rq = make_requant(in.fmt.frac_bits, out.fmt, relu);
+  const size_t groups = outer * (size_t)(out.c_stride / 4);
+  const int grid = stream_grid(groups, 256, 8);
+  requant_rows_kernel<<<grid, 256, 0, stream>>>(
+      in.fmt.n_bits > 8 ? reinterpret_cast<const uint32_t*>(in.hi) : nullptr,
+      reinterpret_cast<const uint32_t*>(in.lo), in.c_stride, outer, (int64_t)inner, out.c_stride,
+      quant_out_of(out), in.fmt.frac_bits, out.fmt.frac_bits, d_fmt, rq, d_stats);
+  return cuda_status(cudaGetLastError());
+}
+
+int measure_range_impl(const float* d_x, size_t numel, int32_t n_bits, float* d_max_abs,
+                       adaption_qfmt* d_fmt_out, cudaStream_t stream) {
+  if (n_bits < 1 || n_bits > 16 || d_max_abs == nullptr) return ADAPTION_ERR_INVALID_ARG;
+  if (numel > 0 && d_x == nullptr) return ADAPTION_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_x) & 3u) != 0 || (reinterpret_cast<uintptr_t>(d_max_abs) & 3u) != 0)
+    return ADAPTION_ERR_ALIGNMENT;
+  if (numel > 0) {
+    size_t head = ((16 - (reinterpret_cast<uintptr_t>(d_x) & 15u)) & 15u) / 4;
+    if (head > numel) head = numel;
+    const size_t n4 = (numel - head) / 4;
+    int grid = stream_grid((n4 + 3) / 4 + 4, 256, 8);
+    range_max_abs_kernel<<<grid, 256, 0, stream>>>(d_x, numel, head, n4, d_max_abs);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return ADAPTION_ERR_CUDA;
+  }
+  if (d_fmt_out != nullptr) choose_fmt_kernel<<<1, 1, 0, stream>>>(d_max_abs, n_bits, d_fmt_out);
+  return cuda_status(cudaGetLastError());
+}
+
+int maxpool_impl(const adaption_qtensor& x, int32_t N, int32_t H, int32_t W, int32_t C,
+                 const adaption_qtensor& y, cudaStream_t stream) {
+  if (N < 0 || H < 0 || W < 0 || C < 0 || (H & 1) || (W & 1)) return ADAPTION_ERR_INVALID_ARG;
+  int rc = check_qtensor_in(x, C);
+  if (rc != ADAPTION_OK) return rc;
+  rc = check_qtensor_out(y, C);
+  if (rc != ADAPTION_OK) return rc;
+  if (x.fmt.n_bits != y.fmt.n_bits || x.fmt.frac_bits != y.fmt.frac_bits) return ADAPTION_ERR_INVALID_ARG;
+  const size_t total = (size_t)N * (H / 2) * (W / 2) * (size_t)(y.c_stride / 16);
+  if (total == 0) return ADAPTION_OK;
+  const bool two = x.fmt.n_bits > 8;
+  const int grid = stream_grid(total, 256, 8);
+  maxpool2x2_kernel<<<grid, 256, 0, stream>>>(
+      two ? reinterpret_cast<const uint4*>(x.hi) : nullptr, reinterpret_cast<const uint4*>(x.lo),
+      two ? reinterpret_cast<uint4*>(y.hi) : nullptr, reinterpret_cast<uint4*>(y.lo), y.q16, N, H, W,
+      x.c_stride / 16, y.c_stride / 16);
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace adaption

@@ -1,0 +1,267 @@
+"""Host-side orchestration of a stack of low-precision layers on one GPU.
+
+Only sequencing, buffer ownership and format bookkeeping live here; every step of the path
+(range measurement, quantization, convolution / inner product with fused bias + ReLU +
+requantization, pooling) is a call into the CUDA library through ``binding``.
+
+Workflow (paper Sec. 2.1): ``calibrate`` runs a batch through the stack and fixes one decimal
+point per layer from the measured ranges; ``forward`` then runs with those fixed formats and
+never synchronises with the host.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def act_c_stride(c: int) -> int:
+    """Channel pitch of activation / weight planes: a multiple of 32 so that every layer can take
+    the tensor-core path."""
+    return B.pad_to(c, 32)
+
+
+@dataclass
+class _Layer:
+    type: str
+    name: str = ""
+    relu: bool = True
+    # geometry
+    N: int = 0
+    H: int = 0
+    W: int = 0
+    C: int = 0
+    K: int = 0
+    R: int = 0
+    pad: int = 0
+    stride: int = 1
+    OH: int = 0
+    OW: int = 0
+    ip_k: int = 0            # reduction length of an inner product (padded flatten)
+    # buffers
+    w_f32: torch.Tensor | None = None
+    b_f32: torch.Tensor | None = None
+    w: B.QTensor | None = None
+    b: B.QTensor | None = None
+    w_fmt_dev: torch.Tensor | None = None
+    w_max_dev: torch.Tensor | None = None
+    y: B.QTensor | None = None
+    stats: torch.Tensor | None = None
+    workspace: torch.Tensor | None = None
+    shape: object = None
+    macs: int = 0
+    extra: dict = field(default_factory=dict)
+
+
+class LPNetwork:
+    def __init__(self, params: list[dict], batch: int, in_hw: tuple[int, int], in_c: int, n_bits: int,
+                 algo: int = B.ALGO_AUTO, keep_q16: bool = False, device="cuda"):
+        self.n_bits = n_bits
+        self.algo = algo
+        self.device = device
+        self.batch = batch
+        self.in_h, self.in_w = in_hw
+        self.in_c = in_c
+        self.keep_q16 = keep_q16
+        self.layers: list[_Layer] = []
+        self.calibrated = False
+        self.launches_per_forward = 0
+
+        self.x_fmt_dev = torch.zeros(2, dtype=torch.int32, device=device)
+        self.x_max_dev = torch.zeros(1, dtype=torch.float32, device=device)
+        self.x_stats = B.new_stats(device)
+        self.xq = B.QTensor.empty(batch * self.in_h * self.in_w, in_c, n_bits, 0, act_c_stride(in_c),
+                                  keep_q16, device)
+        h, w, c, cs = self.in_h, self.in_w, in_c, self.xq.c_stride
+        flat = False
+        for p in params:
+            L = _Layer(p["type"], p.get("name", ""))
+            if p["type"] == "pool":
+                L.N, L.H, L.W, L.C = batch, h, w, c
+                h, w = h // 2, w // 2
+                L.y = B.QTensor.empty(batch * h * w, c, n_bits, 0, cs, keep_q16, device)
+            elif p["type"] == "conv":
+                K, R, S, Cin = p["w"].shape
+                assert Cin == c and R == S and not flat
+                L.N, L.H, L.W, L.C, L.K, L.R = batch, h, w, c, K, R
+                L.pad, L.stride, L.relu = p["pad"], p["stride"], p["relu"]
+                L.OH = (h + 2 * L.pad - R) // L.stride + 1
+                L.OW = (w + 2 * L.pad - S) // L.stride + 1
+                L.shape = B.conv_shape(batch, h, w, c, K, R, S, L.pad, L.stride)
+                L.w_f32 = torch.from_numpy(np.ascontiguousarray(p["w"])).to(device)
+                L.w = B.QTensor.empty(K * R * S, c, n_bits, 0, cs, False, device)
+                L.macs = batch * L.OH * L.OW * K * R * S * c
+                h, w, c = L.OH, L.OW, K
+                cs = act_c_stride(K)
+                L.y = B.QTensor.empty(batch * h * w, K, n_bits, 0, cs, keep_q16, device)
+            elif p["type"] == "ip":
+                O, Kin = p["w"].shape
+                L.relu = p["relu"]
+                if not flat:
+                    assert Kin == h * w * c
+                    # weights follow the padded NHWC flatten of the previous activation
+                    L.ip_k = h * w * cs
+                    wsrc = np.ascontiguousarray(p["w"]).reshape(O * h * w, c)
+                    L.w = B.QTensor.empty(O * h * w, c, n_bits, 0, cs, False, device)
+                    L.extra["w_view"] = (O, L.ip_k)
+                    flat = True
+                else:
+                    assert Kin == c
+                    L.ip_k = cs
+                    wsrc = np.ascontiguousarray(p["w"])
+                    L.w = B.QTensor.empty(O, c, n_bits, 0, cs, False, device)
+                    L.extra["w_view"] = (O, cs)
+                L.w_f32 = torch.from_numpy(wsrc).to(device)
+                L.N, L.C, L.K = batch, Kin, O
+                L.macs = batch * Kin * O
+                h, w, c = 1, 1, O
+                cs = B.pad_to(O, 16)
+                L.y = B.QTensor.empty(batch, O, n_bits, 0, cs, keep_q16, device)
+            else:
+                raise ValueError(p["type"])
+            if L.type in ("conv", "ip"):
+                L.b_f32 = torch.from_numpy(np.ascontiguousarray(p["b"])).to(device)
+                L.b = B.QTensor.empty(1, L.K, n_bits, 0, None, True, device)
+                L.w_fmt_dev = torch.zeros(2, dtype=torch.int32, device=device)
+                L.w_max_dev = torch.zeros(1, dtype=torch.float32, device=device)
+                L.stats = B.new_stats(device)
+            self.layers.append(L)
+        self.total_macs = sum(L.macs for L in self.layers)
+
+    # ------------------------------------------------------------------ parameters
+    def quantize_params(self, measure: bool = True):
+        """Weights and biases -> fixed point (paper Sec. 2.1: quantized in the forward pass).  With
+        ``measure`` the decimal point of each layer's weights is taken from max|w| on the device."""
+        for L in self.layers:
+            if L.type not in ("conv", "ip"):
+                continue
+            if measure:
+                L.w_max_dev.zero_()
+                B.adaption_measure_range(L.w_f32, self.n_bits, L.w_max_dev, L.w_fmt_dev)
+                B.adaption_quantize(L.w_f32, L.w.outer, L.w.inner, L.w, L.w_fmt_dev)
+                B.adaption_quantize(L.b_f32, 1, L.K, L.b, L.w_fmt_dev)
+            else:
+                B.adaption_quantize(L.w_f32, L.w.outer, L.w.inner, L.w)
+                B.adaption_quantize(L.b_f32, 1, L.K, L.b)
+        if measure:
+            for L in self.layers:
+                if L.type in ("conv", "ip"):
+                    f = int(L.w_fmt_dev.cpu()[1])
+                    L.w.frac_bits = f
+                    L.b.frac_bits = f
+
+    # ------------------------------------------------------------------ one layer
+    def _workspace(self, L: _Layer, x: B.QTensor) -> torch.Tensor | None:
+        if L.type == "conv":
+            need = B.adaption_lp_conv_workspace_bytes(L.shape, x.fmt(), L.w.fmt(), x.c_stride, self.algo)
+        else:
+            need = B.adaption_lp_ip_workspace_bytes(L.N, L.ip_k, L.K, x.fmt(), L.w.fmt(), self.algo)
+        if need == 0:
+            return None
+        if L.workspace is None or L.workspace.numel() < need:
+            L.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return L.workspace
+
+    def _run_layer(self, L: _Layer, x: B.QTensor, mode: int) -> B.QTensor:
+        if L.type == "pool":
+            L.y.frac_bits = x.frac_bits
+            B.adaption_maxpool2x2(x, L.N, L.H, L.W, L.C, L.y)
+            return L.y
+        ws = self._workspace(L, x)
+        y = L.y if mode == B.MODE_REQUANT else None
+        if L.type == "conv":
+            B.adaption_lp_conv_fwd(L.shape, x, L.w, L.b.q16, L.b.frac_bits, L.relu, mode, self.algo, y,
+                                   L.stats, ws)
+        else:
+            xin = x.reshaped(L.N, L.ip_k, L.ip_k)
+            O, kp = L.extra["w_view"]
+            win = L.w.reshaped(O, kp, kp)
+            B.adaption_lp_ip_fwd(L.N, L.ip_k, L.K, xin, win, L.b.q16, L.b.frac_bits, L.relu, mode,
+                                 self.algo, y, L.stats, ws)
+        return L.y
+
+    # ------------------------------------------------------------------ calibration
+    def calibrate(self, x_f32: torch.Tensor, x_fmt: tuple[int, int] | None = None):
+        """Run one batch layer by layer, measuring each layer's range on it and fixing its decimal
+        point (paper Sec. 2.1, 2.3).  Returns the per-layer records (formats, counters, ranges)."""
+        self.quantize_params(measure=True)
+        rec = []
+        self.x_stats.zero_()
+        if x_fmt is None:
+            self.x_max_dev.zero_()
+            B.adaption_measure_range(x_f32, self.n_bits, self.x_max_dev, self.x_fmt_dev)
+            self.xq.frac_bits = int(self.x_fmt_dev.cpu()[1])
+        else:
+            assert x_fmt[0] == self.n_bits
+            self.xq.frac_bits = x_fmt[1]
+        B.adaption_quantize(x_f32, self.xq.outer, self.xq.inner, self.xq, None, B.ROUND_DETERMINISTIC,
+                            self.x_stats)
+        rec.append({"type": "input", "frac_bits": self.xq.frac_bits, "stats": B.read_stats(self.x_stats)})
+        a = self.xq
+        for L in self.layers:
+            if L.type == "pool":
+                a = self._run_layer(L, a, B.MODE_REQUANT)
+                rec.append({"type": "pool", "frac_bits": a.frac_bits})
+                continue
+            L.stats.zero_()
+            self._run_layer(L, a, B.MODE_RANGE)
+            st = B.read_stats(L.stats)
+            if st.status != 0:
+                raise B.AdaptionError(st.status, f"layer {L.name} (range)")
+            F = a.frac_bits + L.w.frac_bits
+            L.y.frac_bits = B.adaption_choose_frac_bits_from_acc(int(st.max_abs_acc), F, self.n_bits)
+            L.stats.zero_()
+            a = self._run_layer(L, a, B.MODE_REQUANT)
+            st2 = B.read_stats(L.stats)
+            if st2.status != 0:
+                raise B.AdaptionError(st2.status, f"layer {L.name}")
+            rec.append({"type": L.type, "name": L.name, "frac_bits": L.y.frac_bits,
+                        "w_frac_bits": L.w.frac_bits, "max_abs_acc": int(st.max_abs_acc),
+                        "acc_frac_bits": F, "stats": st2})
+        self.calibrated = True
+        return rec
+
+    # ------------------------------------------------------------------ inference
+    def forward(self, x_f32: torch.Tensor, requantize_params: bool = True, measure_input: bool = True):
+        """One forward pass with the calibrated formats; enqueues work only (no host sync).
+        Returns the output QTensor and the number of kernel launches issued."""
+        assert self.calibrated
+        launches = 0
+        if measure_input:
+            # range of the incoming batch (monitoring; the calibrated input format stays in force)
+            B.adaption_measure_range(x_f32, self.n_bits, self.x_max_dev, self.x_fmt_dev)
+            launches += 2
+        B.adaption_quantize(x_f32, self.xq.outer, self.xq.inner, self.xq, None, B.ROUND_DETERMINISTIC,
+                            self.x_stats)
+        launches += 1
+        if requantize_params:
+            self.quantize_params(measure=False)
+            launches += 2 * sum(1 for L in self.layers if L.type in ("conv", "ip"))
+        a = self.xq
+        for L in self.layers:
+            a = self._run_layer(L, a, B.MODE_REQUANT)
+            launches += 1
+            if L.workspace is not None and L.type != "pool":
+                launches += 1  # split-K finalize
+        self.launches_per_forward = launches
+        return a, launches
+
+    def zero_stats(self):
+        self.x_stats.zero_()
+        for L in self.layers:
+            if L.stats is not None:
+                L.stats.zero_()
+
+    def layer_stats(self):
+        out = []
+        for L in self.layers:
+            if L.stats is not None:
+                st = B.read_stats(L.stats)
+                total = L.y.outer * L.y.inner
+                out.append({"name": L.name, "zeros": int(st.zeros), "sat_pos": int(st.sat_pos),
+                            "sat_neg": int(st.sat_neg), "total": total, "status": int(st.status),
+                            "frac_bits": L.y.frac_bits})
+        return out

@@ -1,0 +1,255 @@
+"""GPU parity of LPConvolution / LPInnerProduct (both kernels: plain integer and tensor core)
+against the CPU oracle, bit-exact, through the C ABI.  Shapes span several 128-row tiles and
+ragged tails in M, N and K."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import reference as orc
+from paper_1711_04713_b200 import binding as B
+from tests.util import dev, from_qtensor, q16_of, stats_tuple, to_qtensor
+
+pytestmark = pytest.mark.gpu
+
+
+def _rand_q(rng, shape, n_bits, zero_frac=0.0):
+    q = rng.integers(-(1 << (n_bits - 1)), 1 << (n_bits - 1), shape).astype(np.int16)
+    if zero_frac > 0:
+        q[rng.random(shape) < zero_frac] = 0
+    return q
+
+
+def _pick_f_out(acc, bq, fb, F, relu, n_out):
+    A = orc.epilogue_range(acc, bq, fb, F, relu)
+    return A, n_out - 1 - orc.int_bits_from_acc(A, F, n_out)
+
+
+def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, algo, with_bias=True,
+                  extreme=False, f_out=None):
+    cs = B.pad_to(Cin, 32)
+    xq = _rand_q(rng, (N, H, W, Cin), nx, 0.4)
+    wq = _rand_q(rng, (K, R, R, Cin), nw)
+    if extreme:   # drive every byte plane to its extremes
+        xq[:] = np.where(rng.random(xq.shape) < 0.5, -(1 << (nx - 1)), (1 << (nx - 1)) - 1)
+        wq[:] = np.where(rng.random(wq.shape) < 0.5, -(1 << (nw - 1)), (1 << (nw - 1)) - 1)
+    fx, fw = nx - 3, nw - 1
+    bq = _rand_q(rng, (K,), nw) if with_bias else None
+    acc = orc.conv_acc(xq, wq, (pad, pad), (stride, stride))
+    F = fx + fw
+    A, f_auto = _pick_f_out(acc, bq, fw, F, relu, n_out)
+    f_out = f_auto if f_out is None else f_out
+    want, cnt = orc.epilogue(acc, bq, fw, F, relu, n_out, f_out)
+    OH, OW = acc.shape[1], acc.shape[2]
+
+    x = to_qtensor(xq.reshape(-1, Cin), nx, fx, cs)
+    w = to_qtensor(wq.reshape(-1, Cin), nw, fw, cs)
+    ycs = B.pad_to(K, 32)
+    y = B.QTensor.empty(N * OH * OW, K, n_out, f_out, ycs, with_q16=True)
+    y.lo.fill_(0x3C)
+    if y.hi is not None:
+        y.hi.fill_(0x3C)
+    shp = B.conv_shape(N, H, W, Cin, K, R, R, pad, stride)
+    bias_dev = dev(bq) if with_bias else None
+    need = B.adaption_lp_conv_workspace_bytes(shp, x.fmt(), w.fmt(), cs, algo)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+    st = B.new_stats()
+    B.adaption_lp_conv_fwd(shp, x, w, bias_dev, fw, relu, B.MODE_RANGE, algo, None, st, ws)
+    s = B.read_stats(st)
+    assert s.status == 0
+    assert int(s.max_abs_acc) == A
+    assert B.adaption_choose_frac_bits_from_acc(A, F, n_out) == f_auto
+    st = B.new_stats()
+    B.adaption_lp_conv_fwd(shp, x, w, bias_dev, fw, relu, B.MODE_REQUANT, algo, y, st, ws)
+    s = B.read_stats(st)
+    assert s.status == 0
+    got = from_qtensor(y).reshape(want.shape)
+    bad = np.argwhere(got != want)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}: got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}"
+    assert np.array_equal(q16_of(y).reshape(want.shape), want)
+    assert y.padding_is_zero()
+    assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+
+
+def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out=None):
+    xq = _rand_q(rng, (Bsz, K), nx, 0.4)
+    wq = _rand_q(rng, (O, K), nw)
+    fx, fw = nx - 2, nw - 1
+    bq = _rand_q(rng, (O,), nw) if with_bias else None
+    acc = orc.ip_acc(xq, wq)
+    F = fx + fw
+    A, f_auto = _pick_f_out(acc, bq, fw, F, relu, n_out)
+    f_out = f_auto if f_out is None else f_out
+    want, cnt = orc.epilogue(acc, bq, fw, F, relu, n_out, f_out)
+    x = to_qtensor(xq, nx, fx)
+    w = to_qtensor(wq, nw, fw)
+    y = B.QTensor.empty(Bsz, O, n_out, f_out, None, with_q16=True)
+    y.lo.fill_(0x3C)
+    bias_dev = dev(bq) if with_bias else None
+    need = B.adaption_lp_ip_workspace_bytes(Bsz, K, O, x.fmt(), w.fmt(), algo)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+    st = B.new_stats()
+    B.adaption_lp_ip_fwd(Bsz, K, O, x, w, bias_dev, fw, relu, B.MODE_RANGE, algo, None, st, ws)
+    s = B.read_stats(st)
+    assert s.status == 0 and int(s.max_abs_acc) == A
+    st = B.new_stats()
+    B.adaption_lp_ip_fwd(Bsz, K, O, x, w, bias_dev, fw, relu, B.MODE_REQUANT, algo, y, st, ws)
+    s = B.read_stats(st)
+    assert s.status == 0
+    got = from_qtensor(y)
+    bad = np.argwhere(got != want)
+    assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
+    assert np.array_equal(q16_of(y), want)
+    assert y.padding_is_zero()
+    assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+    return need
+
+
+# ------------------------------------------------------------------ plain integer kernels
+@pytest.mark.parametrize("case", [
+    # N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu
+    (2, 7, 6, 5, 4, 3, 1, 1, 16, 16, 16, True), (1, 9, 9, 3, 7, 5, 0, 1, 16, 16, 16, False),
+    (2, 8, 10, 4, 3, 3, 1, 2, 8, 8, 8, True), (1, 5, 5, 20, 50, 5, 0, 1, 16, 16, 16, True),
+    (1, 6, 6, 9, 5, 1, 0, 1, 16, 8, 12, False), (2, 6, 6, 16, 8, 3, 2, 1, 4, 4, 4, True),
+    (1, 8, 8, 33, 17, 3, 1, 1, 12, 16, 8, True),
+])
+def test_conv_direct(case):
+    N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu = case
+    run_conv_case(np.random.default_rng(sum(case)), N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu,
+                  B.ALGO_DIRECT)
+
+
+@pytest.mark.parametrize("case", [(8, 800, 500, 16, 16, 16, True), (8, 500, 10, 16, 16, 16, False),
+                                  (3, 17, 5, 8, 8, 8, True), (5, 64, 33, 16, 8, 16, False),
+                                  (1, 1, 1, 16, 16, 16, False)])
+def test_ip_direct(case):
+    Bsz, K, O, nx, nw, n_out, relu = case
+    run_ip_case(np.random.default_rng(sum(case)), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_DIRECT)
+
+
+def test_direct_without_bias_and_fixed_saturating_format():
+    rng = np.random.default_rng(3)
+    run_conv_case(rng, 1, 6, 6, 8, 6, 3, 1, 1, 16, 16, 16, False, B.ALGO_DIRECT, with_bias=False)
+    # a format with too few integer bits saturates on both sides; counters must agree
+    run_ip_case(rng, 6, 40, 12, 16, 16, 16, False, B.ALGO_DIRECT, f_out=15)
+    run_ip_case(rng, 6, 40, 12, 16, 16, 8, True, B.ALGO_DIRECT, f_out=7)
+
+
+# ------------------------------------------------------------------ tensor-core kernels
+TC_CONV = [
+    # N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu      (N*H*W*pitch >= 128 KiB)
+    (6, 20, 20, 64, 96, 3, 1, 1, 16, 16, 16, True),      # BK=64, ragged N tile, 18.75 M tiles
+    (2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True),    # BK=128
+    (2, 30, 30, 256, 64, 3, 1, 1, 16, 16, 16, False),    # two channel blocks per tap, BN=64
+    (8, 28, 28, 20, 50, 5, 0, 1, 16, 16, 16, True),      # valid 5x5, pitch 32 (BK=32), ragged N
+    (8, 32, 32, 3, 64, 3, 1, 1, 16, 16, 16, True),       # first-layer shape: 3 channels padded to 32
+    (4, 33, 31, 64, 130, 3, 1, 2, 16, 16, 16, True),     # stride 2, odd sizes, N spills into 2nd tile
+    (2, 40, 40, 64, 32, 1, 0, 1, 16, 16, 16, False),     # 1x1
+    (2, 24, 24, 128, 128, 3, 1, 1, 8, 8, 8, True),       # single int8 pass
+    (2, 24, 24, 128, 72, 3, 1, 1, 4, 4, 4, True),        # 4-bit operands in the int8 pass
+    (2, 24, 24, 128, 128, 3, 1, 1, 16, 8, 16, True),     # 16-bit activations x 8-bit weights
+    (2, 24, 24, 128, 128, 3, 1, 1, 8, 16, 12, False),    # 8-bit activations x 16-bit weights
+    (2, 24, 24, 128, 128, 3, 1, 1, 12, 12, 12, True),    # 12-bit operands in planes
+    (1, 64, 64, 32, 16, 3, 1, 1, 16, 16, 8, True),       # 16-bit in, 8-bit out, BN=32
+]
+
+
+@pytest.mark.parametrize("case", TC_CONV)
+def test_conv_tensor(case):
+    N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu = case
+    run_conv_case(np.random.default_rng(sum(case)), N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu,
+                  B.ALGO_TENSOR)
+
+
+def test_conv_tensor_extreme_operands():
+    # every operand at +-full scale: largest possible partial sums in all three accumulators
+    run_conv_case(np.random.default_rng(1), 1, 32, 32, 256, 128, 3, 1, 1, 16, 16, 16, False, B.ALGO_TENSOR,
+                  extreme=True)
+    run_conv_case(np.random.default_rng(2), 1, 32, 32, 256, 128, 3, 1, 1, 8, 8, 8, False, B.ALGO_TENSOR,
+                  extreme=True)
+
+
+TC_IP = [(8, 800, 500, 16, 16, 16, True), (70, 1000, 260, 16, 16, 16, False), (200, 4096, 100, 16, 16, 16, True),
+         (130, 256, 128, 8, 8, 8, True), (64, 1184, 96, 16, 8, 16, True), (3, 64, 10, 16, 16, 16, False),
+         (256, 512, 512, 12, 12, 12, True)]
+
+
+@pytest.mark.parametrize("case", TC_IP)
+def test_ip_tensor(case):
+    Bsz, K, O, nx, nw, n_out, relu = case
+    run_ip_case(np.random.default_rng(sum(case)), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_TENSOR)
+
+
+def test_ip_tensor_split_k_paths():
+    # long reduction with few output tiles: the library splits K and needs its workspace
+    need = run_ip_case(np.random.default_rng(11), 64, 25088, 256, 16, 16, 16, True, B.ALGO_TENSOR)
+    assert need == 64 * 256 * 8
+    # forcing other split factors gives the same bits
+    for splits in ("3", "7"):
+        os.environ["ADAPTION_TC_SPLITS"] = splits
+        try:
+            need = run_ip_case(np.random.default_rng(12), 40, 2048, 200, 16, 16, 16, False, B.ALGO_TENSOR)
+            assert need == 40 * 200 * 8
+            run_conv_case(np.random.default_rng(13), 2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True,
+                          B.ALGO_TENSOR)
+        finally:
+            del os.environ["ADAPTION_TC_SPLITS"]
+
+
+def test_workspace_too_small_is_rejected():
+    rng = np.random.default_rng(14)
+    xq, wq = _rand_q(rng, (64, 25088), 16), _rand_q(rng, (256, 25088), 16)
+    x, w = to_qtensor(xq, 16, 10), to_qtensor(wq, 16, 15)
+    y = B.QTensor.empty(64, 256, 16, 5)
+    st = B.new_stats()
+    with pytest.raises(B.AdaptionError) as e:
+        B.adaption_lp_ip_fwd(64, 25088, 256, x, w, None, 0, True, B.MODE_REQUANT, B.ALGO_TENSOR, y, st,
+                             torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == B.ERR_WORKSPACE
+
+
+def test_eight_bit_data_through_plane_path_equals_single_pass():
+    """Cross-path identity: 8-bit values stored as 16-bit planes (hi = sign extension) go through
+    the four-product path and must give the bits of the single int8 pass."""
+    rng = np.random.default_rng(15)
+    N, H, W, Cin, K = 4, 24, 24, 64, 64
+    xq, wq = _rand_q(rng, (N, H, W, Cin), 8, 0.3), _rand_q(rng, (K, 3, 3, Cin), 8)
+    shp = B.conv_shape(N, H, W, Cin, K, 3, 3, 1, 1)
+    outs = []
+    for nb in (8, 16):
+        x, w = to_qtensor(xq.reshape(-1, Cin), nb, 4, 64), to_qtensor(wq.reshape(-1, Cin), nb, 7, 64)
+        y = B.QTensor.empty(N * H * W, K, 16, 6, 64)
+        st = B.new_stats()
+        B.adaption_lp_conv_fwd(shp, x, w, None, 0, True, B.MODE_REQUANT, B.ALGO_TENSOR, y, st, None)
+        outs.append((from_qtensor(y), stats_tuple(st)))
+    assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+    want, _ = orc.epilogue(orc.conv_acc(xq, wq, (1, 1)), None, 0, 11, True, 16, 6)
+    assert np.array_equal(outs[0][0].reshape(want.shape), want)
+
+
+def test_one_by_one_conv_equals_inner_product_on_gpu():
+    rng = np.random.default_rng(16)
+    N, H, W, Cin, K = 2, 40, 40, 64, 48
+    xq, wq = _rand_q(rng, (N, H, W, Cin), 16, 0.3), _rand_q(rng, (K, 1, 1, Cin), 16)
+    x, w = to_qtensor(xq.reshape(-1, Cin), 16, 9, 64), to_qtensor(wq.reshape(-1, Cin), 16, 14, 64)
+    st = B.new_stats()
+    y1 = B.QTensor.empty(N * H * W, K, 16, 4, 64)
+    B.adaption_lp_conv_fwd(B.conv_shape(N, H, W, Cin, K, 1, 1, 0, 1), x, w, None, 0, False, B.MODE_REQUANT,
+                           B.ALGO_TENSOR, y1, st, None)
+    y2 = B.QTensor.empty(N * H * W, K, 16, 4, 64)
+    B.adaption_lp_ip_fwd(N * H * W, Cin, K, x, w, None, 0, False, B.MODE_REQUANT, B.ALGO_TENSOR, y2, st, None)
+    assert np.array_equal(from_qtensor(y1), from_qtensor(y2))
+
+
+def test_auto_falls_back_to_direct_for_small_or_odd_pitch():
+    rng = np.random.default_rng(17)
+    # pitch 48 is not a multiple of 32 and the tensor is tiny: AUTO must still be exact
+    run_conv_case(rng, 1, 6, 6, 8, 6, 3, 1, 1, 16, 16, 16, True, B.ALGO_AUTO)
+    run_ip_case(rng, 4, 20, 6, 16, 16, 16, True, B.ALGO_AUTO)
+    xq, wq = _rand_q(rng, (1, 4, 4, 8), 16), _rand_q(rng, (4, 3, 3, 8), 16)
+    x, w = to_qtensor(xq.reshape(-1, 8), 16, 9, 32), to_qtensor(wq.reshape(-1, 8), 16, 9, 32)
+    with pytest.raises(B.AdaptionError) as e:
+        B.adaption_lp_conv_fwd(B.conv_shape(1, 4, 4, 8, 4, 3, 3, 1, 1), x, w, None, 0, False, B.MODE_RANGE,
+                               B.ALGO_TENSOR, None, B.new_stats(), None)
+    assert e.value.status == B.ERR_UNSUPPORTED
