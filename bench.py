@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Benchmark of the low-precision forward path on B200.
+
+Workload: full VGG16 forward, 16-bit weights and activations, batch 64 per GPU, seeded synthetic
+input (N(0,1) images, He-normal weights), every decimal point fixed beforehand by range
+measurement on the batch.  One step = one forward pass of the batch through the whole path:
+range measurement of the input, LPAct of the input, quantization of all weights and biases,
+13 LPConvolution + 3 LPInnerProduct layers with fused bias / ReLU / requantization / zero
+counting, 5 max-pools.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--batch B] [--n-bits 16]
+
+Prints one JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of
+the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "effective fixed-point TOPS & images/s for VGG16 16-bit forward; % of INT8 peak"
+INT8_NOMINAL_TOPS = 4500.0          # dense INT8, datasheet
+NOMINAL_INT8_OVER_BF16 = 2.0        # nominal dense INT8 : bf16 ratio (4.5 : 2.25 POPS)
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_BF16_SUSTAINED = 1400.0
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_burst": float(p["bf16_tflops"]),
+                "bf16_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_burst": FALLBACK_BF16_TFLOPS, "bf16_sustained": FALLBACK_BF16_SUSTAINED,
+                "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = f"/tmp/adaption_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=self.fh, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, mx, pw, reasons = [], [], [], set()
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                    pw.append(float(f[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["sm_max_mhz"] = max(mx)
+            out["power_w_max"] = max(pw) if pw else None
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle on a bounded sample
+# ---------------------------------------------------------------------------------------------
+def oracle_sample_step(params, x_sample, formats, n_bits):
+    from oracle import reference as orc
+    t0 = time.perf_counter()
+    orc.run_network(params, x_sample, formats["input"], n_bits, fixed_formats=formats["layers"])
+    return time.perf_counter() - t0
+
+
+def oracle_formats(params, x_sample, n_bits):
+    """Formats fixed by a calibration pass of the oracle on the sample itself (untimed)."""
+    from oracle import reference as orc
+    rec = orc.run_network(params, x_sample, None, n_bits)
+    return {"input": (rec[0]["n_bits"], rec[0]["frac_bits"]),
+            "layers": [r["frac_bits"] for r in rec if r["type"] in ("conv", "ip")]}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import reference as orc
+    from paper_1711_04713_b200 import workloads as wl
+    params = wl.make_params(wl.vgg16_specs(), seed=0)
+    macs_img = wl.vgg16_macs_per_image()
+    sample_images = 1
+    x = wl.vgg16_input(sample_images, seed=0)
+    formats = oracle_formats(params, x, args.n_bits)
+    for _ in range(args.warmup):
+        oracle_sample_step(params, x, formats, args.n_bits)
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_sample_step(params, x, formats, args.n_bits)
+    ms = t / args.steps * 1e3
+    ips = sample_images / (ms / 1e3)
+    cores = orc.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": ips, "unit": "images/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": f"int{args.n_bits}", "data": "synthetic",
+        "effective_tops": 2.0 * macs_img * ips / 1e12,
+        "config": {"workload": f"VGG16 forward, {args.n_bits}-bit weights and activations (full stack); "
+                               f"each step = {sample_images} image through the CPU oracle",
+                   "global_batch": sample_images, "n_bits": args.n_bits},
+        "cpu_baseline": {"value": ips, "unit": "images/s", "cores": cores, "kind": "oracle",
+                         "sample": f"{sample_images} image(s) per step, whole VGG16 stack, fixed formats"},
+        "e2e": {"value": ips, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------------
+def run_gpu(args):
+    import torch
+
+    from paper_1711_04713_b200 import binding as B
+    from paper_1711_04713_b200 import build as bld
+    from paper_1711_04713_b200 import workloads as wl
+    from paper_1711_04713_b200.network import LPNetwork
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (no CPU fallback exists)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        bld.build_library()
+    if dist is not None:
+        dist.barrier()
+    B.load()
+    peaks = read_peaks()
+
+    # ---- workload: each rank owns its own batch of images (weak scaling, no data-path collective)
+    specs = wl.vgg16_specs()
+    params = wl.make_params(specs, seed=0)
+    batch = args.batch
+    x_host = torch.from_numpy(wl.vgg16_input(batch, seed=100 + rank).reshape(-1, 3)).pin_memory()
+    x_dev = x_host.cuda()
+    net = LPNetwork(params, batch, (224, 224), 3, args.n_bits)
+    del params
+    net.calibrate(x_dev)
+    macs_step = net.total_macs
+    torch.cuda.synchronize()
+
+    gemm_layers = [L for L in net.layers if L.type in ("conv", "ip")]
+    n_gemm = len(gemm_layers)
+
+    def step(timed_events=None):
+        """One forward pass of the batch; optional CUDA events around every layer-GEMM launch."""
+        B.adaption_measure_range(x_dev, net.n_bits, net.x_max_dev, net.x_fmt_dev)
+        B.adaption_lp_act(x_dev, None, net.xq.outer, net.xq.inner, False, net.xq, None,
+                          B.ROUND_DETERMINISTIC, net.x_stats)
+        net.quantize_params(measure=False)
+        a = net.xq
+        for L in net.layers:
+            if timed_events is not None and L.type != "pool":
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                a = net._run_layer(L, a, B.MODE_REQUANT)
+                e1.record()
+                timed_events.append((L, e0, e1))
+            else:
+                a = net._run_layer(L, a, B.MODE_REQUANT)
+        return a
+
+    # kernels of ours per step: range (2) + input LPAct (1) + weight/bias quantize (2 per layer)
+    # + one per layer (+1 finalize where K is split)
+    launches_step = 3 + 2 * n_gemm + len(net.layers) + sum(1 for L in gemm_layers if L.workspace is not None)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    net.zero_stats()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    events = []
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        out = step(events)
+    t1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    elapsed_ms = t0.elapsed_time(t1)
+    clocks = sampler.stop() if rank == 0 else {}
+    if dist is not None:
+        tt = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tt[0])
+    ms_per_step = elapsed_ms / args.steps
+    ips = world * batch / (ms_per_step / 1e3)
+    eff_tops = 2.0 * macs_step * world / (ms_per_step / 1e3) / 1e12
+
+    # ---- per-launch durations of the dominant kernel (the tensor-core layer GEMM), from the
+    #      events recorded inside the timed region
+    per_layer = {}
+    gemm_ms = 0.0
+    for L, e0, e1 in events:
+        d = e0.elapsed_time(e1)
+        per_layer.setdefault(L.name, []).append(d)
+        gemm_ms += d
+    gemm_launches = len(events)
+    gemm_ops = 2.0 * macs_step * args.steps                  # logical n-bit operations in those launches
+    achieved_tops = gemm_ops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
+    planes = 4.0 if args.n_bits > 8 else 1.0                  # int8 products per logical MAC
+    peak_int8 = peaks["bf16_sustained"] * NOMINAL_INT8_OVER_BF16
+    peak = peak_int8 / planes
+    roofline = {
+        "bound": "tensor", "kernel": "lp_gemm_kernel (all LPConvolution / LPInnerProduct launches)",
+        "achieved": achieved_tops, "peak": peak, "unit": "TFLOP/s", "frac": achieved_tops / peak,
+        "traffic": None,
+        "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']} x{NOMINAL_INT8_OVER_BF16:g} "
+                       f"(nominal INT8:bf16) / {planes:g} int8 products per {args.n_bits}-bit MAC",
+        "frac_of_burst": achieved_tops / (peaks["bf16_burst"] * NOMINAL_INT8_OVER_BF16 / planes),
+        "frac_of_nominal_int8": achieved_tops / (INT8_NOMINAL_TOPS / planes),
+        "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
+        "share_of_step": gemm_ms / elapsed_ms if world == 1 else None,
+    }
+    layer_table = {k: {"ms": statistics.mean(v)} for k, v in per_layer.items()}
+    for L in gemm_layers:
+        layer_table[L.name]["tops"] = 2.0 * L.macs / (layer_table[L.name]["ms"] / 1e3) / 1e12
+
+    stats = net.layer_stats()
+    sparsity = {s["name"]: round(s["zeros"] / max(s["total"], 1) / args.steps, 4) for s in stats}
+    sat = {s["name"]: [s["sat_pos"] // args.steps, s["sat_neg"] // args.steps] for s in stats}
+
+    # ---- end to end: host buffers in, host result out, copies inside the timed region
+    out_host_lo = torch.empty_like(out.lo, device="cpu").pin_memory()
+    out_host_hi = torch.empty_like(out.hi, device="cpu").pin_memory() if out.hi is not None else None
+    e2e_steps = max(3, min(args.steps, 10))
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        x_dev.copy_(x_host, non_blocking=True)
+        o = step()
+        out_host_lo.copy_(o.lo, non_blocking=True)
+        if out_host_hi is not None:
+            out_host_hi.copy_(o.hi, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tt = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt[0])
+    e2e_ips = world * batch / (e2e_ms / e2e_steps / 1e3)
+    h2d = x_host.numel() * 4
+    d2h = out.lo.numel() + (out.hi.numel() if out.hi is not None else 0)
+
+    bad = [s for s in net.layer_stats() if s["status"] != 0]
+    if bad:
+        raise RuntimeError(f"device-side timeout flagged in {bad}")
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- the oracle on the host cores, on a bounded sample of the same workload
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import reference as orc
+        params = wl.make_params(specs, seed=0)
+        xs = wl.vgg16_input(1, seed=100)
+        formats = oracle_formats(params, xs, args.n_bits)
+        t_one = oracle_sample_step(params, xs, formats, args.n_bits)
+        n_img = int(max(1, min(8, 12.0 / max(t_one, 1e-3))))
+        xs = wl.vgg16_input(n_img, seed=100)
+        t_s = oracle_sample_step(params, xs, formats, args.n_bits)
+        cpu_baseline = {"value": n_img / t_s, "unit": "images/s", "cores": orc.num_threads(), "kind": "oracle",
+                        "sample": f"{n_img} image(s) of the same VGG16 {args.n_bits}-bit forward "
+                                  f"(whole stack, fixed formats), {t_s:.1f} s",
+                        "effective_tops": 2.0 * wl.vgg16_macs_per_image() * n_img / t_s / 1e12}
+
+    line = {
+        "metric": METRIC, "value": ips, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": f"int{args.n_bits}", "data": "synthetic",
+        "effective_tops": eff_tops,
+        "pct_of_int8_peak": {"nominal_4500_div_planes": 100.0 * eff_tops / (INT8_NOMINAL_TOPS / planes),
+                             "measured_bf16_sustained_x2_div_planes": 100.0 * eff_tops / peak},
+        "config": {"workload": f"VGG16 full forward, {args.n_bits}-bit weights and activations, batch {batch} "
+                               "per GPU, 224x224x3 N(0,1) inputs, He-normal weights, per-layer decimal points "
+                               "from range measurement; step includes input range + LPAct and per-forward "
+                               "weight/bias quantization",
+                   "global_batch": batch * world, "n_bits": args.n_bits,
+                   "l2": "activations and weights touched per step (about 2.5 GB) exceed the 126 MB L2; "
+                         "no explicit flush"},
+        "clocks": clocks, "gpu_launches": launches_step * args.steps,
+        "e2e": {"value": e2e_ips, "unit": "images/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "layers": layer_table, "sparsity": sparsity, "saturations": sat,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--n-bits", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
