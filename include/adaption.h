@@ -143,6 +143,31 @@ ADAPTION_API int adaption_lp_ip_fwd(int64_t B, int64_t K, int64_t O, adaption_qt
                        int32_t mode, int32_t algo, adaption_qtensor y, adaption_stats* d_stats,
                        void* d_workspace, size_t workspace_bytes, void* stream);
 
+/* No counterpart in the paper: a convenience for callers that cannot allocate device memory.
+ * Same operation, arguments, results and status codes as adaption_lp_ip_fwd, but the split-K
+ * workspace is not passed in: it is a fixed array of ADAPTION_STATIC_WORKSPACE_BYTES inside the
+ * library image (every GPU that loads the library carries it until the process exits).  It is
+ * meant for code that must not call cudaMalloc where it runs: plug-ins handed a fixed memory
+ * arena by their host application, or real-time loops in which an allocation would stall or
+ * synchronise the device.  The call itself allocates and frees nothing.
+ *   - Limit: if the shape needs more workspace than the array holds (the amount
+ *     adaption_lp_ip_workspace_bytes reports, i.e. 8 bytes per output element when the reduction
+ *     is split), the call returns ADAPTION_ERR_WORKSPACE and launches nothing; use
+ *     adaption_lp_ip_fwd with your own buffer for such shapes.
+ *   - The first call on each device looks the array's device address up (one runtime query with
+ *     that device current; a failure is reported as ADAPTION_ERR_CUDA).  Make that first call
+ *     before any stream capture begins.
+ *   - All calls on a device share the one array and it keeps the previous call's contents; each
+ *     call clears the part it uses before accumulating.  Two calls whose GPU work can overlap
+ *     (different streams, or different host threads on the same device) race on it: run them on
+ *     one stream or order them yourself. */
+#define ADAPTION_STATIC_WORKSPACE_BYTES (4u << 20)
+ADAPTION_API int adaption_lp_ip_fwd_static_ws(int64_t B, int64_t K, int64_t O, adaption_qtensor x,
+                                              adaption_qtensor w, const int16_t* d_bias_q,
+                                              int32_t bias_frac_bits, int32_t relu, int32_t mode,
+                                              int32_t algo, adaption_qtensor y, adaption_stats* d_stats,
+                                              void* stream);
+
 /* The 2x2, stride-2 max pooling that sits between the low-precision layers of the networks
  * the paper studies (VGG16; Table 1, "Pooling").  Works on the stored integers, same format
  * in and out; H and W even.  x is [N][H][W][C], y is [N][H/2][W/2][C]. */

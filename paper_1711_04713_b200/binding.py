@@ -46,7 +46,7 @@ STATS_BYTES = C.sizeof(adaption_stats)
 EXPORTS = [
     "adaption_measure_range", "adaption_quantize", "adaption_lp_act",
     "adaption_lp_conv_workspace_bytes", "adaption_lp_conv_fwd", "adaption_lp_ip_workspace_bytes",
-    "adaption_lp_ip_fwd", "adaption_maxpool2x2", "adaption_choose_frac_bits_from_acc",
+    "adaption_lp_ip_fwd", "adaption_lp_ip_fwd_static_ws", "adaption_maxpool2x2", "adaption_choose_frac_bits_from_acc",
     "adaption_status_string",
 ]
 
@@ -82,6 +82,8 @@ def load(path: str | None = None):
     lib.adaption_lp_ip_workspace_bytes.restype = SZ
     lib.adaption_lp_ip_fwd.argtypes = [I64, I64, I64, adaption_qtensor, adaption_qtensor, P, I32, I32, I32,
                                        I32, adaption_qtensor, P, P, SZ, P]
+    lib.adaption_lp_ip_fwd_static_ws.argtypes = [I64, I64, I64, adaption_qtensor, adaption_qtensor, P, I32, I32,
+                                                 I32, I32, adaption_qtensor, P, P]
     lib.adaption_maxpool2x2.argtypes = [adaption_qtensor, I32, I32, I32, I32, adaption_qtensor, P]
     lib.adaption_choose_frac_bits_from_acc.argtypes = [I64, I32, I32, C.POINTER(adaption_qfmt)]
     lib.adaption_status_string.argtypes = [C.c_int]
@@ -232,6 +234,21 @@ def adaption_lp_ip_fwd(B: int, K: int, O: int, x: QTensor, w: QTensor, bias_q: t
     _check(load().adaption_lp_ip_fwd(B, K, O, x.c_struct(), w.c_struct(), _ptr(bias_q), bias_frac_bits,
                                      int(relu), mode, algo, ys, _ptr(d_stats), _ptr(workspace), wsb,
                                      _stream()), "adaption_lp_ip_fwd")
+
+
+STATIC_WORKSPACE_BYTES = 4 << 20
+
+
+def adaption_lp_ip_fwd_static_ws(B: int, K: int, O: int, x: QTensor, w: QTensor, bias_q: torch.Tensor | None,
+                                 bias_frac_bits: int, relu: bool, mode: int, algo: int, y: QTensor | None,
+                                 d_stats: torch.Tensor):
+    """adaption_lp_ip_fwd without a workspace argument: the library's built-in scratch array is used.
+    For callers that must not allocate; shapes whose workspace exceeds STATIC_WORKSPACE_BYTES raise
+    AdaptionError(ERR_WORKSPACE).  Calls that may overlap on the GPU must be ordered by the caller."""
+    ys = y.c_struct() if y is not None else adaption_qtensor()
+    _check(load().adaption_lp_ip_fwd_static_ws(B, K, O, x.c_struct(), w.c_struct(), _ptr(bias_q),
+                                               bias_frac_bits, int(relu), mode, algo, ys, _ptr(d_stats),
+                                               _stream()), "adaption_lp_ip_fwd_static_ws")
 
 
 def adaption_maxpool2x2(x: QTensor, N: int, H: int, W: int, Cc: int, y: QTensor):
