@@ -50,7 +50,7 @@ def read_peaks():
 # clocks
 # ---------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -63,12 +63,15 @@ class ClockSampler:
         try:
             self.fh = open(self.path, "w")
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.gpu)], stdout=self.fh, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self) -> dict:
+    def stop(self, t_begin: float | None = None, t_end: float | None = None) -> dict:
+        """Median SM clock and the throttle reasons seen; with t_begin/t_end (time.time()) only the
+        samples taken inside that window count."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
         if self.proc is None:
             return out
@@ -84,6 +87,13 @@ class ClockSampler:
                 f = [t.strip() for t in line.split(",")]
                 if len(f) < 9:
                     continue
+                if t_begin is not None:
+                    try:
+                        ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    except ValueError:
+                        continue
+                    if ts < t_begin - 0.05 or ts > t_end + 0.05:
+                        continue
                 try:
                     sm.append(float(f[1]))
                     mx.append(float(f[2]))
@@ -223,28 +233,35 @@ def run_gpu(args):
     # + one per layer (+1 finalize where K is split)
     launches_step = 3 + 2 * n_gemm + len(net.layers) + sum(1 for L in gemm_layers if L.workspace is not None)
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()          # nvidia-smi needs a moment to start: launch it before the warm-up
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
+    if rank == 0:
+        t_spin = time.time()
+        while time.time() - t_spin < 1.0:       # untimed extra warm-up until the sampler is running
+            step()
+            torch.cuda.synchronize()
 
     net.zero_stats()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     events = []
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
     t0.record()
     for _ in range(args.steps):
         out = step(events)
     t1.record()
     torch.cuda.synchronize()
+    wall1 = time.time()
     if dist is not None:
         dist.barrier()
     elapsed_ms = t0.elapsed_time(t1)
-    clocks = sampler.stop() if rank == 0 else {}
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else {}
     if dist is not None:
         tt = torch.tensor([elapsed_ms], device="cuda")
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
@@ -366,7 +383,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=64)

@@ -145,15 +145,21 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
+// Operand descriptors are passed as 32-bit halves: the high word (group stride, version, swizzle)
+// is the same for every operand tile of a launch, the low word is the shared-memory address in
+// 16-byte units, so stepping along K or to another plane is one 32-bit add.
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                       uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n"
+      ".reg .b64 da, db;\n"
+      "setp.ne.b32 p, %5, 0;\n"
+      "mov.b64 da, {%1, %3};\n"
+      "mov.b64 db, {%2, %3};\n"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n"
       "}\n" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int32_t (&r)[32]) {
@@ -175,15 +181,14 @@ __device__ __forceinline__ void tmem_ld_wait() {
 
 // Shared-memory matrix descriptor of a K-major operand tile whose rows are BK bytes long and
 // swizzled with a span of BK bytes: eight-row groups are `sbo` bytes apart; the two 16-byte
-// halves of one 32-byte k-step are adjacent.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t sbo, uint32_t layout_type) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
-  d |= (uint64_t)1 << 16;
-  d |= (uint64_t)((sbo >> 4) & 0x3FFF) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)layout_type << 61;
-  return d;
+// halves of one 32-byte k-step are adjacent (leading offset 1).
+// High word: group stride / 16 in bits 0-13, descriptor version 1 in bit 14, swizzle in bits 29-31.
+__device__ __forceinline__ uint32_t smem_desc_hi(uint32_t sbo, uint32_t layout_type) {
+  return ((sbo >> 4) & 0x3FFFu) | (1u << 14) | (layout_type << 29);
+}
+// Low word: start address / 16 in bits 0-13, leading offset 1 in bits 16-29.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr) {
+  return ((saddr >> 4) & 0x3FFFu) | (1u << 16);
 }
 
 // Instruction descriptor: int32 accumulate, 8-bit operands with independent signedness,
@@ -238,6 +243,82 @@ __device__ __forceinline__ long long combine(int32_t a0, int32_t a1, int32_t a2)
   return (long long)a0;
 }
 
+// Requantization of one pre-activation value for the common case of a rounding right shift
+// (shift >= 1): v / 2^shift rounded half away from zero, saturated to [qmin, qmax].  The shifted
+// value is narrowed to 32 bits with saturation first, so clamping and counting are 32-bit work.
+// With ReLU the value is non-negative and the lower bound cannot be crossed.
+template <bool RELU, bool COUNT_ALL>
+__device__ __forceinline__ int32_t requant_shift_right(long long v, long long half, int shift, int32_t qmin,
+                                                       int32_t qmax, bool counted, Counts& c) {
+  if (RELU) v = v < 0 ? 0ll : v;
+  long long t = v + half;
+  if (!RELU) t += (v >> 63);
+  const long long r = t >> shift;
+  const int32_t r32 = (int32_t)r;
+  const int32_t rh = (int32_t)(r >> 32);
+  const int32_t rs = (rh == (r32 >> 31)) ? r32 : (rh < 0 ? (int32_t)0x80000000 : 0x7fffffff);
+  const int32_t q = min(max(rs, qmin), qmax);
+  if (COUNT_ALL) {
+    c.sat_pos += (rs > qmax);
+    if (!RELU) c.sat_neg += (rs < qmin);
+    c.zeros += (q == 0);
+  } else {
+    c.sat_pos += (counted && rs > qmax);
+    if (!RELU) c.sat_neg += (counted && rs < qmin);
+    c.zeros += (counted && q == 0);
+  }
+  return q;
+}
+
+// Sixteen consecutive output columns of one row: recombine, add bias, requantize, pack into
+// byte planes (and the optional int16 copy) and store 16 bytes per plane.
+template <int NACC, bool RELU>
+__device__ __forceinline__ void requant_store16(const int32_t* a0, const int32_t* a1, const int32_t* a2,
+                                                const long long* bias64, const TcParams& p, bool row_ok,
+                                                int m, int col, Counts& cnt) {
+  int32_t q[16];
+  const int nvalid = row_ok ? min(max(p.N - col, 0), 16) : 0;
+  if (p.rq.shift > 0) {
+    const long long half = 1ll << (p.rq.shift - 1);
+    if (nvalid == 16) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        q[j] = requant_shift_right<RELU, true>(
+            combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bias64[j], half, p.rq.shift,
+            p.rq.qmin, p.rq.qmax, true, cnt);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        q[j] = requant_shift_right<RELU, false>(
+            combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bias64[j], half, p.rq.shift,
+            p.rq.qmin, p.rq.qmax, j < nvalid, cnt);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      q[j] = requant_value(combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bias64[j],
+                           p.rq, j < nvalid, cnt);
+  }
+  if (row_ok && col < p.y_stride) {
+    uint32_t w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) w[j] = __byte_perm((uint32_t)q[2 * j], (uint32_t)q[2 * j + 1], 0x5410);
+    const size_t off = (size_t)m * (size_t)p.y_stride + (size_t)col;
+    *reinterpret_cast<uint4*>(p.y_lo + off) =
+        make_uint4(__byte_perm(w[0], w[1], 0x6420), __byte_perm(w[2], w[3], 0x6420),
+                   __byte_perm(w[4], w[5], 0x6420), __byte_perm(w[6], w[7], 0x6420));
+    if (p.rq.out_planes == 2)
+      *reinterpret_cast<uint4*>(p.y_hi + off) =
+          make_uint4(__byte_perm(w[0], w[1], 0x7531), __byte_perm(w[2], w[3], 0x7531),
+                     __byte_perm(w[4], w[5], 0x7531), __byte_perm(w[6], w[7], 0x7531));
+    if (p.y_q16 != nullptr) {
+      uint4* dst = reinterpret_cast<uint4*>(p.y_q16 + off);
+      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------- kernel
 template <int NAX, int NBW>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -277,11 +358,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t it = 0;
+      uint32_t it = 0, ph = 0;
+      int s = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x) {
         const TileCoord tc = decode_tile(t, p);
         int img = 0, base_h = 0, base_w = 0;
+        int tap = 0, cb = 0, r = 0, sx = 0;       // position of kb in the (tap, channel block) order
         if (p.is_conv) {
           const int ow = tc.m0 % p.OW;
           const int rest = tc.m0 / p.OW;
@@ -289,20 +372,18 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           img = rest / p.OH;
           base_w = ow * p.stride_w - p.pad_w;
           base_h = oh * p.stride_h - p.pad_h;
+          tap = tc.kb_begin / p.cblks;
+          cb = tc.kb_begin - tap * p.cblks;
+          r = tap / p.S;
+          sx = tap - r * p.S;
         }
         for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb, ++it) {
-          const int s = (int)(it % (uint32_t)p.stages);
-          const uint32_t ph = (it / (uint32_t)p.stages) & 1u;
           if (!wait_bar(smem_u32(&ctrl.empty[s]), ph ^ 1u, &ctrl, p)) { ok = false; break; }
           const uint32_t full = smem_u32(&ctrl.full[s]);
           mbar_expect_tx(full, p.stage_bytes);
           const uint32_t sa = ring + (uint32_t)s * p.stage_bytes;
           const uint32_t sb = sa + NAX * p.a_bytes;
           if (p.is_conv) {
-            const int tap = kb / p.cblks;
-            const int cb = kb - tap * p.cblks;
-            const int r = tap / p.S;
-            const int sx = tap - r * p.S;
             tma_load_im2col(sa, &map_a0, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx, (uint16_t)r);
             if (NAX == 2)
               tma_load_im2col(sa + p.a_bytes, &map_a1, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx,
@@ -310,6 +391,11 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             const int kcol = tap * p.w_pitch + cb * p.BK;
             tma_load_2d(sb, &map_b0, full, kcol, tc.n0);
             if (NBW == 2) tma_load_2d(sb + p.b_bytes, &map_b1, full, kcol, tc.n0);
+            if (++cb == p.cblks) {
+              cb = 0;
+              ++tap;
+              if (++sx == p.S) { sx = 0; ++r; }
+            }
           } else {
             const int kcol = kb * p.BK;
             tma_load_2d(sa, &map_a0, full, kcol, tc.m0);
@@ -317,16 +403,17 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             tma_load_2d(sb, &map_b0, full, kcol, tc.n0);
             if (NBW == 2) tma_load_2d(sb + p.b_bytes, &map_b1, full, kcol, tc.n0);
           }
+          if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
       }
       if (!ok || ctrl.abort) {
         // gave up: let the copies already issued land before the CTA releases its shared memory
         const uint32_t n = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
         for (uint32_t j = it - n; j < it; ++j) {
-          const int s = (int)(j % (uint32_t)p.stages);
-          const uint32_t ph = (j / (uint32_t)p.stages) & 1u;
+          const int sj = (int)(j % (uint32_t)p.stages);
+          const uint32_t pj = (j / (uint32_t)p.stages) & 1u;
           const unsigned long long t0 = global_ns();
-          while (!mbar_try_wait(smem_u32(&ctrl.full[s]), ph) && global_ns() - t0 < 50000000ull) {
+          while (!mbar_try_wait(smem_u32(&ctrl.full[sj]), pj) && global_ns() - t0 < 50000000ull) {
           }
         }
       }
@@ -339,7 +426,11 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       const uint32_t id_su = make_idesc(true, false, p.BN);
       const uint32_t id_us = make_idesc(false, true, p.BN);
       const uint32_t id_uu = make_idesc(false, false, p.BN);
-      uint32_t it = 0, tile_iter = 0;
+      const uint32_t dhi = smem_desc_hi(p.sbo, p.layout_type);
+      const uint32_t ring_lo = smem_desc_lo(ring);
+      const uint32_t stage_u = p.stage_bytes >> 4, a_u = p.a_bytes >> 4, b_u = p.b_bytes >> 4;
+      uint32_t it = 0, tile_iter = 0, ph = 0;
+      int s = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, ++tile_iter) {
         const TileCoord tc = decode_tile(t, p);
@@ -348,37 +439,34 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         if (!wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
+        const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
         for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb, ++it) {
-          const int s = (int)(it % (uint32_t)p.stages);
-          const uint32_t ph = (it / (uint32_t)p.stages) & 1u;
           if (!wait_bar(smem_u32(&ctrl.full[s]), ph, &ctrl, p)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = ring + (uint32_t)s * p.stage_bytes;
-          const uint32_t sb = sa + NAX * p.a_bytes;
-          for (int ks = 0; ks < p.ksteps; ++ks) {
-            const uint32_t acc = (kb > tc.kb_begin || ks > 0) ? 1u : 0u;
-            const uint64_t a0 = make_smem_desc(sa + ks * 32, p.sbo, p.layout_type);
-            const uint64_t b0 = make_smem_desc(sb + ks * 32, p.sbo, p.layout_type);
+          // low descriptor words of the operand planes of this stage (16-byte units)
+          const uint32_t a0 = ring_lo + (uint32_t)s * stage_u;
+          const uint32_t a1 = a0 + a_u;
+          const uint32_t b0 = a0 + NAX * a_u;
+          const uint32_t b1 = b0 + b_u;
+          uint32_t acc = kb > tc.kb_begin ? 1u : 0u;
+          for (uint32_t ks = 0; ks < 2u * (uint32_t)p.ksteps; ks += 2u, acc = 1u) {   // 32 bytes per k-step
             if (NAX == 2 && NBW == 2) {
-              const uint64_t a1 = make_smem_desc(sa + p.a_bytes + ks * 32, p.sbo, p.layout_type);
-              const uint64_t b1 = make_smem_desc(sb + p.b_bytes + ks * 32, p.sbo, p.layout_type);
-              mma_i8(d0, a0, b0, id_ss, acc);                 // hi*hi            weight 2^16
-              mma_i8(d0 + p.BN, a0, b1, id_su, acc);          // hi*lo            weight 2^8
-              mma_i8(d0 + p.BN, a1, b0, id_us, 1u);           // lo*hi            weight 2^8
-              mma_i8(d0 + 2 * p.BN, a1, b1, id_uu, acc);      // lo*lo            weight 1
+              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);          // hi*hi   weight 2^16
+              mma_i8(d1, a0 + ks, b1 + ks, dhi, id_su, acc);          // hi*lo   weight 2^8
+              mma_i8(d1, a1 + ks, b0 + ks, dhi, id_us, 1u);           // lo*hi   weight 2^8
+              mma_i8(d2, a1 + ks, b1 + ks, dhi, id_uu, acc);          // lo*lo   weight 1
             } else if (NAX == 2 && NBW == 1) {
-              const uint64_t a1 = make_smem_desc(sa + p.a_bytes + ks * 32, p.sbo, p.layout_type);
-              mma_i8(d0, a0, b0, id_ss, acc);                 // hi*w             weight 2^8
-              mma_i8(d0 + p.BN, a1, b0, id_us, acc);          // lo*w             weight 1
+              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);          // hi*w    weight 2^8
+              mma_i8(d1, a1 + ks, b0 + ks, dhi, id_us, acc);          // lo*w    weight 1
             } else if (NAX == 1 && NBW == 2) {
-              const uint64_t b1 = make_smem_desc(sb + p.b_bytes + ks * 32, p.sbo, p.layout_type);
-              mma_i8(d0, a0, b0, id_ss, acc);                 // x*hi             weight 2^8
-              mma_i8(d0 + p.BN, a0, b1, id_su, acc);          // x*lo             weight 1
+              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);          // x*hi    weight 2^8
+              mma_i8(d1, a0 + ks, b1 + ks, dhi, id_su, acc);          // x*lo    weight 1
             } else {
-              mma_i8(d0, a0, b0, id_ss, acc);
+              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);
             }
           }
           tc_commit(smem_u32(&ctrl.empty[s]));                // stage reusable once these MMAs retire
+          if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
         if (ok) tc_commit(smem_u32(&ctrl.tmem_full[buf]));    // accumulators of this tile complete
       }
@@ -448,29 +536,12 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
               v = v < 0 ? -v : v;
               if (row_ok && col + j < p.N) vmax = v > vmax ? v : vmax;
             }
+          } else if (p.rq.relu) {
+            requant_store16<NACC, true>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + c0 + 16 * g, p, row_ok, m,
+                                        col, cnt);
           } else {
-            uint32_t lo_w[4] = {0, 0, 0, 0}, hi_w[4] = {0, 0, 0, 0}, q_w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const long long v = combine<NACC>(a0[16 * g + j], NACC >= 2 ? a1[16 * g + j] : 0,
-                                                NACC == 3 ? a2[16 * g + j] : 0) +
-                                  bias64[c0 + 16 * g + j];
-              const int32_t q = requant_value(v, p.rq, row_ok && col + j < p.N, cnt);
-              lo_w[j >> 2] |= (uint32_t)(q & 255) << (8 * (j & 3));
-              hi_w[j >> 2] |= (uint32_t)((q >> 8) & 255) << (8 * (j & 3));
-              q_w[j >> 1] |= (uint32_t)(q & 0xffff) << (16 * (j & 1));
-            }
-            if (row_ok && col < p.y_stride) {
-              const size_t off = (size_t)m * (size_t)p.y_stride + (size_t)col;
-              *reinterpret_cast<uint4*>(p.y_lo + off) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
-              if (p.rq.out_planes == 2)
-                *reinterpret_cast<uint4*>(p.y_hi + off) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
-              if (p.y_q16 != nullptr) {
-                uint4* dst = reinterpret_cast<uint4*>(p.y_q16 + off);
-                dst[0] = make_uint4(q_w[0], q_w[1], q_w[2], q_w[3]);
-                dst[1] = make_uint4(q_w[4], q_w[5], q_w[6], q_w[7]);
-              }
-            }
+            requant_store16<NACC, false>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + c0 + 16 * g, p, row_ok,
+                                         m, col, cnt);
           }
         }
       }
