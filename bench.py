@@ -145,17 +145,25 @@ def run_reference(args):
     sample_images = 1
     x = wl.vgg16_input(sample_images, seed=0)
     formats = oracle_formats(params, x, args.n_bits)
-    for _ in range(args.warmup):
+    # keep the whole run within a few minutes: the oracle is slow by design, so when K + W steps
+    # of one image each would take longer than the budget, fewer steps are executed and said so
+    budget_s = 240.0
+    t_probe = oracle_sample_step(params, x, formats, args.n_bits)
+    can_run = max(1, int(budget_s / max(t_probe, 1e-3)))
+    warm = min(args.warmup, max(0, can_run - 1) // 4)
+    steps_exec = max(1, min(args.steps, can_run - warm))
+    for _ in range(warm):
         oracle_sample_step(params, x, formats, args.n_bits)
     t = 0.0
-    for _ in range(args.steps):
+    for _ in range(steps_exec):
         t += oracle_sample_step(params, x, formats, args.n_bits)
-    ms = t / args.steps * 1e3
+    ms = t / steps_exec * 1e3
     ips = sample_images / (ms / 1e3)
     cores = orc.num_threads()
     line = {
         "impl": "reference", "metric": METRIC, "value": ips, "unit": "images/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "steps_executed": steps_exec, "warmup_executed": warm,
+        "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": f"int{args.n_bits}", "data": "synthetic",
         "effective_tops": 2.0 * macs_img * ips / 1e12,
         "config": {"workload": f"VGG16 forward, {args.n_bits}-bit weights and activations (full stack); "

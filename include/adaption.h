@@ -179,6 +179,17 @@ ADAPTION_API int adaption_maxpool2x2(adaption_qtensor x, int32_t N, int32_t H, i
 ADAPTION_API int adaption_choose_frac_bits_from_acc(int64_t max_abs_acc, int32_t acc_frac_bits,
                                        int32_t n_bits, adaption_qfmt* h_out);
 
+/* Measurement aid for the roofline of the layer calls (no counterpart in the paper): every SM
+ * (pair != 0: every pair of SMs working on 256-row tiles) issues 4*iters back-to-back int8
+ * tensor-core instructions of shape 128 (256) x bn x 32 on operands resident in shared memory.
+ * d_cycles receives, per launched block (one per SM; at least 148 entries), the SM clock cycles
+ * the issuing block needed (entries of non-issuing blocks are left untouched); *d_status is set to
+ * ADAPTION_ERR_TIMEOUT if a wait gave up.  bn is 64, 128 or 256.  commit_every > 0 adds a
+ * completion signal (tcgen05.commit) after every commit_every groups of four instructions, as a
+ * pipelined mainloop issues them; 0 issues none.  Asynchronous on `stream`. */
+ADAPTION_API int adaption_probe_i8_peak(int32_t bn, int32_t pair, int32_t iters, int32_t commit_every,
+                                        uint64_t* d_cycles, int32_t* d_status, void* stream);
+
 ADAPTION_API const char* adaption_status_string(int status);
 
 #ifdef __cplusplus

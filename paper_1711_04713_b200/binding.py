@@ -47,7 +47,7 @@ EXPORTS = [
     "adaption_measure_range", "adaption_quantize", "adaption_lp_act",
     "adaption_lp_conv_workspace_bytes", "adaption_lp_conv_fwd", "adaption_lp_ip_workspace_bytes",
     "adaption_lp_ip_fwd", "adaption_lp_ip_fwd_static_ws", "adaption_maxpool2x2", "adaption_choose_frac_bits_from_acc",
-    "adaption_status_string",
+    "adaption_probe_i8_peak", "adaption_status_string",
 ]
 
 _lib = None
@@ -86,6 +86,7 @@ def load(path: str | None = None):
                                                  I32, I32, adaption_qtensor, P, P]
     lib.adaption_maxpool2x2.argtypes = [adaption_qtensor, I32, I32, I32, I32, adaption_qtensor, P]
     lib.adaption_choose_frac_bits_from_acc.argtypes = [I64, I32, I32, C.POINTER(adaption_qfmt)]
+    lib.adaption_probe_i8_peak.argtypes = [I32, I32, I32, I32, P, P, P]
     lib.adaption_status_string.argtypes = [C.c_int]
     lib.adaption_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -254,6 +255,13 @@ def adaption_lp_ip_fwd_static_ws(B: int, K: int, O: int, x: QTensor, w: QTensor,
 def adaption_maxpool2x2(x: QTensor, N: int, H: int, W: int, Cc: int, y: QTensor):
     _check(load().adaption_maxpool2x2(x.c_struct(), N, H, W, Cc, y.c_struct(), _stream()),
            "adaption_maxpool2x2")
+
+
+def adaption_probe_i8_peak(bn: int, pair: bool, iters: int, d_cycles: torch.Tensor, d_status: torch.Tensor,
+                           commit_every: int = 0):
+    """d_cycles: int64 CUDA tensor with one entry per SM; d_status: one int32."""
+    _check(load().adaption_probe_i8_peak(bn, int(pair), iters, commit_every, _ptr(d_cycles), _ptr(d_status), _stream()),
+           "adaption_probe_i8_peak")
 
 
 def adaption_choose_frac_bits_from_acc(max_abs_acc: int, acc_frac_bits: int, n_bits: int) -> int:

@@ -10,6 +10,10 @@ int measure_range_impl(const float*, size_t, int32_t, float*, adaption_qfmt*, cu
 int maxpool_impl(const adaption_qtensor&, int32_t, int32_t, int32_t, int32_t, const adaption_qtensor&,
                  cudaStream_t);
 
+int probe_i8_peak(int bn, int pair, int iters, int commit_every, unsigned long long* d_cycles, int* d_status,
+                  cudaStream_t stream);
+int num_sms();
+
 // Longest reduction the direct kernels and the int64 workspace can take without overflow:
 // |q_x * q_w| <= 2^30, so 2^31 terms still leave a sign bit and headroom for the bias.
 static const int64_t kMaxReduction = (int64_t)1 << 31;
@@ -212,6 +216,16 @@ int adaption_choose_frac_bits_from_acc(int64_t max_abs_acc, int32_t acc_frac_bit
   h_out->n_bits = n_bits;
   h_out->frac_bits = n_bits - 1 - m;
   return ADAPTION_OK;
+}
+
+int adaption_probe_i8_peak(int32_t bn, int32_t pair, int32_t iters, int32_t commit_every, uint64_t* d_cycles,
+                           int32_t* d_status, void* stream) {
+  if ((bn != 64 && bn != 128 && bn != 256) || iters < 1 || iters > (1 << 19) || commit_every < 0 ||
+      d_cycles == nullptr ||
+      d_status == nullptr)
+    return ADAPTION_ERR_INVALID_ARG;
+  return probe_i8_peak(bn, pair ? 1 : 0, iters, commit_every, reinterpret_cast<unsigned long long*>(d_cycles), d_status,
+                       reinterpret_cast<cudaStream_t>(stream));
 }
 
 const char* adaption_status_string(int status) {

@@ -11,9 +11,10 @@
 // take a single product.
 //
 // One persistent CTA per SM walks over output tiles (128 rows x BN columns):
-//   warp 0     : TMA producer (im2col / tiled loads into a ring of shared-memory stages)
-//   warp 1     : TMEM allocation and the single MMA-issuing thread
-//   warps 2-5  : epilogue (tcgen05.ld -> int64 recombination -> bias, ReLU, requantize with
+//   warps 0-3  : TMA producers, one per operand plane (im2col / tiled loads into a ring of
+//                shared-memory stages; a single warp issues bulk-tensor copies too slowly)
+//   warp 4     : TMEM allocation and the single MMA-issuing thread
+//   warps 5-12 : epilogue (tcgen05.ld -> int64 recombination -> bias, ReLU, requantize with
 //                saturation, zero / saturation counters, byte-plane stores; or range / split-K)
 // Every device-side wait is bounded; on expiry the kernel flags ADAPTION_ERR_TIMEOUT in the
 // caller's stats word, drains what it has in flight, frees its TMEM and returns.
@@ -33,7 +34,11 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kMaxStages = 8;
 constexpr int kMaxAccBufs = 4;
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter, each takes half the columns
+constexpr int kProducerWarps = 4;            // one per operand plane: TMA issue is slow per warp
+constexpr int kMmaWarp = kProducerWarps;
+constexpr int kFirstEpiWarp = kProducerWarps + 1;
+constexpr int kThreads = 32 * (kProducerWarps + 1 + kEpiWarps);
 constexpr int kMaxBN = 256;
 // int32 accumulators: the shared middle accumulator takes two products of magnitude
 // <= 128*255 per k, so a reduction of up to 32768 stays below 2^31.
@@ -41,6 +46,7 @@ constexpr int64_t kMaxKPerAccumulation = 32768;
 
 struct TcParams {
   int M, N;
+  int tile_m;                 // rows per tile: 128, or 256 for a CTA pair
   int tiles_m, tiles_n, splits, total_tiles;
   int num_kb, kb_per_split;
   int BN, BK, ksteps;
@@ -64,6 +70,17 @@ struct TcParams {
   unsigned long long timeout_ns;
 };
 
+// Optional per-role time stamps of CTA 0 (development builds only: -DADAPTION_TIMELINE).
+#ifdef ADAPTION_TIMELINE
+__device__ long long g_timeline[8192];
+#define TL_STAMP(role, tile, slot)                                                        \
+  do {                                                                                    \
+    if (blockIdx.x == 0 && (tile) < 32u) g_timeline[((role) * 32 + (tile)) * 8 + (slot)] = clock64(); \
+  } while (0)
+#else
+#define TL_STAMP(role, tile, slot) do { } while (0)
+#endif
+
 struct Ctrl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
@@ -72,7 +89,7 @@ struct Ctrl {
   unsigned long long drain;
   uint32_t tmem_base;
   volatile uint32_t abort;
-  long long bias64[4][kMaxBN];
+  long long bias64[kEpiWarps][kMaxBN / 2 < 32 ? 32 : kMaxBN / 2];
 };
 
 // ---------------------------------------------------------------------------------- PTX
@@ -107,33 +124,84 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+// PAIR: the copy lands in this CTA's shared memory but reports its bytes to an mbarrier that may
+// live in the other CTA of the pair (the leader's "full" barrier).
+template <bool PAIR>
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x,
                                             int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-      "l"(map), "r"(bar), "r"(x), "r"(y)
-      : "memory");
+  if (PAIR)
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+  else
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
 }
+template <bool PAIR>
 __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c,
                                                 int w, int h, int n, uint16_t off_w, uint16_t off_h) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(dst),
-      "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
-      : "memory");
+  if (PAIR)
+    asm volatile(
+        "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+  else
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
 }
+template <bool PAIR>
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
-               "r"(ncols)
-               : "memory");
+  if (PAIR)
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+                 "r"(ncols)
+                 : "memory");
+  else
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem),
+                 "r"(ncols)
+                 : "memory");
 }
+template <bool PAIR>
 __device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (PAIR)
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  else
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
+template <bool PAIR>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
-               : "memory");
+  if (PAIR)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+                 : "memory");
+  else
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols)
+                 : "memory");
+}
+// ---- CTA-pair plumbing
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -141,26 +209,52 @@ __device__ __forceinline__ void tc_fence_before() {
 __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
+// Arrive on `bar` once every MMA issued so far by this thread has retired.  PAIR: the arrival is
+// delivered to the barrier at the same offset in both CTAs of the pair.
+template <bool PAIR>
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
+  if (PAIR)
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+            bar),
+        "h"((uint16_t)3)
+        : "memory");
+  else
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
 }
 // Operand descriptors are passed as 32-bit halves: the high word (group stride, version, swizzle)
 // is the same for every operand tile of a launch, the low word is the shared-memory address in
 // 16-byte units, so stepping along K or to another plane is one 32-bit add.
+// PAIR: one instruction computes a 256-row tile across the two CTAs of the pair: each CTA supplies
+// its own 128 rows of A and half of the B rows, and receives its 128 rows of the result in its TMEM.
+template <bool PAIR>
 __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
                                        uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      ".reg .b64 da, db;\n"
-      "setp.ne.b32 p, %5, 0;\n"
-      "mov.b64 da, {%1, %3};\n"
-      "mov.b64 db, {%2, %3};\n"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n"
-      "}\n" ::"r"(d_tmem),
-      "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if (PAIR)
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "mov.b64 da, {%1, %3};\n"
+        "mov.b64 db, {%2, %3};\n"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %4, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "mov.b64 da, {%1, %3};\n"
+        "mov.b64 db, {%2, %3};\n"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int32_t (&r)[32]) {
   asm volatile(
@@ -191,19 +285,77 @@ __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr) {
   return ((saddr >> 4) & 0x3FFFu) | (1u << 16);
 }
 
+
+// One 32-byte k-step of a tile, issued as a single instruction sequence so that the issuing thread
+// spends as few instructions per MMA as possible (its instruction stream, not the tensor pipe, is
+// what limits the mainloop otherwise).  Operand descriptors: low words a0/a1/b0/b1, shared high
+// word dhi.  acc = 0 overwrites the accumulators (first k-step of a tile).
+#define ADAPTION_MMA_KSTEP_2X2(CG)                                                              \
+  asm volatile(                                                                                 \
+      "{\n"                                                                                     \
+      ".reg .pred p, q;\n"                                                                      \
+      ".reg .b64 da0, da1, db0, db1;\n"                                                         \
+      "setp.ne.b32 p, %12, 0;\n"                                                                \
+      "setp.eq.b32 q, %7, %7;\n"                                                                \
+      "mov.b64 da0, {%3, %7};\n"                                                                \
+      "mov.b64 da1, {%4, %7};\n"                                                                \
+      "mov.b64 db0, {%5, %7};\n"                                                                \
+      "mov.b64 db1, {%6, %7};\n"                                                                \
+      "tcgen05.mma.cta_group::" CG ".kind::i8 [%0], da0, db0, %8, p;\n"                         \
+      "tcgen05.mma.cta_group::" CG ".kind::i8 [%1], da0, db1, %9, p;\n"                         \
+      "tcgen05.mma.cta_group::" CG ".kind::i8 [%1], da1, db0, %10, q;\n"                        \
+      "tcgen05.mma.cta_group::" CG ".kind::i8 [%2], da1, db1, %11, p;\n"                        \
+      "}\n" ::"r"(d0),                                                                          \
+      "r"(d1), "r"(d2), "r"(a0), "r"(a1), "r"(b0), "r"(b1), "r"(dhi), "r"(id_ss), "r"(id_su),  \
+      "r"(id_us), "r"(id_uu), "r"(acc)                                                          \
+      : "memory")
+
+template <bool PAIR>
+__device__ __forceinline__ void mma_kstep_2x2(uint32_t d0, uint32_t d1, uint32_t d2, uint32_t a0, uint32_t a1,
+                                              uint32_t b0, uint32_t b1, uint32_t dhi, uint32_t id_ss,
+                                              uint32_t id_su, uint32_t id_us, uint32_t id_uu, uint32_t acc) {
+  // hi*hi -> d0 (weight 2^16); hi*lo and lo*hi -> d1 (weight 2^8); lo*lo -> d2 (weight 1)
+  if (PAIR)
+    ADAPTION_MMA_KSTEP_2X2("2");
+  else
+    ADAPTION_MMA_KSTEP_2X2("1");
+}
+#undef ADAPTION_MMA_KSTEP_2X2
+
+template <int NAX, int NBW, bool PAIR>
+__device__ __forceinline__ void mma_kstep(uint32_t d0, uint32_t d1, uint32_t d2, uint32_t a0, uint32_t a1,
+                                          uint32_t b0, uint32_t b1, uint32_t dhi, uint32_t id_ss, uint32_t id_su,
+                                          uint32_t id_us, uint32_t id_uu, uint32_t acc) {
+  if (NAX == 2 && NBW == 2) {
+    mma_kstep_2x2<PAIR>(d0, d1, d2, a0, a1, b0, b1, dhi, id_ss, id_su, id_us, id_uu, acc);
+  } else if (NAX == 2 && NBW == 1) {
+    mma_i8<PAIR>(d0, a0, b0, dhi, id_ss, acc);          // hi*w    weight 2^8
+    mma_i8<PAIR>(d1, a1, b0, dhi, id_us, acc);          // lo*w    weight 1
+  } else if (NAX == 1 && NBW == 2) {
+    mma_i8<PAIR>(d0, a0, b0, dhi, id_ss, acc);          // x*hi    weight 2^8
+    mma_i8<PAIR>(d1, a0, b1, dhi, id_su, acc);          // x*lo    weight 1
+  } else {
+    mma_i8<PAIR>(d0, a0, b0, dhi, id_ss, acc);
+  }
+}
+
 // Instruction descriptor: int32 accumulate, 8-bit operands with independent signedness,
 // both K-major, M = 128, N = bn.
-__device__ __forceinline__ uint32_t make_idesc(bool a_signed, bool b_signed, int bn) {
+__device__ __forceinline__ uint32_t make_idesc(bool a_signed, bool b_signed, int bn, int m) {
   return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | ((b_signed ? 1u : 0u) << 10) |
-         ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+         ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // Bounded wait on an mbarrier phase.  Returns false once the time limit is hit (or another
 // role already gave up); the caller then leaves its loop.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Ctrl* ctrl, const TcParams& p) {
+// `relaxed` waiters (producers, epilogue) sleep between polls so that their spinning does not take
+// issue slots from the MMA-issuing thread, whose instruction stream is the critical path.
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Ctrl* ctrl, const TcParams& p,
+                                       bool relaxed) {
   const unsigned long long t0 = global_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
+    if (relaxed) __nanosleep(40);
     if ((++spins & 127u) == 0) {
       if (ctrl->abort) return false;
       if (global_ns() - t0 > p.timeout_ns) {
@@ -215,9 +367,10 @@ __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Ctrl* ctrl
   }
   return true;
 }
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctrl* ctrl, const TcParams& p) {
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctrl* ctrl, const TcParams& p,
+                                         bool relaxed = true) {
   if (mbar_try_wait(bar, parity)) return true;
-  return wait_slow(bar, parity, ctrl, p);
+  return wait_slow(bar, parity, ctrl, p, relaxed);
 }
 
 struct TileCoord {
@@ -229,7 +382,7 @@ __device__ __forceinline__ TileCoord decode_tile(int t, const TcParams& p) {
   const int rest = t / p.tiles_n;
   const int split = rest % p.splits;
   const int tm = rest / p.splits;
-  tc.m0 = tm * kBM;
+  tc.m0 = tm * p.tile_m;
   tc.n0 = tn * p.BN;
   tc.kb_begin = split * p.kb_per_split;
   tc.kb_end = min(p.num_kb, tc.kb_begin + p.kb_per_split);
@@ -320,7 +473,7 @@ __device__ __forceinline__ void requant_store16(const int32_t* a0, const int32_t
 }
 
 // ---------------------------------------------------------------------------------- kernel
-template <int NAX, int NBW>
+template <int NAX, int NBW, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
@@ -332,6 +485,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  // PAIR: two CTAs (a cluster of two) share every tile of 256 rows.  Rank 0 is the leader: it owns
+  // the "full" and "tmem_empty" barriers that are in use and issues the MMAs for both.
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  // rows of B this CTA stages per k-block, and where they start inside the tile's columns
+  const int b_rows = PAIR ? p.BN / 2 : p.BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -340,34 +500,46 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     }
     for (int b = 0; b < p.acc_bufs; ++b) {
       mbar_init(smem_u32(&ctrl.tmem_full[b]), 1);
-      mbar_init(smem_u32(&ctrl.tmem_empty[b]), 4);
+      mbar_init(smem_u32(&ctrl.tmem_empty[b]), PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
     mbar_init(smem_u32(&ctrl.drain), 1);
     ctrl.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {
-    tmem_alloc(smem_u32(&ctrl.tmem_base), p.tmem_cols);
-    tmem_relinquish();
+  if (warp == kMmaWarp) {
+    tmem_alloc<PAIR>(smem_u32(&ctrl.tmem_base), p.tmem_cols);
+    tmem_relinquish<PAIR>();
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();      // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = ctrl.tmem_base;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+  if (warp < kProducerWarps) {
+    // ------------------------------------------------------------------ TMA producers
+    // One warp per operand plane (A planes first, then B planes): every producer walks the same
+    // sequence of stages and issues only its own copy, so the copies of a stage are in flight
+    // side by side (one thread issues a bulk-tensor copy only every few hundred cycles).
+    constexpr int NPLANES = NAX + NBW;
+    if (lane == 0 && warp < NPLANES) {
+      const bool is_a = warp < NAX;
+      const int plane = is_a ? warp : warp - NAX;
+      const CUtensorMap* my_map = is_a ? (plane == 0 ? &map_a0 : &map_a1) : (plane == 0 ? &map_b0 : &map_b1);
+      const uint32_t my_off = is_a ? (uint32_t)plane * p.a_bytes : NAX * p.a_bytes + (uint32_t)plane * p.b_bytes;
       uint32_t it = 0, ph = 0;
       int s = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x) {
+      for (int t = worker; t < p.total_tiles && ok; t += workers) {
         const TileCoord tc = decode_tile(t, p);
+        const int m_begin = tc.m0 + (int)rank * kBM;        // first of the 128 rows this CTA stages
+        const int n_begin = tc.n0 + (int)rank * b_rows;     // first weight row this CTA stages
         int img = 0, base_h = 0, base_w = 0;
         int tap = 0, cb = 0, r = 0, sx = 0;       // position of kb in the (tap, channel block) order
+        TL_STAMP(0, (uint32_t)((t - worker) / workers), 0);
         if (p.is_conv) {
-          const int ow = tc.m0 % p.OW;
-          const int rest = tc.m0 / p.OW;
+          const int ow = m_begin % p.OW;
+          const int rest = m_begin / p.OW;
           const int oh = rest % p.OH;
           img = rest / p.OH;
           base_w = ow * p.stride_w - p.pad_w;
@@ -379,100 +551,114 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         }
         for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb, ++it) {
           if (!wait_bar(smem_u32(&ctrl.empty[s]), ph ^ 1u, &ctrl, p)) { ok = false; break; }
-          const uint32_t full = smem_u32(&ctrl.full[s]);
-          mbar_expect_tx(full, p.stage_bytes);
-          const uint32_t sa = ring + (uint32_t)s * p.stage_bytes;
-          const uint32_t sb = sa + NAX * p.a_bytes;
+          // bytes are reported to the leader's barrier; the leader arms it for both CTAs' copies
+          uint32_t full = smem_u32(&ctrl.full[s]);
+          if (PAIR) {
+            if (rank == 0 && warp == 0) mbar_expect_tx(full, 2u * p.stage_bytes);
+            full = mapa_rank(full, 0);
+          } else {
+            if (warp == 0) mbar_expect_tx(full, p.stage_bytes);
+          }
+          const uint32_t dst = ring + (uint32_t)s * p.stage_bytes + my_off;
           if (p.is_conv) {
-            tma_load_im2col(sa, &map_a0, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx, (uint16_t)r);
-            if (NAX == 2)
-              tma_load_im2col(sa + p.a_bytes, &map_a1, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx,
-                              (uint16_t)r);
-            const int kcol = tap * p.w_pitch + cb * p.BK;
-            tma_load_2d(sb, &map_b0, full, kcol, tc.n0);
-            if (NBW == 2) tma_load_2d(sb + p.b_bytes, &map_b1, full, kcol, tc.n0);
+            if (is_a)
+              tma_load_im2col<PAIR>(dst, my_map, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx, (uint16_t)r);
+            else
+              tma_load_2d<PAIR>(dst, my_map, full, tap * p.w_pitch + cb * p.BK, n_begin);
             if (++cb == p.cblks) {
               cb = 0;
               ++tap;
               if (++sx == p.S) { sx = 0; ++r; }
             }
           } else {
-            const int kcol = kb * p.BK;
-            tma_load_2d(sa, &map_a0, full, kcol, tc.m0);
-            if (NAX == 2) tma_load_2d(sa + p.a_bytes, &map_a1, full, kcol, tc.m0);
-            tma_load_2d(sb, &map_b0, full, kcol, tc.n0);
-            if (NBW == 2) tma_load_2d(sb + p.b_bytes, &map_b1, full, kcol, tc.n0);
+            tma_load_2d<PAIR>(dst, my_map, full, kb * p.BK, is_a ? m_begin : n_begin);
           }
           if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
       }
       if (!ok || ctrl.abort) {
-        // gave up: let the copies already issued land before the CTA releases its shared memory
+        // gave up: let the copies already issued land before the CTA releases its shared memory.
+        // (In a pair the bytes are counted on the leader's barriers, so the follower just waits.)
         const uint32_t n = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
         for (uint32_t j = it - n; j < it; ++j) {
           const int sj = (int)(j % (uint32_t)p.stages);
           const uint32_t pj = (j / (uint32_t)p.stages) & 1u;
           const unsigned long long t0 = global_ns();
+          if (PAIR && rank != 0) {
+            while (global_ns() - t0 < 2000000ull) {
+            }
+            break;
+          }
           while (!mbar_try_wait(smem_u32(&ctrl.full[sj]), pj) && global_ns() - t0 < 50000000ull) {
           }
         }
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t id_ss = make_idesc(true, true, p.BN);
-      const uint32_t id_su = make_idesc(true, false, p.BN);
-      const uint32_t id_us = make_idesc(false, true, p.BN);
-      const uint32_t id_uu = make_idesc(false, false, p.BN);
+  } else if (warp == kMmaWarp) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      const int tile_rows = PAIR ? 2 * kBM : kBM;
+      const uint32_t id_ss = make_idesc(true, true, p.BN, tile_rows);
+      const uint32_t id_su = make_idesc(true, false, p.BN, tile_rows);
+      const uint32_t id_us = make_idesc(false, true, p.BN, tile_rows);
+      const uint32_t id_uu = make_idesc(false, false, p.BN, tile_rows);
       const uint32_t dhi = smem_desc_hi(p.sbo, p.layout_type);
       const uint32_t ring_lo = smem_desc_lo(ring);
       const uint32_t stage_u = p.stage_bytes >> 4, a_u = p.a_bytes >> 4, b_u = p.b_bytes >> 4;
-      uint32_t it = 0, tile_iter = 0, ph = 0;
+      const uint32_t off_a1 = a_u, off_b0 = NAX * a_u, off_b1 = NAX * a_u + b_u;
+      const int ksteps = p.ksteps;
+      const uint32_t full_bar0 = smem_u32(&ctrl.full[0]), empty_bar0 = smem_u32(&ctrl.empty[0]);
+      uint32_t tile_iter = 0, ph = 0;
+      uint32_t a0 = ring_lo, full_bar = full_bar0, empty_bar = empty_bar0;
       int s = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, ++tile_iter) {
+      for (int t = worker; t < p.total_tiles && ok; t += workers, ++tile_iter) {
         const TileCoord tc = decode_tile(t, p);
         const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
         const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
-        if (!wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p)) { ok = false; break; }
+        TL_STAMP(1, tile_iter, 0);
+        if (!wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p, false)) { ok = false; break; }
         tc_fence_after();
+        TL_STAMP(1, tile_iter, 1);
         const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
         const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
-        for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb, ++it) {
-          if (!wait_bar(smem_u32(&ctrl.full[s]), ph, &ctrl, p)) { ok = false; break; }
+        uint32_t acc = 0u;
+        for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
+          if (!wait_bar(full_bar, ph, &ctrl, p, false)) { ok = false; break; }
           tc_fence_after();
-          // low descriptor words of the operand planes of this stage (16-byte units)
-          const uint32_t a0 = ring_lo + (uint32_t)s * stage_u;
-          const uint32_t a1 = a0 + a_u;
-          const uint32_t b0 = a0 + NAX * a_u;
-          const uint32_t b1 = b0 + b_u;
-          uint32_t acc = kb > tc.kb_begin ? 1u : 0u;
-          for (uint32_t ks = 0; ks < 2u * (uint32_t)p.ksteps; ks += 2u, acc = 1u) {   // 32 bytes per k-step
-            if (NAX == 2 && NBW == 2) {
-              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);          // hi*hi   weight 2^16
-              mma_i8(d1, a0 + ks, b1 + ks, dhi, id_su, acc);          // hi*lo   weight 2^8
-              mma_i8(d1, a1 + ks, b0 + ks, dhi, id_us, 1u);           // lo*hi   weight 2^8
-              mma_i8(d2, a1 + ks, b1 + ks, dhi, id_uu, acc);          // lo*lo   weight 1
-            } else if (NAX == 2 && NBW == 1) {
-              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);          // hi*w    weight 2^8
-              mma_i8(d1, a1 + ks, b0 + ks, dhi, id_us, acc);          // lo*w    weight 1
-            } else if (NAX == 1 && NBW == 2) {
-              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);          // x*hi    weight 2^8
-              mma_i8(d1, a0 + ks, b1 + ks, dhi, id_su, acc);          // x*lo    weight 1
-            } else {
-              mma_i8(d0, a0 + ks, b0 + ks, dhi, id_ss, acc);
-            }
+          // a0: low descriptor word of the first A plane of this stage; the other planes and the
+          // k-steps are fixed offsets (16-byte units) from it
+          mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0, a0 + off_a1, a0 + off_b0, a0 + off_b1, dhi, id_ss, id_su,
+                                    id_us, id_uu, acc);
+          if (ksteps > 1)
+            mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 2u, a0 + off_a1 + 2u, a0 + off_b0 + 2u, a0 + off_b1 + 2u,
+                                      dhi, id_ss, id_su, id_us, id_uu, 1u);
+          if (ksteps > 2) {
+            mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 4u, a0 + off_a1 + 4u, a0 + off_b0 + 4u, a0 + off_b1 + 4u,
+                                      dhi, id_ss, id_su, id_us, id_uu, 1u);
+            mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 6u, a0 + off_a1 + 6u, a0 + off_b0 + 6u, a0 + off_b1 + 6u,
+                                      dhi, id_ss, id_su, id_us, id_uu, 1u);
           }
-          tc_commit(smem_u32(&ctrl.empty[s]));                // stage reusable once these MMAs retire
-          if (++s == p.stages) { s = 0; ph ^= 1u; }
+          acc = 1u;
+          tc_commit<PAIR>(empty_bar);                          // stage reusable once these MMAs retire
+          a0 += stage_u;
+          full_bar += 8u;
+          empty_bar += 8u;
+          if (++s == p.stages) {
+            s = 0;
+            ph ^= 1u;
+            a0 = ring_lo;
+            full_bar = full_bar0;
+            empty_bar = empty_bar0;
+          }
         }
-        if (ok) tc_commit(smem_u32(&ctrl.tmem_full[buf]));    // accumulators of this tile complete
+        if (ok) tc_commit<PAIR>(smem_u32(&ctrl.tmem_full[buf]));   // accumulators of this tile complete
+        TL_STAMP(1, tile_iter, 2);
       }
       if (!ok || ctrl.abort) {
-        // make sure no MMA still reads shared memory or writes TMEM when the CTA tears down
-        tc_commit(smem_u32(&ctrl.drain));
+        // make sure no MMA still reads shared memory or writes TMEM when the CTAs tear down
+        tc_commit<false>(smem_u32(&ctrl.drain));
         const unsigned long long t0 = global_ns();
         while (!mbar_try_wait(smem_u32(&ctrl.drain), 0) && global_ns() - t0 < 50000000ull) {
         }
@@ -482,32 +668,38 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;          // TMEM lanes 32*quarter .. 32*quarter+31
-    const int ew = warp - 2;               // private bias staging slot
+    const int ew = warp - kFirstEpiWarp;   // private bias staging slot
+    // the two warps of a lane quarter split the columns of the tile
+    const int cols_per_warp = p.BN >= 64 ? p.BN / 2 : 32;
+    const int col_begin = (ew >> 2) * cols_per_warp;
+    const int col_end = min(p.BN, col_begin + cols_per_warp);
     long long* bias64 = ctrl.bias64[ew];
     uint32_t tile_iter = 0;
     Counts cnt;
     long long vmax = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, ++tile_iter) {
+    for (int t = worker; t < p.total_tiles && ok; t += workers, ++tile_iter) {
       const TileCoord tc = decode_tile(t, p);
       const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
       const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
       __syncwarp();
-      for (int c = lane; c < p.BN; c += 32) {
+      for (int c = col_begin + lane; c < col_end; c += 32) {
         const int n = tc.n0 + c;
         long long b = 0;
         if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
-        bias64[c] = b;
+        bias64[c - col_begin] = b;
       }
       __syncwarp();
+      if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 0);
       bool w = wait_bar(smem_u32(&ctrl.tmem_full[buf]), bph, &ctrl, p);
       w = __all_sync(0xffffffffu, w);
+      if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 1);
       if (!w) { ok = false; break; }
       tc_fence_after();
-      const int m = tc.m0 + quarter * 32 + lane;
+      const int m = tc.m0 + (int)rank * kBM + quarter * 32 + lane;
       const bool row_ok = m < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)(NACC * p.BN);
-      for (int c0 = 0; c0 < p.BN; c0 += 32) {
+      for (int c0 = col_begin; c0 < col_end; c0 += 32) {
         int32_t a0[32], a1[32], a2[32];
         tmem_ld32(taddr + c0, a0);
         if (NACC >= 2) tmem_ld32(taddr + p.BN + c0, a1);
@@ -531,24 +723,31 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             for (int j = 0; j < 16; ++j) {
               long long v = combine<NACC>(a0[16 * g + j], NACC >= 2 ? a1[16 * g + j] : 0,
                                           NACC == 3 ? a2[16 * g + j] : 0) +
-                            bias64[c0 + 16 * g + j];
+                            bias64[c0 - col_begin + 16 * g + j];
               if (p.rq.relu && v < 0) v = 0;
               v = v < 0 ? -v : v;
               if (row_ok && col + j < p.N) vmax = v > vmax ? v : vmax;
             }
           } else if (p.rq.relu) {
-            requant_store16<NACC, true>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + c0 + 16 * g, p, row_ok, m,
-                                        col, cnt);
+            requant_store16<NACC, true>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + (c0 - col_begin) + 16 * g, p,
+                                        row_ok, m, col, cnt);
           } else {
-            requant_store16<NACC, false>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + c0 + 16 * g, p, row_ok,
-                                         m, col, cnt);
+            requant_store16<NACC, false>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + (c0 - col_begin) + 16 * g, p,
+                                         row_ok, m, col, cnt);
           }
         }
       }
-      // accumulators of this buffer are in registers / memory: hand the buffer back
+      // accumulators of this buffer are in registers / memory: hand the buffer back to the leader
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctrl.tmem_empty[buf]));
+      if (lane == 0) {
+        const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
+        if (PAIR)
+          mbar_arrive_cluster(mapa_rank(bar, 0));
+        else
+          mbar_arrive(bar);
+      }
+      if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 2);
     }
     if (p.splits == 1) {
       if (p.mode == ADAPTION_MODE_RANGE)
@@ -560,9 +759,10 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (PAIR) cluster_sync_all();      // neither CTA leaves (or frees TMEM) while the other may still signal it
+  if (warp == kMmaWarp) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, p.tmem_cols);
+    tmem_dealloc<PAIR>(tmem_base, p.tmem_cols);
   }
 }
 
@@ -608,6 +808,8 @@ struct TcConfig {
   int num_kb = 0, splits = 1, kb_per_split = 0;
   int tiles_m = 0, tiles_n = 0;
   int cblks = 1;
+  bool pair = false;           // two CTAs per 256-row tile (cta_group::2)
+  int tile_m = kBM;
   size_t smem_bytes = 0;
   size_t workspace_bytes = 0;
 };
@@ -643,6 +845,8 @@ TcConfig make_config(const GemmProblem& g) {
   } else {
     if (g.K < 32) return c;
     c.BK = g.K >= 128 ? 128 : (g.K >= 64 ? 64 : 32);
+    const int forced_bk = env_int("ADAPTION_TC_BK", 0);   // experiment knob: narrower K-blocks
+    if ((forced_bk == 32 || forced_bk == 64) && forced_bk < c.BK) c.BK = forced_bk;
     c.num_kb = (int)((g.K + c.BK - 1) / c.BK);
     k_padded = g.K;
     if (g.K > (int64_t)1 << 30) return c;
@@ -653,14 +857,6 @@ TcConfig make_config(const GemmProblem& g) {
   c.BN = g.N <= 32 ? 32 : (g.N <= 64 ? 64 : 128);
   c.tiles_m = (int)((g.M + kBM - 1) / kBM);
   c.tiles_n = (int)((g.N + c.BN - 1) / c.BN);
-  c.a_bytes = (uint32_t)(kBM * c.BK);
-  c.b_bytes = (uint32_t)(c.BN * c.BK);
-  c.stage_bytes = c.nax * c.a_bytes + c.nbw * c.b_bytes;
-  const size_t budget = 232448 - sizeof(Ctrl) - 2048;
-  c.stages = (int)((budget - 1024) / c.stage_bytes);
-  if (c.stages > kMaxStages) c.stages = kMaxStages;
-  if (c.stages < 2) return c;
-  c.smem_bytes = (size_t)c.stages * c.stage_bytes + 1024;
   c.acc_bufs = 512 / (c.nacc * c.BN);
   if (c.acc_bufs > kMaxAccBufs) c.acc_bufs = kMaxAccBufs;
   if (c.acc_bufs < 1) return c;
@@ -688,6 +884,26 @@ TcConfig make_config(const GemmProblem& g) {
   if ((int64_t)c.kb_per_split * c.BK > kMaxKPerAccumulation) return c;
   if ((int64_t)tiles * c.splits > (int64_t)1 << 30) return c;
   c.workspace_bytes = c.splits > 1 ? (size_t)g.M * (size_t)g.N * sizeof(long long) : 0;
+  // Large unsplit problems run as CTA pairs: 256-row tiles, each CTA stages its own 128 rows of A
+  // and only half of the weight rows, which cuts the bytes (and TMA rows) per MAC by a quarter.
+  const int pair_env = env_int("ADAPTION_TC_PAIR", -1);
+  c.pair = c.splits == 1 && g.M >= 1024 && (sms % 2) == 0;
+  if (pair_env == 0) c.pair = false;
+  if (pair_env == 1 && c.splits == 1 && (sms % 2) == 0) c.pair = true;
+  if (c.pair) {
+    c.tile_m = 2 * kBM;
+    c.tiles_m = (int)((g.M + c.tile_m - 1) / c.tile_m);
+  }
+  c.a_bytes = (uint32_t)(kBM * c.BK);
+  c.b_bytes = (uint32_t)((c.pair ? c.BN / 2 : c.BN) * c.BK);
+  c.stage_bytes = c.nax * c.a_bytes + c.nbw * c.b_bytes;
+  const size_t budget = 232448 - sizeof(Ctrl) - 2048;
+  c.stages = (int)((budget - 1024) / c.stage_bytes);
+  if (c.stages > kMaxStages) c.stages = kMaxStages;
+  const int stage_cap = env_int("ADAPTION_TC_STAGES", 0);   // experiment knob: shallower ring
+  if (stage_cap >= 2 && stage_cap < c.stages) c.stages = stage_cap;
+  if (c.stages < 2) return c;
+  c.smem_bytes = (size_t)c.stages * c.stage_bytes + 1024;
   c.ok = true;
   return c;
 }
@@ -717,22 +933,156 @@ bool encode_im2col_nhwc(CUtensorMap* map, const void* base, const adaption_conv_
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NAX, int NBW>
+template <int NAX, int NBW, bool PAIR>
 int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem, cudaStream_t stream) {
-  static bool attr_set = false;
   static size_t attr_size = 0;
-  if (!attr_set || smem > attr_size) {
-    if (cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (smem > attr_size) {
+    if (cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
       return ADAPTION_ERR_CUDA;
-    attr_set = true;
     attr_size = smem;
   }
-  lp_gemm_kernel<NAX, NBW><<<grid, kThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], p);
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  if (PAIR) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  if (cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR>, maps[0], maps[1], maps[2], maps[3], p) !=
+      cudaSuccess) {
+    (void)cudaGetLastError();
+    return ADAPTION_ERR_CUDA;
+  }
   return cuda_status(cudaGetLastError());
 }
 
+template <int NAX, int NBW>
+int launch_either(bool pair, const CUtensorMap* maps, const TcParams& p, int grid, size_t smem,
+                  cudaStream_t stream) {
+  return pair ? launch_kernel<NAX, NBW, true>(maps, p, grid, smem, stream)
+              : launch_kernel<NAX, NBW, false>(maps, p, grid, smem, stream);
+}
+
+
+// ---------------------------------------------------------------------------------- peak probe
+// Issue-rate probe for the roofline denominator: every SM (or SM pair) runs back-to-back
+// tcgen05.mma kind::i8 instructions on operand tiles that stay resident in shared memory (no
+// loads), so the time per instruction is the tensor pipe's own.
+template <bool PAIR>
+__global__ void __launch_bounds__(128, 1)
+i8_peak_kernel(int bn, int iters, int commit_every, unsigned long long* out_cycles, int* out_status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ unsigned long long done_bar;
+  __shared__ unsigned long long side_bar;      // target of the optional intermediate commits
+  __shared__ uint32_t tmem_slot;
+  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  // A: 128 rows x 128 bytes, B: up to 256 rows x 128 bytes, filled with a fixed byte pattern
+  uint32_t* words = reinterpret_cast<uint32_t*>(smem_raw + (ring - smem_u32(smem_raw)));
+  for (int i = threadIdx.x; i < (16384 + 32768) / 4; i += blockDim.x) words[i] = 0x9E3779B9u * (uint32_t)(i + 1);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&done_bar), 1);
+    mbar_init(smem_u32(&side_bar), (1u << 20) - 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if ((threadIdx.x >> 5) == 0) {
+    tmem_alloc<PAIR>(smem_u32(&tmem_slot), 512);
+    tmem_relinquish<PAIR>();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (PAIR) cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+  if (threadIdx.x == 0 && rank == 0) {
+    const uint32_t idesc = make_idesc(true, true, bn, PAIR ? 256 : 128);
+    const uint32_t dhi = smem_desc_hi(1024, 2);
+    const uint32_t a_lo = smem_desc_lo(ring), b_lo = smem_desc_lo(ring + 16384);
+    const long long t0 = clock64();
+    for (int i = 0; i < iters; ++i) {
+#pragma unroll
+      for (uint32_t ks = 0; ks < 8; ks += 2) mma_i8<PAIR>(tmem_base, a_lo + ks, b_lo + ks, dhi, idesc, 1u);
+      // optional: an intermediate commit every `commit_every` groups of four instructions, as a
+      // pipelined mainloop issues when it hands a shared-memory stage back
+      if (commit_every > 0 && (i + 1) % commit_every == 0) tc_commit<PAIR>(smem_u32(&side_bar));
+    }
+    tc_commit<PAIR>(smem_u32(&done_bar));
+    const unsigned long long w0 = global_ns();
+    bool ok = true;
+    while (!mbar_try_wait(smem_u32(&done_bar), 0)) {
+      if (global_ns() - w0 > 2000000000ull) { ok = false; break; }
+    }
+    const long long t1 = clock64();
+    if (!ok) atomicExch(out_status, (int)ADAPTION_ERR_TIMEOUT);
+    out_cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (PAIR) cluster_sync_all();
+  if ((threadIdx.x >> 5) == 0) {
+    tc_fence_after();
+    tmem_dealloc<PAIR>(tmem_base, 512);
+  }
+}
+
+template <bool PAIR>
+int launch_peak(int bn, int iters, int commit_every, unsigned long long* d_cycles, int* d_status, int grid,
+                cudaStream_t stream) {
+  const size_t smem = 16384 + 32768 + 1024;
+  if (cudaFuncSetAttribute(i8_peak_kernel<PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+      cudaSuccess)
+    return ADAPTION_ERR_CUDA;
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  if (PAIR) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  if (cudaLaunchKernelEx(&cfg, i8_peak_kernel<PAIR>, bn, iters, commit_every, d_cycles, d_status) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ADAPTION_ERR_CUDA;
+  }
+  return ADAPTION_OK;
+}
+
 }  // namespace
+
+int probe_i8_peak(int bn, int pair, int iters, int commit_every, unsigned long long* d_cycles, int* d_status,
+                  cudaStream_t stream) {
+  const int sms = num_sms();
+  const int grid = pair ? (sms / 2) * 2 : sms;
+  return pair ? launch_peak<true>(bn, iters, commit_every, d_cycles, d_status, grid, stream)
+              : launch_peak<false>(bn, iters, commit_every, d_cycles, d_status, grid, stream);
+}
+
+namespace {
+
+}  // namespace
+
+#ifdef ADAPTION_TIMELINE
+extern "C" __attribute__((visibility("default"))) int adaption_debug_timeline(long long* h_out, int n) {
+  return cudaMemcpyFromSymbol(h_out, g_timeline, sizeof(long long) * (size_t)n) == cudaSuccess ? 0 : 6;
+}
+#endif
 
 bool tensor_path_supported(const GemmProblem& g) { return make_config(g).ok; }
 
@@ -758,14 +1108,14 @@ int launch_tensor(const GemmProblem& g) {
     if (!ok) return ADAPTION_ERR_CUDA;
     const uint64_t wk = g.is_conv ? (uint64_t)g.cs.R * g.cs.S * g.w.c_stride : (uint64_t)g.K;
     const uint64_t wpitch = g.is_conv ? wk : (uint64_t)g.w.c_stride;
-    if (!encode_tiled_2d(&maps[2 + i], wb[i], wk, (uint64_t)g.N, wpitch, (uint32_t)c.BK, (uint32_t)c.BN,
-                         c.swizzle))
+    if (!encode_tiled_2d(&maps[2 + i], wb[i], wk, (uint64_t)g.N, wpitch, (uint32_t)c.BK,
+                         (uint32_t)(c.pair ? c.BN / 2 : c.BN), c.swizzle))
       return ADAPTION_ERR_CUDA;
   }
 
   TcParams p;
   std::memset(&p, 0, sizeof(p));
-  p.M = (int)g.M; p.N = (int)g.N;
+  p.M = (int)g.M; p.N = (int)g.N; p.tile_m = c.tile_m;
   p.tiles_m = c.tiles_m; p.tiles_n = c.tiles_n; p.splits = c.splits;
   p.total_tiles = c.tiles_m * c.tiles_n * c.splits;
   p.num_kb = c.num_kb; p.kb_per_split = c.kb_per_split;
@@ -793,12 +1143,18 @@ int launch_tensor(const GemmProblem& g) {
   if (c.splits > 1) {
     if (cudaMemsetAsync(g.workspace, 0, c.workspace_bytes, g.stream) != cudaSuccess) return ADAPTION_ERR_CUDA;
   }
-  int grid = p.total_tiles < num_sms() ? p.total_tiles : num_sms();
+  int grid;
+  if (c.pair) {
+    const int pairs = num_sms() / 2;
+    grid = 2 * (p.total_tiles < pairs ? p.total_tiles : pairs);
+  } else {
+    grid = p.total_tiles < num_sms() ? p.total_tiles : num_sms();
+  }
   int rc;
-  if (c.nax == 2 && c.nbw == 2) rc = launch_kernel<2, 2>(maps, p, grid, c.smem_bytes, g.stream);
-  else if (c.nax == 2) rc = launch_kernel<2, 1>(maps, p, grid, c.smem_bytes, g.stream);
-  else if (c.nbw == 2) rc = launch_kernel<1, 2>(maps, p, grid, c.smem_bytes, g.stream);
-  else rc = launch_kernel<1, 1>(maps, p, grid, c.smem_bytes, g.stream);
+  if (c.nax == 2 && c.nbw == 2) rc = launch_either<2, 2>(c.pair, maps, p, grid, c.smem_bytes, g.stream);
+  else if (c.nax == 2) rc = launch_either<2, 1>(c.pair, maps, p, grid, c.smem_bytes, g.stream);
+  else if (c.nbw == 2) rc = launch_either<1, 2>(c.pair, maps, p, grid, c.smem_bytes, g.stream);
+  else rc = launch_either<1, 1>(c.pair, maps, p, grid, c.smem_bytes, g.stream);
   if (rc != ADAPTION_OK) return rc;
   if (c.splits > 1) return launch_finalize((const int64_t*)g.workspace, g.N, g);
   return ADAPTION_OK;

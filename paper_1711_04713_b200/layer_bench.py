@@ -145,9 +145,35 @@ def bench_stream(a) -> dict:
             "algorithmic_bytes": bytes_}
 
 
+def bench_peak(a) -> dict:
+    """Back-to-back int8 tensor-core instructions on resident operands (the roofline denominator)."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    out = {"kind": "peak", "iters": a.iters, "sms": sms, "configs": []}
+    for pair, bn, ce in [(False, 64, 0), (False, 128, 0), (False, 256, 0), (True, 64, 0), (True, 128, 0),
+                         (True, 256, 0), (False, 128, 4), (False, 128, 1), (True, 128, 4), (True, 128, 1)]:
+        if True:
+            cyc = torch.zeros(max(sms, 148), dtype=torch.int64, device="cuda")
+            st = torch.zeros(1, dtype=torch.int32, device="cuda")
+            n = 4096
+
+            def run():
+                B.adaption_probe_i8_peak(bn, pair, n, cyc, st, ce)
+
+            ms = _time(run, max(a.iters, 3))
+            if int(st.cpu()[0]) != 0:
+                raise B.AdaptionError(int(st.cpu()[0]), "peak probe")
+            c = cyc.cpu()
+            issuing = c[c > 0].double()
+            units = sms // 2 if pair else sms
+            macs = units * 4 * n * (256 if pair else 128) * bn * 32
+            out["configs"].append({"pair": pair, "bn": bn, "commit_every": ce, "cycles_per_mma": float(issuing.mean()) / (4 * n),
+                                   "int8_tops": 2.0 * macs / (ms / 1e3) / 1e12, "ms": ms})
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["conv", "ip", "range", "quantize", "act", "requant", "pool"])
+    ap.add_argument("kind", choices=["conv", "ip", "range", "quantize", "act", "requant", "pool", "peak"])
     ap.add_argument("--N", type=int, default=8)
     ap.add_argument("--H", type=int, default=28)
     ap.add_argument("--C", type=int, default=512)
@@ -173,6 +199,8 @@ def main():
         out = bench_conv(a)
     elif a.kind == "ip":
         out = bench_ip(a)
+    elif a.kind == "peak":
+        out = bench_peak(a)
     else:
         out = bench_stream(a)
     print(json.dumps(out), flush=True)

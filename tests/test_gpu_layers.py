@@ -155,14 +155,22 @@ TC_CONV = [
 ]
 
 
+@pytest.fixture(params=["single", "pair"])
+def cta_mode(request, monkeypatch):
+    """Run a tensor-core case with one CTA per 128-row tile and with CTA pairs on 256-row tiles
+    (cross-path identity: both must give the oracle's bits)."""
+    monkeypatch.setenv("ADAPTION_TC_PAIR", "1" if request.param == "pair" else "0")
+    return request.param
+
+
 @pytest.mark.parametrize("case", TC_CONV)
-def test_conv_tensor(case):
+def test_conv_tensor(case, cta_mode):
     N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu = case
     run_conv_case(np.random.default_rng(sum(case)), N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu,
                   B.ALGO_TENSOR)
 
 
-def test_conv_tensor_extreme_operands():
+def test_conv_tensor_extreme_operands(cta_mode):
     # every operand at +-full scale: largest possible partial sums in all three accumulators
     run_conv_case(np.random.default_rng(1), 1, 32, 32, 256, 128, 3, 1, 1, 16, 16, 16, False, B.ALGO_TENSOR,
                   extreme=True)
@@ -176,7 +184,7 @@ TC_IP = [(8, 800, 500, 16, 16, 16, True), (70, 1000, 260, 16, 16, 16, False), (2
 
 
 @pytest.mark.parametrize("case", TC_IP)
-def test_ip_tensor(case):
+def test_ip_tensor(case, cta_mode):
     Bsz, K, O, nx, nw, n_out, relu = case
     run_ip_case(np.random.default_rng(sum(case)), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_TENSOR)
 
