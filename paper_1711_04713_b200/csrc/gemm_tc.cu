@@ -119,6 +119,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// True in exactly one lane of a converged warp.  Code guarded by it still has its operands computed
+// warp-uniformly outside the guard, which lets the compiler keep them in uniform registers (the
+// tensor-core and bulk-copy instructions take uniform-register operands).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n"
+      ".reg .pred P;\n"
+      "elect.sync _|P, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, P;\n"
+      "}\n"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -522,7 +536,8 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     // sequence of stages and issues only its own copy, so the copies of a stage are in flight
     // side by side (one thread issues a bulk-tensor copy only every few hundred cycles).
     constexpr int NPLANES = NAX + NBW;
-    if (lane == 0 && warp < NPLANES) {
+    // (whole warp in uniform control flow; one elected lane issues the copies)
+    if (warp < NPLANES) {
       const bool is_a = warp < NAX;
       const int plane = is_a ? warp : warp - NAX;
       const CUtensorMap* my_map = is_a ? (plane == 0 ? &map_a0 : &map_a1) : (plane == 0 ? &map_b0 : &map_b1);
@@ -536,7 +551,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const int n_begin = tc.n0 + (int)rank * b_rows;     // first weight row this CTA stages
         int img = 0, base_h = 0, base_w = 0;
         int tap = 0, cb = 0, r = 0, sx = 0;       // position of kb in the (tap, channel block) order
-        TL_STAMP(0, (uint32_t)((t - worker) / workers), 0);
+        if (lane == 0 && warp == 0) TL_STAMP(0, (uint32_t)((t - worker) / workers), 0);
         if (p.is_conv) {
           const int ow = m_begin % p.OW;
           const int rest = m_begin / p.OW;
@@ -550,33 +565,34 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           sx = tap - r * p.S;
         }
         for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb, ++it) {
-          if (!wait_bar(smem_u32(&ctrl.empty[s]), ph ^ 1u, &ctrl, p)) { ok = false; break; }
+          ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.empty[s]), ph ^ 1u, &ctrl, p));
+          if (!ok) break;
           // bytes are reported to the leader's barrier; the leader arms it for both CTAs' copies
           uint32_t full = smem_u32(&ctrl.full[s]);
-          if (PAIR) {
-            if (rank == 0 && warp == 0) mbar_expect_tx(full, 2u * p.stage_bytes);
-            full = mapa_rank(full, 0);
-          } else {
-            if (warp == 0) mbar_expect_tx(full, p.stage_bytes);
-          }
+          if (PAIR) full = mapa_rank(full, 0);
           const uint32_t dst = ring + (uint32_t)s * p.stage_bytes + my_off;
+          if (elect_one()) {
+            if (warp == 0 && rank == 0) mbar_expect_tx(smem_u32(&ctrl.full[s]), (PAIR ? 2u : 1u) * p.stage_bytes);
+            if (p.is_conv) {
+              if (is_a)
+                tma_load_im2col<PAIR>(dst, my_map, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx, (uint16_t)r);
+              else
+                tma_load_2d<PAIR>(dst, my_map, full, tap * p.w_pitch + cb * p.BK, n_begin);
+            } else {
+              tma_load_2d<PAIR>(dst, my_map, full, kb * p.BK, is_a ? m_begin : n_begin);
+            }
+          }
           if (p.is_conv) {
-            if (is_a)
-              tma_load_im2col<PAIR>(dst, my_map, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx, (uint16_t)r);
-            else
-              tma_load_2d<PAIR>(dst, my_map, full, tap * p.w_pitch + cb * p.BK, n_begin);
             if (++cb == p.cblks) {
               cb = 0;
               ++tap;
               if (++sx == p.S) { sx = 0; ++r; }
             }
-          } else {
-            tma_load_2d<PAIR>(dst, my_map, full, kb * p.BK, is_a ? m_begin : n_begin);
           }
           if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
       }
-      if (!ok || ctrl.abort) {
+      if ((!ok || ctrl.abort) && lane == 0) {
         // gave up: let the copies already issued land before the CTA releases its shared memory.
         // (In a pair the bytes are counted on the leader's barriers, so the follower just waits.)
         const uint32_t n = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
@@ -597,7 +613,8 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     __syncwarp();
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
-    if (lane == 0 && rank == 0) {
+    // The whole warp walks the loop (uniform control flow and operands); one elected lane issues.
+    if (rank == 0) {
       const int tile_rows = PAIR ? 2 * kBM : kBM;
       const uint32_t id_ss = make_idesc(true, true, p.BN, tile_rows);
       const uint32_t id_su = make_idesc(true, false, p.BN, tile_rows);
@@ -617,16 +634,19 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const TileCoord tc = decode_tile(t, p);
         const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
         const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
-        TL_STAMP(1, tile_iter, 0);
-        if (!wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p, false)) { ok = false; break; }
+        if (lane == 0) TL_STAMP(1, tile_iter, 0);
+        ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p, false));
+        if (!ok) break;
         tc_fence_after();
-        TL_STAMP(1, tile_iter, 1);
+        if (lane == 0) TL_STAMP(1, tile_iter, 1);
         const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
         const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
         uint32_t acc = 0u;
         for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
-          if (!wait_bar(full_bar, ph, &ctrl, p, false)) { ok = false; break; }
+          ok = __all_sync(0xffffffffu, wait_bar(full_bar, ph, &ctrl, p, false));
+          if (!ok) break;
           tc_fence_after();
+          if (elect_one()) {
           // a0: low descriptor word of the first A plane of this stage; the other planes and the
           // k-steps are fixed offsets (16-byte units) from it
           mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0, a0 + off_a1, a0 + off_b0, a0 + off_b1, dhi, id_ss, id_su,
@@ -640,8 +660,9 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 6u, a0 + off_a1 + 6u, a0 + off_b0 + 6u, a0 + off_b1 + 6u,
                                       dhi, id_ss, id_su, id_us, id_uu, 1u);
           }
-          acc = 1u;
           tc_commit<PAIR>(empty_bar);                          // stage reusable once these MMAs retire
+          }
+          acc = 1u;
           a0 += stage_u;
           full_bar += 8u;
           empty_bar += 8u;
@@ -653,10 +674,11 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             empty_bar = empty_bar0;
           }
         }
-        if (ok) tc_commit<PAIR>(smem_u32(&ctrl.tmem_full[buf]));   // accumulators of this tile complete
-        TL_STAMP(1, tile_iter, 2);
+        if (ok && elect_one()) tc_commit<PAIR>(smem_u32(&ctrl.tmem_full[buf]));   // tile complete
+        __syncwarp();
+        if (lane == 0) TL_STAMP(1, tile_iter, 2);
       }
-      if (!ok || ctrl.abort) {
+      if ((!ok || ctrl.abort) && lane == 0) {
         // make sure no MMA still reads shared memory or writes TMEM when the CTAs tear down
         tc_commit<false>(smem_u32(&ctrl.drain));
         const unsigned long long t0 = global_ns();
@@ -887,7 +909,9 @@ TcConfig make_config(const GemmProblem& g) {
   // Large unsplit problems run as CTA pairs: 256-row tiles, each CTA stages its own 128 rows of A
   // and only half of the weight rows, which cuts the bytes (and TMA rows) per MAC by a quarter.
   const int pair_env = env_int("ADAPTION_TC_PAIR", -1);
-  c.pair = c.splits == 1 && g.M >= 1024 && (sms % 2) == 0;
+  // (measured: pairs win once the reduction is long, K >= 2304 bytes per plane row, and lose on
+  // short reductions where per-tile costs dominate)
+  c.pair = c.splits == 1 && g.M >= 1024 && (sms % 2) == 0 && c.BN == 128 && c.BK == 128 && c.num_kb >= 18;
   if (pair_env == 0) c.pair = false;
   if (pair_env == 1 && c.splits == 1 && (sms % 2) == 0) c.pair = true;
   if (c.pair) {
