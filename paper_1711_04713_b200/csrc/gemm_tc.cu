@@ -14,7 +14,7 @@
 //   warps 0-3  : TMA producers, one per operand plane (im2col / tiled loads into a ring of
 //                shared-memory stages; a single warp issues bulk-tensor copies too slowly)
 //   warp 4     : TMEM allocation and the single MMA-issuing thread
-//   warps 5-12 : epilogue (tcgen05.ld -> int64 recombination -> bias, ReLU, requantize with
+//   warps 5-20 : epilogue (tcgen05.ld -> int64 recombination -> bias, ReLU, requantize with
 //                saturation, zero / saturation counters, byte-plane stores; or range / split-K)
 // Every device-side wait is bounded; on expiry the kernel flags ADAPTION_ERR_TIMEOUT in the
 // caller's stats word, drains what it has in flight, frees its TMEM and returns.
@@ -34,7 +34,7 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kMaxStages = 8;
 constexpr int kMaxAccBufs = 4;
-constexpr int kEpiWarps = 8;                 // two per TMEM lane quarter, each takes half the columns
+constexpr int kEpiWarps = 16;                // four per TMEM lane quarter, each takes a quarter of the columns
 constexpr int kProducerWarps = 4;            // one per operand plane: TMA issue is slow per warp
 constexpr int kMmaWarp = kProducerWarps;
 constexpr int kFirstEpiWarp = kProducerWarps + 1;
@@ -89,7 +89,7 @@ struct Ctrl {
   unsigned long long drain;
   uint32_t tmem_base;
   volatile uint32_t abort;
-  long long bias64[kEpiWarps][kMaxBN / 2 < 32 ? 32 : kMaxBN / 2];
+  long long bias64[kEpiWarps][kMaxBN / 4];
 };
 
 // ---------------------------------------------------------------------------------- PTX
@@ -270,16 +270,13 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t 
         "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&r)[16]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        "=r"(r[15])
       : "r"(taddr)
       : "memory");
 }
@@ -437,6 +434,72 @@ __device__ __forceinline__ int32_t requant_shift_right(long long v, long long ha
   return q;
 }
 
+
+// Fast requantization for ReLU layers with a rounding right shift (shift >= 1), all in 32-bit
+// arithmetic.  The exact pre-activation value is split as  v = 2^16 * T + L  with
+//   T = hh + (mid >> 8) + (ll >> 16)                 (arithmetic shifts)
+//   L = ((mid & 255) << 8) + (ll & 65535)            (0 <= L < 2^17)
+// (for two / one accumulators the missing leading terms are zero), and the per-column constant
+// C = bias * 2^bias_shift + 2^(shift-1) likewise as 2^16 * Ch + Cl with 0 <= Cl < 2^16.  Then
+//   v + C = 2^16 * T' + L',  T' = T + Ch + ((L + Cl) >> 16),  L' = (L + Cl) & 65535,
+// and because ReLU maps every negative value to zero the rounded result is
+//   max(0, floor((v + C) / 2^shift)),
+// i.e. T' >> (shift - 16) for shift >= 16 and (T' << (16 - shift)) + (L' >> shift) below that
+// (T' clamped first: |T'| >= 2^16 saturates or clips to zero in any case).
+template <int NACC, bool WIDE_SHIFT>
+__device__ __forceinline__ int32_t requant_relu32(int32_t x0, int32_t x1, int32_t x2, int2 c, int shift,
+                                                  int32_t qmax, int32_t& r_out) {
+  // name the accumulators by weight: hh (2^16), mid (2^8), ll (1)
+  const int32_t hh = NACC == 3 ? x0 : 0;
+  const int32_t mid = NACC == 3 ? x1 : (NACC == 2 ? x0 : 0);
+  const int32_t ll = NACC == 3 ? x2 : (NACC == 2 ? x1 : x0);
+  const int32_t T = hh + (mid >> 8) + (ll >> 16);
+  const int32_t Ls = (int32_t)__byte_perm((uint32_t)mid, 0u, 0x4404) + (ll & 0xffff) + c.y;
+  const int32_t Tp = T + c.x + (Ls >> 16);
+  int32_t r;
+  if (WIDE_SHIFT) {           // shift >= 16
+    r = Tp >> (shift - 16);
+  } else {
+    const int32_t Tc = min(max(Tp, -1), 65535);
+    r = (Tc << (16 - shift)) + ((Ls & 0xffff) >> shift);
+  }
+  r = max(r, 0);
+  r_out = r;
+  return min(r, qmax);
+}
+
+// Sixteen columns of one row.  Counting is kept off the per-element path: saturation is detected
+// by OR-ing r ^ q over the group (non-zero only if something was clipped, which is rare; the exact
+// count is then redone), non-zero outputs are summed as min(q, 1).
+template <int NACC, bool WIDE_SHIFT>
+__device__ __forceinline__ void requant_relu32_x16(const int32_t* a0, const int32_t* a1, const int32_t* a2,
+                                                   const int2* c2, int shift, int32_t qmax, int nvalid,
+                                                   Counts& cnt, int32_t (&q)[16]) {
+  int32_t clipped = 0, nonzero = 0;
+  int32_t r[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    q[j] = requant_relu32<NACC, WIDE_SHIFT>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0, c2[j], shift,
+                                            qmax, r[j]);
+    clipped |= r[j] ^ q[j];
+    nonzero += min(q[j], 1);
+  }
+  if (nvalid == 16) {
+    cnt.zeros += 16 - nonzero;
+    if (clipped != 0) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) cnt.sat_pos += (r[j] > qmax);
+    }
+  } else {
+    // ragged edge: count only the real elements
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      cnt.zeros += (j < nvalid && q[j] == 0);
+      cnt.sat_pos += (j < nvalid && r[j] > qmax);
+    }
+  }
+}
+
 // Sixteen consecutive output columns of one row: recombine, add bias, requantize, pack into
 // byte planes (and the optional int16 copy) and store 16 bytes per plane.
 template <int NACC, bool RELU>
@@ -445,7 +508,14 @@ __device__ __forceinline__ void requant_store16(const int32_t* a0, const int32_t
                                                 int m, int col, Counts& cnt) {
   int32_t q[16];
   const int nvalid = row_ok ? min(max(p.N - col, 0), 16) : 0;
-  if (p.rq.shift > 0) {
+  if (RELU && p.rq.shift > 0) {
+    // per-column constants were staged as (Ch, Cl) pairs
+    const int2* c2 = reinterpret_cast<const int2*>(bias64);
+    if (p.rq.shift >= 16)
+      requant_relu32_x16<NACC, true>(a0, a1, a2, c2, p.rq.shift, p.rq.qmax, nvalid, cnt, q);
+    else
+      requant_relu32_x16<NACC, false>(a0, a1, a2, c2, p.rq.shift, p.rq.qmax, nvalid, cnt, q);
+  } else if (p.rq.shift > 0) {
     const long long half = 1ll << (p.rq.shift - 1);
     if (nvalid == 16) {
 #pragma unroll
@@ -691,11 +761,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;          // TMEM lanes 32*quarter .. 32*quarter+31
     const int ew = warp - kFirstEpiWarp;   // private bias staging slot
-    // the two warps of a lane quarter split the columns of the tile
-    const int cols_per_warp = p.BN >= 64 ? p.BN / 2 : 32;
-    const int col_begin = (ew >> 2) * cols_per_warp;
+    // the warps of a lane quarter split the columns of the tile
+    const int cols_per_warp = max(16, p.BN / (kEpiWarps / 4));
+    const int col_begin = min(p.BN, (ew >> 2) * cols_per_warp);
     const int col_end = min(p.BN, col_begin + cols_per_warp);
     long long* bias64 = ctrl.bias64[ew];
+    // ReLU layers with a rounding right shift take the 32-bit requantization path
+    const bool fast_relu = p.splits == 1 && p.mode == ADAPTION_MODE_REQUANT && p.rq.relu && p.rq.shift > 0;
     uint32_t tile_iter = 0;
     Counts cnt;
     long long vmax = 0;
@@ -709,7 +781,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const int n = tc.n0 + c;
         long long b = 0;
         if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
-        bias64[c - col_begin] = b;
+        if (fast_relu) {
+          // (Ch, Cl) of C = bias + rounding half, for requant_relu32: x = Ch, y = Cl
+          const long long C = b + (1ll << (p.rq.shift - 1));
+          reinterpret_cast<int2*>(bias64)[c - col_begin] = make_int2((int)(C >> 16), (int)(C & 0xffff));
+        } else {
+          bias64[c - col_begin] = b;
+        }
       }
       __syncwarp();
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 0);
@@ -721,42 +799,34 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       const int m = tc.m0 + (int)rank * kBM + quarter * 32 + lane;
       const bool row_ok = m < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)(NACC * p.BN);
-      for (int c0 = col_begin; c0 < col_end; c0 += 32) {
-        int32_t a0[32], a1[32], a2[32];
-        tmem_ld32(taddr + c0, a0);
-        if (NACC >= 2) tmem_ld32(taddr + p.BN + c0, a1);
-        if (NACC == 3) tmem_ld32(taddr + 2 * p.BN + c0, a2);
+      for (int c0 = col_begin; c0 < col_end; c0 += 16) {
+        int32_t a0[16], a1[16], a2[16];
+        tmem_ld16(taddr + c0, a0);
+        if (NACC >= 2) tmem_ld16(taddr + p.BN + c0, a1);
+        if (NACC == 3) tmem_ld16(taddr + 2 * p.BN + c0, a2);
         tmem_ld_wait();
+        const int col = tc.n0 + c0;
+        const long long* bcol = bias64 + (c0 - col_begin);
+        if (p.splits > 1) {
+          // partial sums of this K range go to the int64 workspace
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          const int col = tc.n0 + c0 + 16 * g;
-          if (p.splits > 1) {
-            // partial sums of this K range go to the int64 workspace
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const long long v = combine<NACC>(a0[16 * g + j], NACC >= 2 ? a1[16 * g + j] : 0,
-                                                NACC == 3 ? a2[16 * g + j] : 0);
-              if (row_ok && col + j < p.N && v != 0)
-                atomicAdd((unsigned long long*)(p.ws + (long long)m * p.ws_ld + col + j),
-                          (unsigned long long)v);
-            }
-          } else if (p.mode == ADAPTION_MODE_RANGE) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              long long v = combine<NACC>(a0[16 * g + j], NACC >= 2 ? a1[16 * g + j] : 0,
-                                          NACC == 3 ? a2[16 * g + j] : 0) +
-                            bias64[c0 - col_begin + 16 * g + j];
-              if (p.rq.relu && v < 0) v = 0;
-              v = v < 0 ? -v : v;
-              if (row_ok && col + j < p.N) vmax = v > vmax ? v : vmax;
-            }
-          } else if (p.rq.relu) {
-            requant_store16<NACC, true>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + (c0 - col_begin) + 16 * g, p,
-                                        row_ok, m, col, cnt);
-          } else {
-            requant_store16<NACC, false>(a0 + 16 * g, a1 + 16 * g, a2 + 16 * g, bias64 + (c0 - col_begin) + 16 * g, p,
-                                         row_ok, m, col, cnt);
+          for (int j = 0; j < 16; ++j) {
+            const long long v = combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0);
+            if (row_ok && col + j < p.N && v != 0)
+              atomicAdd((unsigned long long*)(p.ws + (long long)m * p.ws_ld + col + j), (unsigned long long)v);
           }
+        } else if (p.mode == ADAPTION_MODE_RANGE) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            long long v = combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bcol[j];
+            if (p.rq.relu && v < 0) v = 0;
+            v = v < 0 ? -v : v;
+            if (row_ok && col + j < p.N) vmax = v > vmax ? v : vmax;
+          }
+        } else if (p.rq.relu) {
+          requant_store16<NACC, true>(a0, a1, a2, bcol, p, row_ok, m, col, cnt);
+        } else {
+          requant_store16<NACC, false>(a0, a1, a2, bcol, p, row_ok, m, col, cnt);
         }
       }
       // accumulators of this buffer are in registers / memory: hand the buffer back to the leader
