@@ -184,6 +184,7 @@ def run_gpu(args):
 
     from paper_1711_04713_b200 import binding as B
     from paper_1711_04713_b200 import build as bld
+    from paper_1711_04713_b200 import replicas
     from paper_1711_04713_b200 import workloads as wl
     from paper_1711_04713_b200.network import LPNetwork
 
@@ -208,7 +209,7 @@ def run_gpu(args):
     specs = wl.vgg16_specs()
     params = wl.make_params(specs, seed=0)
     batch = args.batch
-    x_host = torch.from_numpy(wl.vgg16_input(batch, seed=100 + rank).reshape(-1, 3)).pin_memory()
+    x_host = torch.from_numpy(wl.vgg16_input(batch, seed=replicas.shard_seed(100, rank)).reshape(-1, 3)).pin_memory()
     x_dev = x_host.cuda()
     net = LPNetwork(params, batch, (224, 224), 3, args.n_bits)
     del params
@@ -270,12 +271,9 @@ def run_gpu(args):
         dist.barrier()
     elapsed_ms = t0.elapsed_time(t1)
     clocks = sampler.stop(wall0, wall1) if rank == 0 else {}
-    if dist is not None:
-        tt = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt[0])
+    elapsed_ms = replicas.slowest_rank_ms(elapsed_ms, device="cuda")
     ms_per_step = elapsed_ms / args.steps
-    ips = world * batch / (ms_per_step / 1e3)
+    ips = replicas.whole_job_rate(batch, world, ms_per_step)
     eff_tops = 2.0 * macs_step * world / (ms_per_step / 1e3) / 1e12
 
     # ---- per-launch durations of the dominant kernel (the tensor-core layer GEMM), from the
@@ -303,6 +301,27 @@ def run_gpu(args):
         "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
         "share_of_step": gemm_ms / elapsed_ms if world == 1 else None,
     }
+    # the library's own issue-rate probe: back-to-back int8 MMAs on resident operands (context for
+    # the denominator above, which follows the measured bf16 figure)
+    try:
+        cyc = torch.zeros(256, dtype=torch.int64, device="cuda")
+        pst = torch.zeros(1, dtype=torch.int32, device="cuda")
+        n_probe = 4096
+        for _ in range(2):
+            B.adaption_probe_i8_peak(128, False, n_probe, cyc, pst)
+        torch.cuda.synchronize()
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pe0.record()
+        B.adaption_probe_i8_peak(128, False, n_probe, cyc, pst)
+        pe1.record()
+        torch.cuda.synchronize()
+        sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        probe_tops = 2.0 * sms * 4 * n_probe * 128 * 128 * 32 / (pe0.elapsed_time(pe1) / 1e3) / 1e12
+        roofline["int8_probe_tops"] = probe_tops
+        roofline["frac_of_int8_probe"] = achieved_tops / (probe_tops / planes)
+    except Exception as exc:  # the probe is context only
+        roofline["int8_probe_tops"] = None
+        roofline["int8_probe_error"] = str(exc)
     layer_table = {k: {"ms": statistics.mean(v)} for k, v in per_layer.items()}
     for L in gemm_layers:
         layer_table[L.name]["tops"] = 2.0 * L.macs / (layer_table[L.name]["ms"] / 1e3) / 1e12
@@ -330,11 +349,8 @@ def run_gpu(args):
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tt = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt[0])
-    e2e_ips = world * batch / (e2e_ms / e2e_steps / 1e3)
+    e2e_ms = replicas.slowest_rank_ms(e2e_ms, device="cuda")
+    e2e_ips = replicas.whole_job_rate(batch, world, e2e_ms / e2e_steps)
     h2d = x_host.numel() * 4
     d2h = out.lo.numel() + (out.hi.numel() if out.hi is not None else 0)
 
