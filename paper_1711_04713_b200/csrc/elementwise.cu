@@ -83,33 +83,55 @@ __global__ void choose_fmt_kernel(const float* __restrict__ d_max_abs, int32_t n
 // the tie rule is applied on the exact fractional part (trunc + exact remainder), never on a
 // rounded sum.
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ int32_t quantize_f32(float x, float scale, int relu, int32_t qmin,
+// `scale2` is 2^(f+1): z = trunc(2 * x * 2^f) is taken with the saturating float->int conversion
+// (NaN -> 0, +-Inf and anything beyond int32 -> INT_MAX / INT_MIN), and the nearest integer with
+// ties away from zero is sign(z) * ((|z| + 1) >> 1): for 2y = n + e, 0 <= e < 1,
+// floor(y + 1/2) = floor((n + 1) / 2 + e / 2) = (n + 1) >> 1 because (n + 1) / 2 is an integer or a
+// half-integer and e / 2 < 1/2.  Only integer work follows the one conversion.
+__device__ __forceinline__ int32_t quantize_f32(float x, float scale2, int relu, int32_t qmin,
                                                 int32_t qmax, bool counted, Counts& c) {
-  float y = x * scale;
-  int32_t r;
-  if (y != y) {
-    r = 0;  // NaN
-  } else {
-    if (relu && y < 0.0f) y = 0.0f;
-    y = fminf(fmaxf(y, -131072.0f), 131072.0f);  // keeps every in-range value, saturates the rest
-    const float t = truncf(y);
-    const float frac = y - t;  // exact
-    r = (int32_t)t;
-    if (fabsf(frac) >= 0.5f) r += (y > 0.0f) ? 1 : -1;
-  }
-  if (r > qmax) {
-    r = qmax;
-    c.sat_pos += counted;
-  } else if (r < qmin) {
-    r = qmin;
-    c.sat_neg += counted;
-  }
-  c.zeros += (counted && r == 0);
-  return r;
+  int32_t z = __float2int_rz(x * scale2);
+  if (relu) z = max(z, 0);
+  const uint32_t a = (uint32_t)(z < 0 ? -(long long)z : (long long)z);   // |z| up to 2^31
+  const int32_t mag = (int32_t)((a + 1u) >> 1);                          // <= 2^30
+  const int32_t r = z < 0 ? -mag : mag;
+  const int32_t q = min(max(r, qmin), qmax);
+  c.sat_pos += (counted && r > qmax);
+  c.sat_neg += (counted && r < qmin);
+  c.zeros += (counted && q == 0);
+  return q;
 }
 
+// Four elements at once for the dense kernel; the counters are derived per group (clipping is
+// detected by OR-ing r ^ q and only then counted exactly).
+__device__ __forceinline__ void quantize_f32x4(const float4 v, float scale2, int relu, int32_t qmin,
+                                               int32_t qmax, Counts& c, int32_t (&q)[4]) {
+  const float x[4] = {v.x, v.y, v.z, v.w};
+  int32_t r[4], clipped = 0, nonzero = 0;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    int32_t z = __float2int_rz(x[k] * scale2);
+    if (relu) z = max(z, 0);
+    const uint32_t a = (uint32_t)(z < 0 ? -(long long)z : (long long)z);
+    const int32_t mag = (int32_t)((a + 1u) >> 1);
+    r[k] = z < 0 ? -mag : mag;
+    q[k] = min(max(r[k], qmin), qmax);
+    clipped |= r[k] ^ q[k];
+    nonzero += min(abs(q[k]), 1);
+  }
+  c.zeros += 4 - nonzero;
+  if (clipped != 0) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      c.sat_pos += (r[k] > qmax);
+      c.sat_neg += (r[k] < qmin);
+    }
+  }
+}
+
+// 2^(frac_bits + 1), the scale quantize_f32 expects
 __device__ __forceinline__ float scale_of(int32_t frac_bits) {
-  return __int_as_float((127 + frac_bits) << 23);
+  return __int_as_float((128 + frac_bits) << 23);
 }
 
 struct QuantOut {
@@ -155,18 +177,15 @@ __global__ void __launch_bounds__(256) quantize_flat_kernel(const float4* __rest
     for (int u = 0; u < 4; ++u) v[u] = __ldcs(x + i + u * nthreads);
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      store4(out, i + u * nthreads, quantize_f32(v[u].x, scale, relu, qmin, qmax, true, c),
-             quantize_f32(v[u].y, scale, relu, qmin, qmax, true, c),
-             quantize_f32(v[u].z, scale, relu, qmin, qmax, true, c),
-             quantize_f32(v[u].w, scale, relu, qmin, qmax, true, c));
+      int32_t q[4];
+      quantize_f32x4(v[u], scale, relu, qmin, qmax, c, q);
+      store4(out, i + u * nthreads, q[0], q[1], q[2], q[3]);
     }
   }
   for (; i < n4; i += nthreads) {
-    const float4 v = __ldcs(x + i);
-    store4(out, i, quantize_f32(v.x, scale, relu, qmin, qmax, true, c),
-           quantize_f32(v.y, scale, relu, qmin, qmax, true, c),
-           quantize_f32(v.z, scale, relu, qmin, qmax, true, c),
-           quantize_f32(v.w, scale, relu, qmin, qmax, true, c));
+    int32_t q[4];
+    quantize_f32x4(__ldcs(x + i), scale, relu, qmin, qmax, c, q);
+    store4(out, i, q[0], q[1], q[2], q[3]);
   }
   if (stats != nullptr) flush_counts_warp(c, stats);
 }
@@ -198,6 +217,23 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restr
     store4(out, g, q[0], q[1], q[2], q[3]);
   }
   if (stats != nullptr) flush_counts_warp(c, stats);
+}
+
+// Requantization of a stored value (|v| <= 2^15, |shift| <= 15): everything fits in 32 bits.
+__device__ __forceinline__ int32_t requant_small(int32_t v, const RequantParams& rq, bool counted, Counts& c) {
+  if (rq.relu) v = max(v, 0);
+  int32_t r;
+  if (rq.shift > 0) {
+    const int32_t mag = (abs(v) + (1 << (rq.shift - 1))) >> rq.shift;
+    r = v < 0 ? -mag : mag;
+  } else {
+    r = v * (1 << (-rq.shift));
+  }
+  const int32_t q = min(max(r, rq.qmin), rq.qmax);
+  c.sat_pos += (counted && r > rq.qmax);
+  c.sat_neg += (counted && r < rq.qmin);
+  c.zeros += (counted && q == 0);
+  return q;
 }
 
 // Format conversion of a stored fixed-point tensor (LPAct on quantized values): optional ReLU,
@@ -235,9 +271,47 @@ __global__ void __launch_bounds__(256) requant_rows_kernel(const uint32_t* __res
       else
         v = (int32_t)(int8_t)l;
       const bool real = c0 + u < inner;
-      q[u] = requant_value(real ? (int64_t)v : 0, rq, real, c);
+      q[u] = requant_small(real ? v : 0, rq, real, c);
     }
     store4(out, g, q[0], q[1], q[2], q[3]);
+  }
+  if (stats != nullptr) flush_counts_warp(c, stats);
+}
+
+// Dense rows on both sides (pitch == inner extent, no int16 copy): the tensor is one flat array,
+// sixteen elements (one 16-byte vector per plane) per thread and step, no index arithmetic.
+__global__ void __launch_bounds__(256) requant_flat_kernel(const uint4* __restrict__ in_hi,
+                                                           const uint4* __restrict__ in_lo, size_t n16,
+                                                           uint4* __restrict__ out_hi, uint4* __restrict__ out_lo,
+                                                           int32_t in_frac_bits, int32_t out_frac_bits,
+                                                           const adaption_qfmt* __restrict__ d_fmt,
+                                                           RequantParams rq, adaption_stats* __restrict__ stats) {
+  if (d_fmt != nullptr) out_frac_bits = d_fmt->frac_bits;
+  rq.shift = in_frac_bits - out_frac_bits;
+  Counts c;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += nthreads) {
+    const uint4 lo = __ldcs(in_lo + i);
+    const uint4 hi = in_hi != nullptr ? __ldcs(in_hi + i) : make_uint4(0, 0, 0, 0);
+    const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
+    uint32_t olo[4], ohi[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      uint32_t pl = 0, ph = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int32_t l = (lw[w] >> (8 * b)) & 255;
+        const int32_t v = in_hi != nullptr ? ((int32_t)(int8_t)((hw[w] >> (8 * b)) & 255)) * 256 + l
+                                           : (int32_t)(int8_t)l;
+        const int32_t q = requant_small(v, rq, true, c);
+        pl |= (uint32_t)(q & 255) << (8 * b);
+        ph |= (uint32_t)((q >> 8) & 255) << (8 * b);
+      }
+      olo[w] = pl;
+      ohi[w] = ph;
+    }
+    out_lo[i] = make_uint4(olo[0], olo[1], olo[2], olo[3]);
+    if (rq.out_planes == 2) out_hi[i] = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
   }
   if (stats != nullptr) flush_counts_warp(c, stats);
 }
@@ -389,6 +463,14 @@ int requant_impl(const adaption_qtensor& in, size_t outer, size_t inner, int32_t
   if (rc != ADAPTION_OK) return rc;
   if (outer == 0 || inner == 0) return ADAPTION_OK;
   RequantParams rq = make_requant(in.fmt.frac_bits, out.fmt, relu);
+  if ((int64_t)inner == in.c_stride && in.c_stride == out.c_stride && out.q16 == nullptr) {
+    const size_t n16 = outer * inner / 16;
+    requant_flat_kernel<<<stream_grid(n16, 256, 8), 256, 0, stream>>>(
+        in.fmt.n_bits > 8 ? reinterpret_cast<const uint4*>(in.hi) : nullptr,
+        reinterpret_cast<const uint4*>(in.lo), n16, reinterpret_cast<uint4*>(out.hi),
+        reinterpret_cast<uint4*>(out.lo), in.fmt.frac_bits, out.fmt.frac_bits, d_fmt, rq, d_stats);
+    return cuda_status(cudaGetLastError());
+  }
   const size_t groups = outer * (size_t)(out.c_stride / 4);
   const int grid = stream_grid(groups, 256, 8);
   requant_rows_kernel<<<grid, 256, 0, stream>>>(
