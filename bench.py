@@ -30,8 +30,27 @@ if ROOT not in sys.path:
 METRIC = "effective fixed-point TOPS & images/s for VGG16 16-bit forward; % of INT8 peak"
 INT8_NOMINAL_TOPS = 4500.0          # dense INT8, datasheet
 NOMINAL_INT8_OVER_BF16 = 2.0        # nominal dense INT8 : bf16 ratio (4.5 : 2.25 POPS)
+# DRAM traffic of the layer GEMM per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged
+# over the 16 layer launches of a forward pass of this workload), from the ncu launch list summarised
+# in profiles/bench_vgg16_b64_launch_list.md.  Valid only for the kernel source it was taken on.
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 177.5e6
+GEMM_TRAFFIC_SOURCE_SHA1 = "f37fa4455bc8"
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_BF16_SUSTAINED = 1400.0
+
+
+def gemm_traffic(n_bits: int, batch: int):
+    """The captured traffic figure, or None once the kernel source differs from the captured one
+    (or for a workload other than the captured one)."""
+    import hashlib
+    try:
+        src = os.path.join(ROOT, "paper_1711_04713_b200", "csrc", "gemm_tc.cu")
+        sha = hashlib.sha1(open(src, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if not sha.startswith(GEMM_TRAFFIC_SOURCE_SHA1) or n_bits != 16 or batch != 64:
+        return None
+    return GEMM_TRAFFIC_BYTES_PER_LAUNCH
 
 
 def read_peaks():
@@ -293,7 +312,7 @@ def run_gpu(args):
     roofline = {
         "bound": "tensor", "kernel": "lp_gemm_kernel (all LPConvolution / LPInnerProduct launches)",
         "achieved": achieved_tops, "peak": peak, "unit": "TFLOP/s", "frac": achieved_tops / peak,
-        "traffic": None,
+        "traffic": gemm_traffic(args.n_bits, batch), "traffic_unit": "bytes per launch (DRAM read + write)",
         "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']} x{NOMINAL_INT8_OVER_BF16:g} "
                        f"(nominal INT8:bf16) / {planes:g} int8 products per {args.n_bits}-bit MAC",
         "frac_of_burst": achieved_tops / (peaks["bf16_burst"] * NOMINAL_INT8_OVER_BF16 / planes),
