@@ -32,7 +32,7 @@ int num_sms();
 namespace {
 
 constexpr int kBM = 128;
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 12;
 constexpr int kMaxAccBufs = 4;
 constexpr int kEpiWarps = 16;                // four per TMEM lane quarter, each takes a quarter of the columns
 constexpr int kProducerWarps = 4;            // one per operand plane: TMA issue is slow per warp
@@ -53,6 +53,14 @@ struct TcParams {
   uint32_t sbo, layout_type;
   int stages;
   uint32_t a_bytes, b_bytes, stage_bytes;
+  // a stage holds `kps` consecutive k-blocks of `kb_bytes` each (short k-blocks are grouped so
+  // that the per-stage hand-shake is amortised over enough MMAs)
+  int kps;
+  uint32_t kb_bytes;
+  // weights resident in shared memory (one column tile, short reduction): the ring then holds
+  // only activation planes and all weight k-blocks are loaded once per CTA at this offset
+  int b_resident;
+  uint32_t b_res_off;
   int acc_bufs;
   uint32_t tmem_cols;
   int is_conv, OH, OW, S, cblks, w_pitch, stride_h, stride_w, pad_h, pad_w;
@@ -87,6 +95,7 @@ struct Ctrl {
   unsigned long long tmem_full[kMaxAccBufs];
   unsigned long long tmem_empty[kMaxAccBufs];
   unsigned long long drain;
+  unsigned long long b_ready;   // resident weights have landed
   uint32_t tmem_base;
   volatile uint32_t abort;
   long long bias64[kEpiWarps][kMaxBN / 4];
@@ -557,7 +566,9 @@ __device__ __forceinline__ void requant_store16(const int32_t* a0, const int32_t
 }
 
 // ---------------------------------------------------------------------------------- kernel
-template <int NAX, int NBW, bool PAIR>
+// GROUPED: stages hold several k-blocks and / or the weights are resident in shared memory (short
+// reductions); the plain variant keeps the issue loops free of that bookkeeping.
+template <int NAX, int NBW, bool PAIR, bool GROUPED>
 __global__ void __launch_bounds__(kThreads, 1)
 lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
@@ -587,6 +598,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       mbar_init(smem_u32(&ctrl.tmem_empty[b]), PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
     mbar_init(smem_u32(&ctrl.drain), 1);
+    mbar_init(smem_u32(&ctrl.b_ready), 1);
     ctrl.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -607,15 +619,41 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     // side by side (one thread issues a bulk-tensor copy only every few hundred cycles).
     constexpr int NPLANES = NAX + NBW;
     // (whole warp in uniform control flow; one elected lane issues the copies)
-    if (warp < NPLANES) {
-      const bool is_a = warp < NAX;
-      const int plane = is_a ? warp : warp - NAX;
+    // Planes that are streamed through the ring: all of them, or only the activation planes when
+    // the weights are resident.  The four producer warps are spread over these planes; with
+    // several warps per plane they take turns stage by stage, because one warp cannot issue
+    // copies fast enough for short stages.
+    const bool b_res = GROUPED && !PAIR && p.b_resident;
+    const int nact = b_res ? NAX : NPLANES;
+    const int kps = GROUPED ? p.kps : 1;
+    const int nsub = kProducerWarps / nact;            // warps per streamed plane
+    const int act_plane = warp % nact, sub = warp / nact;
+    {
+      const bool is_a = act_plane < NAX;
+      const int plane = is_a ? act_plane : act_plane - NAX;
       const CUtensorMap* my_map = is_a ? (plane == 0 ? &map_a0 : &map_a1) : (plane == 0 ? &map_b0 : &map_b1);
       const uint32_t my_off = is_a ? (uint32_t)plane * p.a_bytes : NAX * p.a_bytes + (uint32_t)plane * p.b_bytes;
       uint32_t it = 0, ph = 0;
       int s = 0;
       bool ok = true;
-      for (int t = worker; t < p.total_tiles && ok; t += workers) {
+      if (b_res && warp >= NAX && warp < NPLANES) {
+        // the whole weight matrix of this (single) column tile, one copy per k-block and plane,
+        // all reporting to one barrier
+        const int bplane = warp - NAX;
+        if (elect_one()) {
+          const uint32_t bar = smem_u32(&ctrl.b_ready);
+          if (bplane == 0) mbar_expect_tx(bar, (uint32_t)p.num_kb * NBW * p.b_bytes);
+          for (int kb = 0; kb < p.num_kb; ++kb) {
+            const uint32_t dst =
+                ring + p.b_res_off + (uint32_t)kb * (NBW * p.b_bytes) + (uint32_t)bplane * p.b_bytes;
+            const int kcol = p.is_conv ? (kb / p.cblks) * p.w_pitch + (kb % p.cblks) * p.BK : kb * p.BK;
+            tma_load_2d<false>(dst, bplane == 0 ? &map_b0 : &map_b1, bar, kcol, 0);
+          }
+        }
+        __syncwarp();
+      }
+      const bool in_tile_loop = sub < nsub;
+      for (int t = worker; t < p.total_tiles && ok && in_tile_loop; t += workers) {
         const TileCoord tc = decode_tile(t, p);
         const int m_begin = tc.m0 + (int)rank * kBM;        // first of the 128 rows this CTA stages
         const int n_begin = tc.n0 + (int)rank * b_rows;     // first weight row this CTA stages
@@ -634,32 +672,49 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           r = tap / p.S;
           sx = tap - r * p.S;
         }
-        for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb, ++it) {
-          ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.empty[s]), ph ^ 1u, &ctrl, p));
-          if (!ok) break;
-          // bytes are reported to the leader's barrier; the leader arms it for both CTAs' copies
-          uint32_t full = smem_u32(&ctrl.full[s]);
-          if (PAIR) full = mapa_rank(full, 0);
-          const uint32_t dst = ring + (uint32_t)s * p.stage_bytes + my_off;
-          if (elect_one()) {
-            if (warp == 0 && rank == 0) mbar_expect_tx(smem_u32(&ctrl.full[s]), (PAIR ? 2u : 1u) * p.stage_bytes);
-            if (p.is_conv) {
-              if (is_a)
-                tma_load_im2col<PAIR>(dst, my_map, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx, (uint16_t)r);
-              else
-                tma_load_2d<PAIR>(dst, my_map, full, tap * p.w_pitch + cb * p.BK, n_begin);
-            } else {
-              tma_load_2d<PAIR>(dst, my_map, full, kb * p.BK, is_a ? m_begin : n_begin);
-            }
+        for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps, ++it) {
+          const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;      // k-blocks in this stage
+          const bool my_turn = (int)(it % (uint32_t)nsub) == sub;
+          uint32_t full = 0, dst = 0;
+          if (my_turn) {                                  // this warp's turn for its plane
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.empty[s]), ph ^ 1u, &ctrl, p));
+            if (!ok) break;
+            // bytes are reported to the leader's barrier; the leader arms it for both CTAs' copies
+            full = smem_u32(&ctrl.full[s]);
+            if (PAIR) full = mapa_rank(full, 0);
+            dst = ring + (uint32_t)s * p.stage_bytes + my_off;
+            if (act_plane == 0 && rank == 0 && elect_one())
+              mbar_expect_tx(smem_u32(&ctrl.full[s]), (PAIR ? 2u : 1u) * (uint32_t)nkb * p.kb_bytes);
           }
-          if (p.is_conv) {
-            if (++cb == p.cblks) {
-              cb = 0;
-              ++tap;
-              if (++sx == p.S) { sx = 0; ++r; }
+          for (int j = 0; j < nkb; ++j) {
+            if (my_turn && elect_one()) {
+              if (p.is_conv) {
+                if (is_a)
+                  tma_load_im2col<PAIR>(dst, my_map, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx,
+                                        (uint16_t)r);
+                else
+                  tma_load_2d<PAIR>(dst, my_map, full, tap * p.w_pitch + cb * p.BK, n_begin);
+              } else {
+                tma_load_2d<PAIR>(dst, my_map, full, (kb + j) * p.BK, is_a ? m_begin : n_begin);
+              }
+            }
+            dst += p.kb_bytes;
+            if (p.is_conv) {
+              if (++cb == p.cblks) {
+                cb = 0;
+                ++tap;
+                if (++sx == p.S) { sx = 0; ++r; }
+              }
             }
           }
           if (++s == p.stages) { s = 0; ph ^= 1u; }
+        }
+      }
+      const bool is_b_loader = b_res && warp >= NAX && warp < NPLANES;
+      if (ctrl.abort && lane == 0 && is_b_loader) {
+        // another role gave up: let the resident-weight copies land before the CTA exits
+        const unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(smem_u32(&ctrl.b_ready), 0) && global_ns() - t0 < 50000000ull) {
         }
       }
       if ((!ok || ctrl.abort) && lane == 0) {
@@ -693,13 +748,21 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       const uint32_t dhi = smem_desc_hi(p.sbo, p.layout_type);
       const uint32_t ring_lo = smem_desc_lo(ring);
       const uint32_t stage_u = p.stage_bytes >> 4, a_u = p.a_bytes >> 4, b_u = p.b_bytes >> 4;
-      const uint32_t off_a1 = a_u, off_b0 = NAX * a_u, off_b1 = NAX * a_u + b_u;
+      const uint32_t kb_u = p.kb_bytes >> 4;
+      const uint32_t off_a1 = a_u, off_b0 = NAX * a_u;
       const int ksteps = p.ksteps;
       const uint32_t full_bar0 = smem_u32(&ctrl.full[0]), empty_bar0 = smem_u32(&ctrl.empty[0]);
       uint32_t tile_iter = 0, ph = 0;
       uint32_t a0 = ring_lo, full_bar = full_bar0, empty_bar = empty_bar0;
       int s = 0;
       bool ok = true;
+      const bool b_res = GROUPED && !PAIR && p.b_resident;
+      const int kps = GROUPED ? p.kps : 1;
+      const uint32_t bres_lo = smem_desc_lo(ring + p.b_res_off), bres_u = NBW * b_u;
+      if (b_res) {
+        ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.b_ready), 0u, &ctrl, p, false));
+        tc_fence_after();
+      }
       for (int t = worker; t < p.total_tiles && ok; t += workers, ++tile_iter) {
         const TileCoord tc = decode_tile(t, p);
         const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
@@ -712,26 +775,50 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
         const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
         uint32_t acc = 0u;
-        for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
+        uint32_t bres = bres_lo + (uint32_t)tc.kb_begin * bres_u;   // resident weights of this k-block
+        for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps) {
+          const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;
           ok = __all_sync(0xffffffffu, wait_bar(full_bar, ph, &ctrl, p, false));
           if (!ok) break;
           tc_fence_after();
           if (elect_one()) {
-          // a0: low descriptor word of the first A plane of this stage; the other planes and the
-          // k-steps are fixed offsets (16-byte units) from it
-          mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0, a0 + off_a1, a0 + off_b0, a0 + off_b1, dhi, id_ss, id_su,
-                                    id_us, id_uu, acc);
-          if (ksteps > 1)
-            mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 2u, a0 + off_a1 + 2u, a0 + off_b0 + 2u, a0 + off_b1 + 2u,
-                                      dhi, id_ss, id_su, id_us, id_uu, 1u);
-          if (ksteps > 2) {
-            mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 4u, a0 + off_a1 + 4u, a0 + off_b0 + 4u, a0 + off_b1 + 4u,
-                                      dhi, id_ss, id_su, id_us, id_uu, 1u);
-            mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 6u, a0 + off_a1 + 6u, a0 + off_b0 + 6u, a0 + off_b1 + 6u,
-                                      dhi, id_ss, id_su, id_us, id_uu, 1u);
+            // a0 / ak: low descriptor word of the first A plane of a k-block; the other planes and
+            // the k-steps are fixed offsets (16-byte units) from it (weights: in the stage or
+            // resident).  The first k-block is straight-line code; grouped stages loop over the rest.
+            {
+              const uint32_t b0 = b_res ? bres : a0 + off_b0;
+              mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0, a0 + off_a1, b0, b0 + b_u, dhi, id_ss, id_su, id_us,
+                                        id_uu, acc);
+              if (ksteps > 1)
+                mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 2u, a0 + off_a1 + 2u, b0 + 2u, b0 + b_u + 2u, dhi,
+                                          id_ss, id_su, id_us, id_uu, 1u);
+              if (ksteps > 2) {
+                mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 4u, a0 + off_a1 + 4u, b0 + 4u, b0 + b_u + 4u, dhi,
+                                          id_ss, id_su, id_us, id_uu, 1u);
+                mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, a0 + 6u, a0 + off_a1 + 6u, b0 + 6u, b0 + b_u + 6u, dhi,
+                                          id_ss, id_su, id_us, id_uu, 1u);
+              }
+            }
+            if (GROUPED && nkb > 1) {
+              uint32_t ak = a0 + kb_u, bk = bres + bres_u;
+              for (int j = 1; j < nkb; ++j, ak += kb_u, bk += bres_u) {
+                const uint32_t b0 = b_res ? bk : ak + off_b0;
+                mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, ak, ak + off_a1, b0, b0 + b_u, dhi, id_ss, id_su, id_us,
+                                          id_uu, 1u);
+                if (ksteps > 1)
+                  mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, ak + 2u, ak + off_a1 + 2u, b0 + 2u, b0 + b_u + 2u, dhi,
+                                            id_ss, id_su, id_us, id_uu, 1u);
+                if (ksteps > 2) {
+                  mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, ak + 4u, ak + off_a1 + 4u, b0 + 4u, b0 + b_u + 4u, dhi,
+                                            id_ss, id_su, id_us, id_uu, 1u);
+                  mma_kstep<NAX, NBW, PAIR>(d0, d1, d2, ak + 6u, ak + off_a1 + 6u, b0 + 6u, b0 + b_u + 6u, dhi,
+                                            id_ss, id_su, id_us, id_uu, 1u);
+                }
+              }
+            }
+            tc_commit<PAIR>(empty_bar);                        // stage reusable once these MMAs retire
           }
-          tc_commit<PAIR>(empty_bar);                          // stage reusable once these MMAs retire
-          }
+          if (GROUPED) bres += (uint32_t)nkb * bres_u;
           acc = 1u;
           a0 += stage_u;
           full_bar += 8u;
@@ -900,6 +987,10 @@ struct TcConfig {
   int num_kb = 0, splits = 1, kb_per_split = 0;
   int tiles_m = 0, tiles_n = 0;
   int cblks = 1;
+  bool b_resident = false;
+  uint32_t b_res_bytes = 0;
+  int kps = 1;
+  uint32_t kb_bytes = 0;
   bool pair = false;           // two CTAs per 256-row tile (cta_group::2)
   int tile_m = kBM;
   size_t smem_bytes = 0;
@@ -947,6 +1038,8 @@ TcConfig make_config(const GemmProblem& g) {
                           : (c.BK == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
   c.layout_type = c.BK == 128 ? 2u : (c.BK == 64 ? 4u : 6u);
   c.BN = g.N <= 32 ? 32 : (g.N <= 64 ? 64 : 128);
+  const int forced_bn = env_int("ADAPTION_TC_BN", 0);    // experiment knob: narrower tiles
+  if ((forced_bn == 32 || forced_bn == 64) && forced_bn < c.BN) c.BN = forced_bn;
   c.tiles_m = (int)((g.M + kBM - 1) / kBM);
   c.tiles_n = (int)((g.N + c.BN - 1) / c.BN);
   c.acc_bufs = 512 / (c.nacc * c.BN);
@@ -981,7 +1074,22 @@ TcConfig make_config(const GemmProblem& g) {
   const int pair_env = env_int("ADAPTION_TC_PAIR", -1);
   // (measured: pairs win once the reduction is long, K >= 2304 bytes per plane row, and lose on
   // short reductions where per-tile costs dominate)
-  c.pair = c.splits == 1 && g.M >= 1024 && (sms % 2) == 0 && c.BN == 128 && c.BK == 128 && c.num_kb >= 18;
+  const bool pair_ok = c.splits == 1 && g.M >= 1024 && (sms % 2) == 0;
+  c.pair = pair_ok && c.BN == 128 && c.BK == 128 && c.num_kb >= 18;
+  // Medium reductions (1152 <= K < 4608 bytes per plane row) do better on 256 x 64 pair tiles: two
+  // accumulator sets fit in TMEM, so the epilogue of one tile overlaps the MMAs of the next, which
+  // outweighs the slower N = 64 instruction (measured +5..7% on the conv2_2 / conv3 / conv4_1 shapes).
+  const bool narrow = pair_ok && c.BN == 128 && c.BK == 128 && c.num_kb >= 9 && c.num_kb < 36 &&
+                      forced_bn == 0 && pair_env != 0;
+  if (narrow) {
+    c.pair = true;
+    c.BN = 64;
+    c.tiles_n = (int)((g.N + c.BN - 1) / c.BN);
+    c.acc_bufs = 512 / (c.nacc * c.BN);
+    if (c.acc_bufs > kMaxAccBufs) c.acc_bufs = kMaxAccBufs;
+    c.tmem_cols = 32;
+    while (c.tmem_cols < (uint32_t)(c.acc_bufs * c.nacc * c.BN)) c.tmem_cols <<= 1;
+  }
   if (pair_env == 0) c.pair = false;
   if (pair_env == 1 && c.splits == 1 && (sms % 2) == 0) c.pair = true;
   if (c.pair) {
@@ -990,14 +1098,37 @@ TcConfig make_config(const GemmProblem& g) {
   }
   c.a_bytes = (uint32_t)(kBM * c.BK);
   c.b_bytes = (uint32_t)((c.pair ? c.BN / 2 : c.BN) * c.BK);
-  c.stage_bytes = c.nax * c.a_bytes + c.nbw * c.b_bytes;
   const size_t budget = 232448 - sizeof(Ctrl) - 2048;
-  c.stages = (int)((budget - 1024) / c.stage_bytes);
+  // group short k-blocks so that a stage carries roughly 768 tensor-pipe cycles of work or more
+  {
+    const int products = c.nax * c.nbw;
+    const int cyc_per_kb = (c.BK / 32) * products * (c.BN >= 128 ? 64 : 48);
+    int kps = (768 + cyc_per_kb - 1) / cyc_per_kb;
+    if (kps > 4) kps = 4;
+    const int kps_env = env_int("ADAPTION_TC_KPS", 0);
+    if (kps_env >= 1 && kps_env <= 4) kps = kps_env;
+    if (kps > c.kb_per_split) kps = c.kb_per_split;
+    if (kps < 1) kps = 1;
+    c.kps = kps;
+  }
+  c.kb_bytes = c.nax * c.a_bytes + c.nbw * c.b_bytes;
+  // One column tile and a short reduction: keep every weight k-block resident in shared memory and
+  // stream only the activation planes (fewer bulk copies per k-block for the 64-channel and
+  // 3-channel layers).  Only if at least three activation stages still fit.
+  const size_t res_bytes = (size_t)c.num_kb * c.nbw * c.b_bytes;
+  if (!c.pair && c.tiles_n == 1 && c.splits == 1 && c.tiles_m >= 4 * sms &&
+      res_bytes + 3 * (size_t)c.kps * c.nax * c.a_bytes + 1024 <= budget && env_int("ADAPTION_TC_BRES", 1) != 0) {
+    c.b_resident = true;
+    c.b_res_bytes = (uint32_t)res_bytes;
+    c.kb_bytes = c.nax * c.a_bytes;
+  }
+  c.stage_bytes = (uint32_t)c.kps * c.kb_bytes;
+  c.stages = (int)((budget - 1024 - c.b_res_bytes) / c.stage_bytes);
   if (c.stages > kMaxStages) c.stages = kMaxStages;
   const int stage_cap = env_int("ADAPTION_TC_STAGES", 0);   // experiment knob: shallower ring
   if (stage_cap >= 2 && stage_cap < c.stages) c.stages = stage_cap;
   if (c.stages < 2) return c;
-  c.smem_bytes = (size_t)c.stages * c.stage_bytes + 1024;
+  c.smem_bytes = (size_t)c.stages * c.stage_bytes + 1024 + c.b_res_bytes;
   c.ok = true;
   return c;
 }
@@ -1027,11 +1158,11 @@ bool encode_im2col_nhwc(CUtensorMap* map, const void* base, const adaption_conv_
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NAX, int NBW, bool PAIR>
+template <int NAX, int NBW, bool PAIR, bool GROUPED>
 int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem, cudaStream_t stream) {
   static size_t attr_size = 0;
   if (smem > attr_size) {
-    if (cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
       return ADAPTION_ERR_CUDA;
     attr_size = smem;
@@ -1051,7 +1182,7 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
     cfg.attrs = attr;
     cfg.numAttrs = 1;
   }
-  if (cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR>, maps[0], maps[1], maps[2], maps[3], p) !=
+  if (cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>, maps[0], maps[1], maps[2], maps[3], p) !=
       cudaSuccess) {
     (void)cudaGetLastError();
     return ADAPTION_ERR_CUDA;
@@ -1062,8 +1193,12 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
 template <int NAX, int NBW>
 int launch_either(bool pair, const CUtensorMap* maps, const TcParams& p, int grid, size_t smem,
                   cudaStream_t stream) {
-  return pair ? launch_kernel<NAX, NBW, true>(maps, p, grid, smem, stream)
-              : launch_kernel<NAX, NBW, false>(maps, p, grid, smem, stream);
+  const bool grouped = p.kps > 1 || p.b_resident != 0;
+  if (pair)
+    return grouped ? launch_kernel<NAX, NBW, true, true>(maps, p, grid, smem, stream)
+                   : launch_kernel<NAX, NBW, true, false>(maps, p, grid, smem, stream);
+  return grouped ? launch_kernel<NAX, NBW, false, true>(maps, p, grid, smem, stream)
+                 : launch_kernel<NAX, NBW, false, false>(maps, p, grid, smem, stream);
 }
 
 
@@ -1216,6 +1351,9 @@ int launch_tensor(const GemmProblem& g) {
   p.BN = c.BN; p.BK = c.BK; p.ksteps = c.BK / 32;
   p.sbo = (uint32_t)(8 * c.BK); p.layout_type = c.layout_type;
   p.stages = c.stages; p.a_bytes = c.a_bytes; p.b_bytes = c.b_bytes; p.stage_bytes = c.stage_bytes;
+  p.kps = c.kps; p.kb_bytes = c.kb_bytes;
+  p.b_resident = c.b_resident ? 1 : 0;
+  p.b_res_off = (uint32_t)c.stages * c.stage_bytes;
   p.acc_bufs = c.acc_bufs; p.tmem_cols = c.tmem_cols;
   p.is_conv = g.is_conv ? 1 : 0;
   if (g.is_conv) {
