@@ -13,8 +13,8 @@
 // One persistent CTA per SM walks over output tiles (128 rows x BN columns):
 //   warps 0-3  : TMA producers, one per operand plane (im2col / tiled loads into a ring of
 //                shared-memory stages; a single warp issues bulk-tensor copies too slowly)
-//   warp 4     : TMEM allocation and the single MMA-issuing thread
-//   warps 5-20 : epilogue (tcgen05.ld -> int64 recombination -> bias, ReLU, requantize with
+//   warps 4-5  : MMA issue (alternating stages; warp 4 also owns the TMEM allocation)
+//   warps 6-21 : epilogue (tcgen05.ld -> int64 recombination -> bias, ReLU, requantize with
 //                saturation, zero / saturation counters, byte-plane stores; or range / split-K)
 // Every device-side wait is bounded; on expiry the kernel flags ADAPTION_ERR_TIMEOUT in the
 // caller's stats word, drains what it has in flight, frees its TMEM and returns.
@@ -36,9 +36,12 @@ constexpr int kMaxStages = 12;
 constexpr int kMaxAccBufs = 4;
 constexpr int kEpiWarps = 16;                // four per TMEM lane quarter, each takes a quarter of the columns
 constexpr int kProducerWarps = 4;            // one per operand plane: TMA issue is slow per warp
+// Two MMA-issuing warps take turns stage by stage: the instruction stream of one issuing thread
+// cannot keep up with the tensor pipe on short stages (N = 64 instructions, 64-byte k-blocks).
+constexpr int kMmaWarps = 2;
 constexpr int kMmaWarp = kProducerWarps;
-constexpr int kFirstEpiWarp = kProducerWarps + 1;
-constexpr int kThreads = 32 * (kProducerWarps + 1 + kEpiWarps);
+constexpr int kFirstEpiWarp = kProducerWarps + kMmaWarps;
+constexpr int kThreads = 32 * (kProducerWarps + kMmaWarps + kEpiWarps);
 constexpr int kMaxBN = 256;
 // int32 accumulators: the shared middle accumulator takes two products of magnitude
 // <= 128*255 per k, so a reduction of up to 32768 stays below 2^31.
@@ -94,7 +97,8 @@ struct Ctrl {
   unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[kMaxAccBufs];
   unsigned long long tmem_empty[kMaxAccBufs];
-  unsigned long long drain;
+  unsigned long long first_issued[kMaxAccBufs];   // first stage of a tile is in the pipe
+  unsigned long long drain[kMmaWarps];
   unsigned long long b_ready;   // resident weights have landed
   uint32_t tmem_base;
   volatile uint32_t abort;
@@ -594,10 +598,11 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       mbar_init(smem_u32(&ctrl.empty[s]), 1);
     }
     for (int b = 0; b < p.acc_bufs; ++b) {
-      mbar_init(smem_u32(&ctrl.tmem_full[b]), 1);
+      mbar_init(smem_u32(&ctrl.tmem_full[b]), kMmaWarps);
+      mbar_init(smem_u32(&ctrl.first_issued[b]), 1);
       mbar_init(smem_u32(&ctrl.tmem_empty[b]), PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
-    mbar_init(smem_u32(&ctrl.drain), 1);
+    for (int w = 0; w < kMmaWarps; ++w) mbar_init(smem_u32(&ctrl.drain[w]), 1);
     mbar_init(smem_u32(&ctrl.b_ready), 1);
     ctrl.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -736,9 +741,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       }
     }
     __syncwarp();
-  } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------------ MMA issuer (leader only)
-    // The whole warp walks the loop (uniform control flow and operands); one elected lane issues.
+  } else if (warp < kFirstEpiWarp) {
+    // ------------------------------------------------------------------ MMA issuers (leader only)
+    // Both warps walk the same loop (uniform control flow and operands) and take the stages in
+    // turn; in each, one elected lane issues.  The warp that issues a tile's first stage (which
+    // overwrites the accumulators) tells the other one through `first_issued` before that one
+    // may add to them.
+    const int mw = warp - kMmaWarp;
     if (rank == 0) {
       const int tile_rows = PAIR ? 2 * kBM : kBM;
       const uint32_t id_ss = make_idesc(true, true, p.BN, tile_rows);
@@ -752,7 +761,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       const uint32_t off_a1 = a_u, off_b0 = NAX * a_u;
       const int ksteps = p.ksteps;
       const uint32_t full_bar0 = smem_u32(&ctrl.full[0]), empty_bar0 = smem_u32(&ctrl.empty[0]);
-      uint32_t tile_iter = 0, ph = 0;
+      uint32_t tile_iter = 0, ph = 0, sit = 0;       // sit: stages so far (decides whose turn it is)
       uint32_t a0 = ring_lo, full_bar = full_bar0, empty_bar = empty_bar0;
       int s = 0;
       bool ok = true;
@@ -767,20 +776,35 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const TileCoord tc = decode_tile(t, p);
         const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
         const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
-        if (lane == 0) TL_STAMP(1, tile_iter, 0);
+        if (lane == 0 && mw == 0) TL_STAMP(1, tile_iter, 0);
         ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p, false));
         if (!ok) break;
         tc_fence_after();
-        if (lane == 0) TL_STAMP(1, tile_iter, 1);
+        if (lane == 0 && mw == 0) TL_STAMP(1, tile_iter, 1);
         const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
         const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
-        uint32_t acc = 0u;
         uint32_t bres = bres_lo + (uint32_t)tc.kb_begin * bres_u;   // resident weights of this k-block
-        for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps) {
+        bool after_first = ((int)(sit & 1u) == mw);   // the first stage's owner needs no hand-shake
+        for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps, ++sit) {
           const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;
+          const bool mine = (int)(sit & 1u) == mw;
+          if (mine) {
+#ifdef ADAPTION_TIMELINE
+          const long long tw0 = clock64();
+#endif
           ok = __all_sync(0xffffffffu, wait_bar(full_bar, ph, &ctrl, p, false));
+#ifdef ADAPTION_TIMELINE
+          if (lane == 0 && blockIdx.x == 0 && tile_iter < 32u)
+            g_timeline[((1 + mw * 3) * 32 + tile_iter) * 8 + 3] += clock64() - tw0;   // time waiting for data
+#endif
           if (!ok) break;
+          if (!after_first) {
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.first_issued[buf]), bph, &ctrl, p, false));
+            if (!ok) break;
+            after_first = true;
+          }
           tc_fence_after();
+          const uint32_t acc = kb == tc.kb_begin ? 0u : 1u;
           if (elect_one()) {
             // a0 / ak: low descriptor word of the first A plane of a k-block; the other planes and
             // the k-steps are fixed offsets (16-byte units) from it (weights: in the stage or
@@ -817,9 +841,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
               }
             }
             tc_commit<PAIR>(empty_bar);                        // stage reusable once these MMAs retire
+            if (kb == tc.kb_begin) {
+              tc_fence_before();
+              mbar_arrive(smem_u32(&ctrl.first_issued[buf]));
+            }
+          }
           }
           if (GROUPED) bres += (uint32_t)nkb * bres_u;
-          acc = 1u;
           a0 += stage_u;
           full_bar += 8u;
           empty_bar += 8u;
@@ -833,13 +861,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         }
         if (ok && elect_one()) tc_commit<PAIR>(smem_u32(&ctrl.tmem_full[buf]));   // tile complete
         __syncwarp();
-        if (lane == 0) TL_STAMP(1, tile_iter, 2);
+        if (lane == 0 && mw == 0) TL_STAMP(1, tile_iter, 2);
       }
       if ((!ok || ctrl.abort) && lane == 0) {
         // make sure no MMA still reads shared memory or writes TMEM when the CTAs tear down
-        tc_commit<false>(smem_u32(&ctrl.drain));
+        tc_commit<false>(smem_u32(&ctrl.drain[mw]));
         const unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(smem_u32(&ctrl.drain), 0) && global_ns() - t0 < 50000000ull) {
+        while (!mbar_try_wait(smem_u32(&ctrl.drain[mw]), 0) && global_ns() - t0 < 50000000ull) {
         }
       }
     }
@@ -1308,6 +1336,10 @@ namespace {
 }  // namespace
 
 #ifdef ADAPTION_TIMELINE
+extern "C" __attribute__((visibility("default"))) int adaption_debug_timeline_reset() {
+  static long long zeros[8192];
+  return cudaMemcpyToSymbol(g_timeline, zeros, sizeof(zeros)) == cudaSuccess ? 0 : 6;
+}
 extern "C" __attribute__((visibility("default"))) int adaption_debug_timeline(long long* h_out, int n) {
   return cudaMemcpyFromSymbol(h_out, g_timeline, sizeof(long long) * (size_t)n) == cudaSuccess ? 0 : 6;
 }
