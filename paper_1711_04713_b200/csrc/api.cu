@@ -1,7 +1,16 @@
 // extern "C" entry points: argument validation and dispatch.  See include/adaption.h.
+#include <cstdio>
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace adaption {
+int cuda_failure(cudaError_t e, const char* where) {
+  if (std::getenv("ADAPTION_LOG") != nullptr)
+    std::fprintf(stderr, "adaption: CUDA error at %s: %s\n", where, cudaGetErrorString(e));
+  return ADAPTION_ERR_CUDA;
+}
+
 int quantize_impl(const float*, size_t, size_t, const adaption_qtensor&, const adaption_qfmt*, int32_t,
                   int32_t, adaption_stats*, cudaStream_t);
 int requant_impl(const adaption_qtensor&, size_t, size_t, int32_t, const adaption_qtensor&,

@@ -113,7 +113,12 @@ int check_qtensor_in(const adaption_qtensor& t, int64_t inner);
 // ... as an output: planes (or at least q16) present
 int check_qtensor_out(const adaption_qtensor& t, int64_t inner);
 
-inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? ADAPTION_OK : ADAPTION_ERR_CUDA; }
+// CUDA runtime failure -> ADAPTION_ERR_CUDA; with ADAPTION_LOG set in the environment the runtime's
+// message goes to stderr.
+int cuda_failure(cudaError_t e, const char* where);
+inline int cuda_status(cudaError_t e, const char* where = "") {
+  return e == cudaSuccess ? ADAPTION_OK : cuda_failure(e, where);
+}
 
 // ---- launches implemented in the other translation units ---------------------------------
 struct GemmProblem {

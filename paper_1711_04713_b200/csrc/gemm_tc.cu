@@ -55,6 +55,7 @@ struct TcParams {
   int BN, BK, ksteps;
   uint32_t sbo, layout_type;
   int stages;
+  int mma_warps;              // 1, or 2 (then ring slot s belongs to issuing warp s & 1)
   uint32_t a_bytes, b_bytes, stage_bytes;
   // a stage holds `kps` consecutive k-blocks of `kb_bytes` each (short k-blocks are grouped so
   // that the per-stage hand-shake is amortised over enough MMAs)
@@ -245,6 +246,19 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
         "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
             bar),
         "h"((uint16_t)3)
+        : "memory");
+  else
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+// Same, but only the issuing (leader) CTA's barrier is signalled.
+template <bool PAIR>
+__device__ __forceinline__ void tc_commit_leader(uint32_t bar) {
+  if (PAIR)
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+            bar),
+        "h"((uint16_t)1)
         : "memory");
   else
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
@@ -598,7 +612,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       mbar_init(smem_u32(&ctrl.empty[s]), 1);
     }
     for (int b = 0; b < p.acc_bufs; ++b) {
-      mbar_init(smem_u32(&ctrl.tmem_full[b]), kMmaWarps);
+      mbar_init(smem_u32(&ctrl.tmem_full[b]), (uint32_t)p.mma_warps);
       mbar_init(smem_u32(&ctrl.first_issued[b]), 1);
       mbar_init(smem_u32(&ctrl.tmem_empty[b]), PAIR ? 2 * kEpiWarps : kEpiWarps);
     }
@@ -679,7 +693,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         }
         for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps, ++it) {
           const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;      // k-blocks in this stage
-          const bool my_turn = (int)(it % (uint32_t)nsub) == sub;
+          const bool my_turn = (s % nsub) == sub;     // ring slots have fixed owners
           uint32_t full = 0, dst = 0;
           if (my_turn) {                                  // this warp's turn for its plane
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.empty[s]), ph ^ 1u, &ctrl, p));
@@ -743,12 +757,16 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     __syncwarp();
   } else if (warp < kFirstEpiWarp) {
     // ------------------------------------------------------------------ MMA issuers (leader only)
-    // Both warps walk the same loop (uniform control flow and operands) and take the stages in
-    // turn; in each, one elected lane issues.  The warp that issues a tile's first stage (which
-    // overwrites the accumulators) tells the other one through `first_issued` before that one
-    // may add to them.
+    // One warp, or two that walk the same loop (uniform control flow and operands) and own the
+    // ring slots of their parity: a slot's "full" barrier is then only ever waited on by the warp
+    // that also releases the slot, so no phase of it can pass unseen.
+    // In each warp one elected lane issues.  The accumulators are overwritten by a tile's first
+    // stage; the other warp may add to them only after that stage has retired, which its owner
+    // reports through a commit on `first_issued` (instructions of different threads are not
+    // ordered otherwise; integer additions commute, so nothing else needs an order).
     const int mw = warp - kMmaWarp;
-    if (rank == 0) {
+    if (rank == 0 && mw < p.mma_warps) {
+      const bool solo = p.mma_warps == 1;
       const int tile_rows = PAIR ? 2 * kBM : kBM;
       const uint32_t id_ss = make_idesc(true, true, p.BN, tile_rows);
       const uint32_t id_su = make_idesc(true, false, p.BN, tile_rows);
@@ -761,7 +779,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       const uint32_t off_a1 = a_u, off_b0 = NAX * a_u;
       const int ksteps = p.ksteps;
       const uint32_t full_bar0 = smem_u32(&ctrl.full[0]), empty_bar0 = smem_u32(&ctrl.empty[0]);
-      uint32_t tile_iter = 0, ph = 0, sit = 0;       // sit: stages so far (decides whose turn it is)
+      uint32_t tile_iter = 0, ph = 0;
       uint32_t a0 = ring_lo, full_bar = full_bar0, empty_bar = empty_bar0;
       int s = 0;
       bool ok = true;
@@ -784,10 +802,10 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
         const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
         uint32_t bres = bres_lo + (uint32_t)tc.kb_begin * bres_u;   // resident weights of this k-block
-        bool after_first = ((int)(sit & 1u) == mw);   // the first stage's owner needs no hand-shake
-        for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps, ++sit) {
+        bool after_first = solo || (s & 1) == mw;     // the first stage's owner needs no hand-shake
+        for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps) {
           const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;
-          const bool mine = (int)(sit & 1u) == mw;
+          const bool mine = solo || (s & 1) == mw;
           if (mine) {
 #ifdef ADAPTION_TIMELINE
           const long long tw0 = clock64();
@@ -841,10 +859,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
               }
             }
             tc_commit<PAIR>(empty_bar);                        // stage reusable once these MMAs retire
-            if (kb == tc.kb_begin) {
-              tc_fence_before();
-              mbar_arrive(smem_u32(&ctrl.first_issued[buf]));
-            }
+            if (!solo && kb == tc.kb_begin) tc_commit_leader<PAIR>(smem_u32(&ctrl.first_issued[buf]));
           }
           }
           if (GROUPED) bres += (uint32_t)nkb * bres_u;
@@ -1009,6 +1024,7 @@ struct TcConfig {
   uint32_t layout_type = 0;
   int nax = 1, nbw = 1, nacc = 1;
   int stages = 0;
+  int mma_warps = 1;
   uint32_t a_bytes = 0, b_bytes = 0, stage_bytes = 0;
   int acc_bufs = 1;
   uint32_t tmem_cols = 32;
@@ -1156,6 +1172,9 @@ TcConfig make_config(const GemmProblem& g) {
   const int stage_cap = env_int("ADAPTION_TC_STAGES", 0);   // experiment knob: shallower ring
   if (stage_cap >= 2 && stage_cap < c.stages) c.stages = stage_cap;
   if (c.stages < 2) return c;
+  c.mma_warps = kMmaWarps;
+  const int mmaw_env = env_int("ADAPTION_TC_MMAW", 0);      // experiment knob: force one issuing warp
+  if (mmaw_env == 1) c.mma_warps = 1;
   c.smem_bytes = (size_t)c.stages * c.stage_bytes + 1024 + c.b_res_bytes;
   c.ok = true;
   return c;
@@ -1190,9 +1209,9 @@ template <int NAX, int NBW, bool PAIR, bool GROUPED>
 int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem, cudaStream_t stream) {
   static size_t attr_size = 0;
   if (smem > attr_size) {
-    if (cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess)
-      return ADAPTION_ERR_CUDA;
+    const cudaError_t ae = cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (ae != cudaSuccess) return cuda_failure(ae, "lp_gemm_kernel shared-memory attribute");
     attr_size = smem;
   }
   cudaLaunchConfig_t cfg;
@@ -1210,12 +1229,13 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
     cfg.attrs = attr;
     cfg.numAttrs = 1;
   }
-  if (cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>, maps[0], maps[1], maps[2], maps[3], p) !=
-      cudaSuccess) {
+  const cudaError_t le =
+      cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>, maps[0], maps[1], maps[2], maps[3], p);
+  if (le != cudaSuccess) {
     (void)cudaGetLastError();
-    return ADAPTION_ERR_CUDA;
+    return cuda_failure(le, "lp_gemm_kernel launch");
   }
-  return cuda_status(cudaGetLastError());
+  return cuda_status(cudaGetLastError(), "after lp_gemm_kernel launch");
 }
 
 template <int NAX, int NBW>
@@ -1382,7 +1402,7 @@ int launch_tensor(const GemmProblem& g) {
   p.num_kb = c.num_kb; p.kb_per_split = c.kb_per_split;
   p.BN = c.BN; p.BK = c.BK; p.ksteps = c.BK / 32;
   p.sbo = (uint32_t)(8 * c.BK); p.layout_type = c.layout_type;
-  p.stages = c.stages; p.a_bytes = c.a_bytes; p.b_bytes = c.b_bytes; p.stage_bytes = c.stage_bytes;
+  p.stages = c.stages; p.mma_warps = c.mma_warps; p.a_bytes = c.a_bytes; p.b_bytes = c.b_bytes; p.stage_bytes = c.stage_bytes;
   p.kps = c.kps; p.kb_bytes = c.kb_bytes;
   p.b_resident = c.b_resident ? 1 : 0;
   p.b_res_off = (uint32_t)c.stages * c.stage_bytes;
@@ -1405,7 +1425,8 @@ int launch_tensor(const GemmProblem& g) {
   p.timeout_ns = 2000000000ull;
 
   if (c.splits > 1) {
-    if (cudaMemsetAsync(g.workspace, 0, c.workspace_bytes, g.stream) != cudaSuccess) return ADAPTION_ERR_CUDA;
+    const cudaError_t me = cudaMemsetAsync(g.workspace, 0, c.workspace_bytes, g.stream);
+    if (me != cudaSuccess) return cuda_failure(me, "split-K workspace memset");
   }
   int grid;
   if (c.pair) {
