@@ -11,11 +11,12 @@
 // take a single product.
 //
 // One persistent CTA per SM walks over output tiles (128 rows x BN columns):
-//   warps 0-3  : TMA producers, one per operand plane (im2col / tiled loads into a ring of
-//                shared-memory stages; a single warp issues bulk-tensor copies too slowly)
-//   warps 4-5  : MMA issue (alternating stages; warp 4 also owns the TMEM allocation)
-//   warps 6-21 : epilogue (tcgen05.ld -> int64 recombination -> bias, ReLU, requantize with
-//                saturation, zero / saturation counters, byte-plane stores; or range / split-K)
+//   warps 0-2  : TMA producers, spread over the operand planes (im2col / tiled loads into a ring
+//                of shared-memory stages; a single warp issues bulk-tensor copies too slowly)
+//   warp  3    : MMA issue; also owns the TMEM allocation
+//   warps 4-19 : epilogue (tcgen05.ld -> 64-bit recombination -> bias, ReLU, requantize with
+//                saturation, zero / saturation counters; byte planes staged in shared memory and
+//                written by bulk-tensor stores; or range / split-K)
 // Every device-side wait is bounded; on expiry the kernel flags ADAPTION_ERR_TIMEOUT in the
 // caller's stats word, drains what it has in flight, frees its TMEM and returns.
 #include <cuda.h>
@@ -35,14 +36,13 @@ constexpr int kBM = 128;
 constexpr int kMaxStages = 12;
 constexpr int kMaxAccBufs = 4;
 constexpr int kEpiWarps = 16;                // four per TMEM lane quarter, each takes a quarter of the columns
-constexpr int kProducerWarps = 4;            // one per operand plane: TMA issue is slow per warp
-// Two MMA-issuing warps take turns stage by stage: the instruction stream of one issuing thread
-// cannot keep up with the tensor pipe on short stages (N = 64 instructions, 64-byte k-blocks).
-constexpr int kMmaWarps = 2;
+constexpr int kProducerWarps = 3;            // spread over the operand planes: TMA issue is slow per warp
+// One MMA-issuing warp (a second one, alternating stages, measured no faster).
+constexpr int kMmaWarps = 1;
 constexpr int kMmaWarp = kProducerWarps;
 constexpr int kFirstEpiWarp = kProducerWarps + kMmaWarps;
-constexpr int kThreads = 32 * (kProducerWarps + kMmaWarps + kEpiWarps);
-constexpr int kMaxBN = 256;
+constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
+constexpr int kMaxBN = 128;
 // int32 accumulators: the shared middle accumulator takes two products of magnitude
 // <= 128*255 per k, so a reduction of up to 32768 stays below 2^31.
 constexpr int64_t kMaxKPerAccumulation = 32768;
@@ -80,6 +80,10 @@ struct TcParams {
   long long ws_ld;
   adaption_stats* stats;
   unsigned long long timeout_ns;
+  // epilogue variants chosen on the host
+  int fast_relu;              // launch the FAST kernel variant (paired 16-bit epilogue)
+  int staged;                 // outputs leave through shared memory and bulk-tensor stores
+  uint32_t stage_off;         // offset of the staging planes from the ring base
 };
 
 // Optional per-role time stamps of CTA 0 (development builds only: -DADAPTION_TIMELINE).
@@ -103,7 +107,7 @@ struct Ctrl {
   unsigned long long b_ready;   // resident weights have landed
   uint32_t tmem_base;
   volatile uint32_t abort;
-  long long bias64[kEpiWarps][kMaxBN / 4];
+  long long colconst[kMaxBN];   // per-column epilogue constants of the current tile
 };
 
 // ---------------------------------------------------------------------------------- PTX
@@ -297,15 +301,18 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t 
         "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-        "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+// Placed after tcgen05.wait::ld: ties the loaded registers to that point so that no use of them can
+// be scheduled before the wait (the load fills them asynchronously).
+__device__ __forceinline__ void pin_after_wait(int32_t (&r)[8]) {
+  asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+               :
+               : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -462,119 +469,184 @@ __device__ __forceinline__ int32_t requant_shift_right(long long v, long long ha
 }
 
 
-// Fast requantization for ReLU layers with a rounding right shift (shift >= 1), all in 32-bit
-// arithmetic.  The exact pre-activation value is split as  v = 2^16 * T + L  with
-//   T = hh + (mid >> 8) + (ll >> 16)                 (arithmetic shifts)
-//   L = ((mid & 255) << 8) + (ll & 65535)            (0 <= L < 2^17)
-// (for two / one accumulators the missing leading terms are zero), and the per-column constant
-// C = bias * 2^bias_shift + 2^(shift-1) likewise as 2^16 * Ch + Cl with 0 <= Cl < 2^16.  Then
-//   v + C = 2^16 * T' + L',  T' = T + Ch + ((L + Cl) >> 16),  L' = (L + Cl) & 65535,
-// and because ReLU maps every negative value to zero the rounded result is
-//   max(0, floor((v + C) / 2^shift)),
-// i.e. T' >> (shift - 16) for shift >= 16 and (T' << (16 - shift)) + (L' >> shift) below that
-// (T' clamped first: |T'| >= 2^16 saturates or clips to zero in any case).
-template <int NACC, bool WIDE_SHIFT>
-__device__ __forceinline__ int32_t requant_relu32(int32_t x0, int32_t x1, int32_t x2, int2 c, int shift,
-                                                  int32_t qmax, int32_t& r_out) {
+// Fast requantization for ReLU layers with a rounding right shift 9 <= shift <= 31, in 32-bit
+// arithmetic.  Wanted: floor((v + C) / 2^shift) with v = 2^16 hh + 2^8 mid + ll and the per-column
+// constant C = bias * 2^bias_shift + 2^(shift-1) (ReLU maps negative values to zero, so rounding
+// half away from zero is this floor).  With C = 2^16 Ch + Cl, 0 <= Cl < 2^16:
+//   T = mid + floor((ll + Cl) / 2^8),  H = hh + Ch,   v + C = 2^8 (2^8 H + T) + (a remainder below 2^8)
+// and because shift >= 8 the remainder cannot change the floor:
+//   shift >= 16:  floor((H + floor(T / 2^8)) / 2^(shift-16))
+//   shift <  16:  H * 2^(16-shift) + floor(T / 2^(shift-8))
+// The host checks from the reduction length that none of these 32-bit quantities can overflow
+// (otherwise the layer takes the generic 64-bit epilogue).  The divisions by 2^8 are taken as the
+// high word of a product with 2^24, which runs on the multiplier beside the integer ALU.
+__device__ __forceinline__ int32_t mad_hi(int32_t a, int32_t b, int32_t c) {
+  int32_t d;
+  asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ int32_t mad_lo(int32_t a, int32_t b, int32_t c) {
+  int32_t d;
+  asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+template <int NACC, bool WIDE>
+__device__ __forceinline__ int32_t shifted32(int32_t x0, int32_t x1, int32_t x2, int2 c, int shift) {
   // name the accumulators by weight: hh (2^16), mid (2^8), ll (1)
   const int32_t hh = NACC == 3 ? x0 : 0;
   const int32_t mid = NACC == 3 ? x1 : (NACC == 2 ? x0 : 0);
   const int32_t ll = NACC == 3 ? x2 : (NACC == 2 ? x1 : x0);
-  const int32_t T = hh + (mid >> 8) + (ll >> 16);
-  const int32_t Ls = (int32_t)__byte_perm((uint32_t)mid, 0u, 0x4404) + (ll & 0xffff) + c.y;
-  const int32_t Tp = T + c.x + (Ls >> 16);
-  int32_t r;
-  if (WIDE_SHIFT) {           // shift >= 16
-    r = Tp >> (shift - 16);
-  } else {
-    const int32_t Tc = min(max(Tp, -1), 65535);
-    r = (Tc << (16 - shift)) + ((Ls & 0xffff) >> shift);
-  }
-  r = max(r, 0);
-  r_out = r;
-  return min(r, qmax);
+  const int32_t T = mad_hi(ll + c.x, 1 << 24, mid);
+  const int32_t H = hh + c.y;
+  if (WIDE) return mad_hi(T, 1 << 24, H) >> (shift - 16);
+  return mad_lo(H, 1 << (16 - shift), T >> (shift - 8));
 }
 
-// Sixteen columns of one row.  Counting is kept off the per-element path: saturation is detected
-// by OR-ing r ^ q over the group (non-zero only if something was clipped, which is rare; the exact
-// count is then redone), non-zero outputs are summed as min(q, 1).
-template <int NACC, bool WIDE_SHIFT>
-__device__ __forceinline__ void requant_relu32_x16(const int32_t* a0, const int32_t* a1, const int32_t* a2,
-                                                   const int2* c2, int shift, int32_t qmax, int nvalid,
-                                                   Counts& cnt, int32_t (&q)[16]) {
-  int32_t clipped = 0, nonzero = 0;
-  int32_t r[16];
+// two 32-bit values -> two 16-bit values saturated to [-32768, 32767]; `lo` lands in the low half
+__device__ __forceinline__ uint32_t pack_sat_s16x2(int32_t hi, int32_t lo) {
+  uint32_t d;
+  asm("cvt.pack.sat.s16.s32 %0, %1, %2;" : "=r"(d) : "r"(hi), "r"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t max_s16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.s16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t min_s16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.s16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+
+// One group of accumulators for eight consecutive columns of one row.
+template <int NACC>
+struct Acc8 {
+  int32_t a[3][8];
+};
+template <int NACC>
+__device__ __forceinline__ void load_acc8(uint32_t taddr, int bn, Acc8<NACC>& x) {
+  tmem_ld8(taddr, x.a[0]);
+  if (NACC >= 2) tmem_ld8(taddr + (uint32_t)bn, x.a[1]);
+  if (NACC == 3) tmem_ld8(taddr + 2u * (uint32_t)bn, x.a[2]);
+}
+template <int NACC>
+__device__ __forceinline__ void pin_acc8(Acc8<NACC>& x) {
+  pin_after_wait(x.a[0]);
+  if (NACC >= 2) pin_after_wait(x.a[1]);
+  if (NACC == 3) pin_after_wait(x.a[2]);
+}
+template <int NACC>
+__device__ __forceinline__ long long acc_value(const Acc8<NACC>& x, int j) {
+  return combine<NACC>(x.a[0][j], NACC >= 2 ? x.a[1][j] : 0, NACC == 3 ? x.a[2][j] : 0);
+}
+
+// Eight columns of one row on the fast path: outputs are handled as pairs of 16-bit lanes
+// (saturating pack, ReLU, upper bound, zero count).  Saturation is only detected here (some lane
+// reached the bound); the exact count is then redone from the accumulators, which is rare.
+// Returns the packed outputs w[j] = q[2j] | q[2j+1] << 16.  `counted`: real columns of a real row
+// (the others are padding and only stored).
+template <int NACC, bool WIDE>
+__device__ __forceinline__ void requant_relu_pairs_x8(const Acc8<NACC>& x, const int2* c2, int shift, int32_t qmax,
+                                                      bool counted, Counts& cnt, uint32_t* w) {
+  const uint32_t qmax2 = (uint32_t)qmax * 0x00010001u;
+  uint32_t top = 0, nonzero = 0;
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    q[j] = requant_relu32<NACC, WIDE_SHIFT>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0, c2[j], shift,
-                                            qmax, r[j]);
-    clipped |= r[j] ^ q[j];
-    nonzero += min(q[j], 1);
+  for (int j = 0; j < 4; ++j) {
+    const int32_t r0 = shifted32<NACC, WIDE>(x.a[0][2 * j], NACC >= 2 ? x.a[1][2 * j] : 0,
+                                             NACC == 3 ? x.a[2][2 * j] : 0, c2[2 * j], shift);
+    const int32_t r1 = shifted32<NACC, WIDE>(x.a[0][2 * j + 1], NACC >= 2 ? x.a[1][2 * j + 1] : 0,
+                                             NACC == 3 ? x.a[2][2 * j + 1] : 0, c2[2 * j + 1], shift);
+    uint32_t v = max_s16x2(pack_sat_s16x2(r1, r0), 0u);
+    top = max_s16x2(top, v);
+    if (qmax != 32767) v = min_s16x2(v, qmax2);
+    nonzero += min_s16x2(v, 0x00010001u);
+    w[j] = v;
   }
-  if (nvalid == 16) {
-    cnt.zeros += 16 - nonzero;
-    if (clipped != 0) {
+  if (counted) cnt.zeros += 8u - (nonzero & 0xffffu) - (nonzero >> 16);
+  const int32_t bound = qmax == 32767 ? 32767 : qmax + 1;      // a lane that reached this may have been clipped
+  if (counted && ((int32_t)(top & 0xffffu) >= bound || (int32_t)(top >> 16) >= bound)) {
 #pragma unroll
-      for (int j = 0; j < 16; ++j) cnt.sat_pos += (r[j] > qmax);
-    }
-  } else {
-    // ragged edge: count only the real elements
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      cnt.zeros += (j < nvalid && q[j] == 0);
-      cnt.sat_pos += (j < nvalid && r[j] > qmax);
+    for (int j = 0; j < 8; ++j) {
+      const long long c = (long long)c2[j].y * 65536ll + (long long)c2[j].x;
+      cnt.sat_pos += (((acc_value<NACC>(x, j) + c) >> shift) > (long long)qmax);
     }
   }
 }
 
-// Sixteen consecutive output columns of one row: recombine, add bias, requantize, pack into
-// byte planes (and the optional int16 copy) and store 16 bytes per plane.
+// Eight consecutive output columns of one row: recombine, add bias, requantize.  Returns the
+// outputs packed in pairs, w[j] = (q[2j] & 0xffff) | q[2j+1] << 16.
+// Fast path (kernels built with FAST): every group of eight columns is either entirely real or
+// entirely padding (N is a multiple of 8), `counted` says which.
+template <int NACC>
+__device__ __forceinline__ void requant8_fast(const Acc8<NACC>& x, const long long* c64, const TcParams& p,
+                                              bool counted, Counts& cnt, uint32_t* w) {
+  // per-column constants were staged as (C mod 2^16, C div 2^16) with the rounding half in C
+  const int2* c2 = reinterpret_cast<const int2*>(c64);
+  if (p.rq.shift >= 16)
+    requant_relu_pairs_x8<NACC, true>(x, c2, p.rq.shift, p.rq.qmax, counted, cnt, w);
+  else
+    requant_relu_pairs_x8<NACC, false>(x, c2, p.rq.shift, p.rq.qmax, counted, cnt, w);
+}
 template <int NACC, bool RELU>
-__device__ __forceinline__ void requant_store16(const int32_t* a0, const int32_t* a1, const int32_t* a2,
-                                                const long long* bias64, const TcParams& p, bool row_ok,
-                                                int m, int col, Counts& cnt) {
-  int32_t q[16];
-  const int nvalid = row_ok ? min(max(p.N - col, 0), 16) : 0;
-  if (RELU && p.rq.shift > 0) {
-    // per-column constants were staged as (Ch, Cl) pairs
-    const int2* c2 = reinterpret_cast<const int2*>(bias64);
-    if (p.rq.shift >= 16)
-      requant_relu32_x16<NACC, true>(a0, a1, a2, c2, p.rq.shift, p.rq.qmax, nvalid, cnt, q);
-    else
-      requant_relu32_x16<NACC, false>(a0, a1, a2, c2, p.rq.shift, p.rq.qmax, nvalid, cnt, q);
-  } else if (p.rq.shift > 0) {
+__device__ __forceinline__ void requant8(const Acc8<NACC>& x, const long long* c64, const TcParams& p, bool row_ok,
+                                         int col, Counts& cnt, uint32_t* w) {
+  const int nvalid = row_ok ? min(max(p.N - col, 0), 8) : 0;
+  int32_t q[8];
+  if (p.rq.shift > 0) {
     const long long half = 1ll << (p.rq.shift - 1);
-    if (nvalid == 16) {
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        q[j] = requant_shift_right<RELU, true>(
-            combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bias64[j], half, p.rq.shift,
-            p.rq.qmin, p.rq.qmax, true, cnt);
-    } else {
+    for (int j = 0; j < 8; ++j)
+      q[j] = requant_shift_right<RELU, false>(acc_value<NACC>(x, j) + c64[j], half, p.rq.shift, p.rq.qmin, p.rq.qmax,
+                                              j < nvalid, cnt);
+  } else {
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        q[j] = requant_shift_right<RELU, false>(
-            combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bias64[j], half, p.rq.shift,
-            p.rq.qmin, p.rq.qmax, j < nvalid, cnt);
+    for (int j = 0; j < 8; ++j) q[j] = requant_value(acc_value<NACC>(x, j) + c64[j], p.rq, j < nvalid, cnt);
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) w[j] = __byte_perm((uint32_t)q[2 * j], (uint32_t)q[2 * j + 1], 0x5410);
+}
+
+// What the epilogue does with eight accumulator columns of one row in the modes that store nothing:
+// split-K partial sums go to the int64 workspace, the range mode keeps the largest magnitude.
+template <int NACC>
+__device__ __forceinline__ void partial_or_range8(const Acc8<NACC>& x, const long long* c64, const TcParams& p,
+                                                  bool row_ok, int m, int col, long long& vmax) {
+  if (p.splits > 1) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const long long v = acc_value<NACC>(x, j);
+      if (row_ok && col + j < p.N && v != 0)
+        atomicAdd((unsigned long long*)(p.ws + (long long)m * p.ws_ld + col + j), (unsigned long long)v);
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < 16; ++j)
-      q[j] = requant_value(combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bias64[j],
-                           p.rq, j < nvalid, cnt);
+    for (int j = 0; j < 8; ++j) {
+      long long v = acc_value<NACC>(x, j) + c64[j];
+      if (p.rq.relu && v < 0) v = 0;
+      v = v < 0 ? -v : v;
+      if (row_ok && col + j < p.N) vmax = v > vmax ? v : vmax;
+    }
   }
+}
+
+// byte planes of sixteen packed outputs: four low bytes / four high bytes per word
+__device__ __forceinline__ uint4 plane_lo(const uint32_t (&w)[8]) {
+  return make_uint4(__byte_perm(w[0], w[1], 0x6420), __byte_perm(w[2], w[3], 0x6420),
+                    __byte_perm(w[4], w[5], 0x6420), __byte_perm(w[6], w[7], 0x6420));
+}
+__device__ __forceinline__ uint4 plane_hi(const uint32_t (&w)[8]) {
+  return make_uint4(__byte_perm(w[0], w[1], 0x7531), __byte_perm(w[2], w[3], 0x7531),
+                    __byte_perm(w[4], w[5], 0x7531), __byte_perm(w[6], w[7], 0x7531));
+}
+
+// Direct stores of sixteen outputs of one row (16 bytes per plane; optional int16 copy).
+__device__ __forceinline__ void store16_global(const uint32_t (&w)[8], const TcParams& p, bool row_ok, int m,
+                                               int col) {
   if (row_ok && col < p.y_stride) {
-    uint32_t w[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) w[j] = __byte_perm((uint32_t)q[2 * j], (uint32_t)q[2 * j + 1], 0x5410);
     const size_t off = (size_t)m * (size_t)p.y_stride + (size_t)col;
-    *reinterpret_cast<uint4*>(p.y_lo + off) =
-        make_uint4(__byte_perm(w[0], w[1], 0x6420), __byte_perm(w[2], w[3], 0x6420),
-                   __byte_perm(w[4], w[5], 0x6420), __byte_perm(w[6], w[7], 0x6420));
-    if (p.rq.out_planes == 2)
-      *reinterpret_cast<uint4*>(p.y_hi + off) =
-          make_uint4(__byte_perm(w[0], w[1], 0x7531), __byte_perm(w[2], w[3], 0x7531),
-                     __byte_perm(w[4], w[5], 0x7531), __byte_perm(w[6], w[7], 0x7531));
+    *reinterpret_cast<uint4*>(p.y_lo + off) = plane_lo(w);
+    if (p.rq.out_planes == 2) *reinterpret_cast<uint4*>(p.y_hi + off) = plane_hi(w);
     if (p.y_q16 != nullptr) {
       uint4* dst = reinterpret_cast<uint4*>(p.y_q16 + off);
       dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -583,13 +655,63 @@ __device__ __forceinline__ void requant_store16(const int32_t* a0, const int32_t
   }
 }
 
+// Staged stores: the tile's byte planes are assembled in shared memory (rows of BN bytes, 16-byte
+// chunks swizzled the way the bulk-tensor store expects for that row length, which also keeps the
+// 16-byte writes of a quarter warp on distinct banks) and leave as one bulk-tensor store per plane.
+__device__ __forceinline__ uint32_t staged_offset(int row, int chunk, int bn) {
+  uint32_t off = (uint32_t)row * (uint32_t)bn + (uint32_t)chunk * 16u;
+  return off ^ (((off >> 7) & (uint32_t)((bn >> 4) - 1) & 7u) << 4);
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map),
+               "r"(src), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// the bulk stores committed so far have read their shared-memory source
+__device__ __forceinline__ void bulk_wait_read_all() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// ... and have completed
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_shared() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// Barrier among the epilogue warps only (barrier 0 belongs to __syncthreads).
+__device__ __forceinline__ void epi_bar_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+}
+// ... that also returns the conjunction of every thread's predicate
+__device__ __forceinline__ bool epi_bar_all(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.b32 p, %1, 0;\n"
+      "bar.red.and.pred q, 2, %2, p;\n"
+      "selp.u32 %0, 1, 0, q;\n"
+      "}\n"
+      : "=r"(r)
+      : "r"((uint32_t)pred), "n"(32 * kEpiWarps)
+      : "memory");
+  return r != 0;
+}
+
 // ---------------------------------------------------------------------------------- kernel
 // GROUPED: stages hold several k-blocks and / or the weights are resident in shared memory (short
 // reductions); the plain variant keeps the issue loops free of that bookkeeping.
-template <int NAX, int NBW, bool PAIR, bool GROUPED>
+// FAST: ReLU layer in requantizing mode whose shift lies in [9, 31], N a multiple of 8, no split-K,
+// magnitudes within the 32-bit bounds of the fast epilogue: it then contains only that path.
+// 20 warps: one block per SM, 96 registers per thread.
+template <int NAX, int NBW, bool PAIR, bool GROUPED, bool FAST>
 __global__ void __launch_bounds__(kThreads, 1)
 lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
+               const __grid_constant__ CUtensorMap map_y_hi, const __grid_constant__ CUtensorMap map_y_lo,
                const TcParams p) {
   constexpr int NACC = NAX + NBW - 1;
   extern __shared__ uint8_t smem_raw[];
@@ -633,40 +755,45 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
 
   if (warp < kProducerWarps) {
     // ------------------------------------------------------------------ TMA producers
-    // One warp per operand plane (A planes first, then B planes): every producer walks the same
-    // sequence of stages and issues only its own copy, so the copies of a stage are in flight
-    // side by side (one thread issues a bulk-tensor copy only every few hundred cycles).
+    // Operand planes are numbered A planes first, then B planes.  Every producer warp walks the same
+    // sequence of stages and issues only the copies of its own planes (warp w takes planes w and
+    // w + 3), so the copies of a stage are in flight side by side.
     constexpr int NPLANES = NAX + NBW;
     // (whole warp in uniform control flow; one elected lane issues the copies)
     // Planes that are streamed through the ring: all of them, or only the activation planes when
-    // the weights are resident.  The four producer warps are spread over these planes; with
-    // several warps per plane they take turns stage by stage, because one warp cannot issue
-    // copies fast enough for short stages.
+    // the weights are resident.  With fewer streamed planes than producer warps, several warps
+    // share a plane and take turns stage by stage.
     const bool b_res = GROUPED && !PAIR && p.b_resident;
     const int nact = b_res ? NAX : NPLANES;
     const int kps = GROUPED ? p.kps : 1;
-    const int nsub = kProducerWarps / nact;            // warps per streamed plane
-    const int act_plane = warp % nact, sub = warp / nact;
+    const int nsub = nact >= kProducerWarps ? 1 : kProducerWarps / nact;   // warps per streamed plane
+    const int act_plane = nact >= kProducerWarps ? warp : warp % nact;
+    const int sub = nact >= kProducerWarps ? 0 : warp / nact;
+    const bool two_planes = act_plane + kProducerWarps < nact;             // this warp also owns a second plane
     {
       const bool is_a = act_plane < NAX;
       const int plane = is_a ? act_plane : act_plane - NAX;
       const CUtensorMap* my_map = is_a ? (plane == 0 ? &map_a0 : &map_a1) : (plane == 0 ? &map_b0 : &map_b1);
       const uint32_t my_off = is_a ? (uint32_t)plane * p.a_bytes : NAX * p.a_bytes + (uint32_t)plane * p.b_bytes;
+      // the second plane, if any, is the last B plane (plane index 3 of 4)
+      const CUtensorMap* my_map2 = &map_b1;
+      const uint32_t my_off2 = NAX * p.a_bytes + (uint32_t)(NBW - 1) * p.b_bytes;
       uint32_t it = 0, ph = 0;
       int s = 0;
       bool ok = true;
-      if (b_res && warp >= NAX && warp < NPLANES) {
+      if (b_res && warp == kProducerWarps - 1) {
         // the whole weight matrix of this (single) column tile, one copy per k-block and plane,
         // all reporting to one barrier
-        const int bplane = warp - NAX;
         if (elect_one()) {
           const uint32_t bar = smem_u32(&ctrl.b_ready);
-          if (bplane == 0) mbar_expect_tx(bar, (uint32_t)p.num_kb * NBW * p.b_bytes);
+          mbar_expect_tx(bar, (uint32_t)p.num_kb * NBW * p.b_bytes);
           for (int kb = 0; kb < p.num_kb; ++kb) {
-            const uint32_t dst =
-                ring + p.b_res_off + (uint32_t)kb * (NBW * p.b_bytes) + (uint32_t)bplane * p.b_bytes;
             const int kcol = p.is_conv ? (kb / p.cblks) * p.w_pitch + (kb % p.cblks) * p.BK : kb * p.BK;
-            tma_load_2d<false>(dst, bplane == 0 ? &map_b0 : &map_b1, bar, kcol, 0);
+            for (int bplane = 0; bplane < NBW; ++bplane) {
+              const uint32_t dst =
+                  ring + p.b_res_off + (uint32_t)kb * (NBW * p.b_bytes) + (uint32_t)bplane * p.b_bytes;
+              tma_load_2d<false>(dst, bplane == 0 ? &map_b0 : &map_b1, bar, kcol, 0);
+            }
           }
         }
         __syncwarp();
@@ -701,7 +828,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             // bytes are reported to the leader's barrier; the leader arms it for both CTAs' copies
             full = smem_u32(&ctrl.full[s]);
             if (PAIR) full = mapa_rank(full, 0);
-            dst = ring + (uint32_t)s * p.stage_bytes + my_off;
+            dst = ring + (uint32_t)s * p.stage_bytes;
             if (act_plane == 0 && rank == 0 && elect_one())
               mbar_expect_tx(smem_u32(&ctrl.full[s]), (PAIR ? 2u : 1u) * (uint32_t)nkb * p.kb_bytes);
           }
@@ -709,12 +836,15 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             if (my_turn && elect_one()) {
               if (p.is_conv) {
                 if (is_a)
-                  tma_load_im2col<PAIR>(dst, my_map, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx,
+                  tma_load_im2col<PAIR>(dst + my_off, my_map, full, cb * p.BK, base_w, base_h, img, (uint16_t)sx,
                                         (uint16_t)r);
                 else
-                  tma_load_2d<PAIR>(dst, my_map, full, tap * p.w_pitch + cb * p.BK, n_begin);
+                  tma_load_2d<PAIR>(dst + my_off, my_map, full, tap * p.w_pitch + cb * p.BK, n_begin);
+                if (two_planes)
+                  tma_load_2d<PAIR>(dst + my_off2, my_map2, full, tap * p.w_pitch + cb * p.BK, n_begin);
               } else {
-                tma_load_2d<PAIR>(dst, my_map, full, (kb + j) * p.BK, is_a ? m_begin : n_begin);
+                tma_load_2d<PAIR>(dst + my_off, my_map, full, (kb + j) * p.BK, is_a ? m_begin : n_begin);
+                if (two_planes) tma_load_2d<PAIR>(dst + my_off2, my_map2, full, (kb + j) * p.BK, n_begin);
               }
             }
             dst += p.kb_bytes;
@@ -729,7 +859,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
       }
-      const bool is_b_loader = b_res && warp >= NAX && warp < NPLANES;
+      const bool is_b_loader = b_res && warp == kProducerWarps - 1;
       if (ctrl.abort && lane == 0 && is_b_loader) {
         // another role gave up: let the resident-weight copies land before the CTA exits
         const unsigned long long t0 = global_ns();
@@ -890,87 +1020,118 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;          // TMEM lanes 32*quarter .. 32*quarter+31
-    const int ew = warp - kFirstEpiWarp;   // private bias staging slot
+    const int ew = warp - kFirstEpiWarp;
     // the warps of a lane quarter split the columns of the tile
     const int cols_per_warp = max(16, p.BN / (kEpiWarps / 4));
     const int col_begin = min(p.BN, (ew >> 2) * cols_per_warp);
     const int col_end = min(p.BN, col_begin + cols_per_warp);
-    long long* bias64 = ctrl.bias64[ew];
-    // ReLU layers with a rounding right shift take the 32-bit requantization path
-    const bool fast_relu = p.splits == 1 && p.mode == ADAPTION_MODE_REQUANT && p.rq.relu && p.rq.shift > 0;
+    const int row = quarter * 32 + lane;   // row of the tile (and of this CTA's staging planes)
+    const uint32_t stage_lo = ring + p.stage_off;
+    const uint32_t stage_hi = stage_lo + (uint32_t)(kBM * p.BN);
+    const bool store_leader = ew == 0 && lane == 0;
     uint32_t tile_iter = 0;
     Counts cnt;
     long long vmax = 0;
     bool ok = true;
-    for (int t = worker; t < p.total_tiles && ok; t += workers, ++tile_iter) {
+    for (int t = worker; t < p.total_tiles; t += workers, ++tile_iter) {
       const TileCoord tc = decode_tile(t, p);
       const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
       const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
-      __syncwarp();
-      for (int c = col_begin + lane; c < col_end; c += 32) {
+      // per-column constants of this tile (the last barrier of the previous tile separates these
+      // writes from its readers): bias aligned to the accumulator, plus the rounding half on the
+      // fast path
+      for (int c = (int)threadIdx.x - 32 * kFirstEpiWarp; c < p.BN; c += 32 * kEpiWarps) {
         const int n = tc.n0 + c;
         long long b = 0;
         if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
-        if (fast_relu) {
-          // (Ch, Cl) of C = bias + rounding half, for requant_relu32: x = Ch, y = Cl
+        if (FAST) {
           const long long C = b + (1ll << (p.rq.shift - 1));
-          reinterpret_cast<int2*>(bias64)[c - col_begin] = make_int2((int)(C >> 16), (int)(C & 0xffff));
+          reinterpret_cast<int2*>(ctrl.colconst)[c] = make_int2((int)(C & 0xffff), (int)(C >> 16));
         } else {
-          bias64[c - col_begin] = b;
+          ctrl.colconst[c] = b;
         }
       }
-      __syncwarp();
+      // the previous tile's bulk stores must have read the staging planes before they are reused
+      if (p.staged && store_leader) bulk_wait_read_all();
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 0);
       bool w = wait_bar(smem_u32(&ctrl.tmem_full[buf]), bph, &ctrl, p);
-      w = __all_sync(0xffffffffu, w);
+      // one decision for all epilogue warps (they meet at barriers below), which also publishes the
+      // constants and the free staging planes
+      w = epi_bar_all(w);
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 1);
       if (!w) { ok = false; break; }
       tc_fence_after();
-      const int m = tc.m0 + (int)rank * kBM + quarter * 32 + lane;
+      const int m = tc.m0 + (int)rank * kBM + row;
       const bool row_ok = m < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)(NACC * p.BN);
-      for (int c0 = col_begin; c0 < col_end; c0 += 16) {
-        int32_t a0[16], a1[16], a2[16];
-        tmem_ld16(taddr + c0, a0);
-        if (NACC >= 2) tmem_ld16(taddr + p.BN + c0, a1);
-        if (NACC == 3) tmem_ld16(taddr + 2 * p.BN + c0, a2);
-        tmem_ld_wait();
+      // Sixteen columns per step.  The accumulators are handed back to the issuing warp as soon as
+      // the last step's values are in registers, before the arithmetic on them.
+      const bool storing = FAST || (p.splits == 1 && p.mode == ADAPTION_MODE_REQUANT);
+      bool released = false;
+      for (int c0 = col_begin; c0 < col_end || !released; c0 += 16) {
+        const bool have = c0 < col_end;
+        Acc8<NACC> xa, xb;
+        if (have) {
+          load_acc8<NACC>(taddr + c0, p.BN, xa);
+          load_acc8<NACC>(taddr + c0 + 8, p.BN, xb);
+          tmem_ld_wait();
+          pin_acc8<NACC>(xa);
+          pin_acc8<NACC>(xb);
+        }
+        if (c0 + 16 >= col_end) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
+            if (PAIR)
+              mbar_arrive_cluster(mapa_rank(bar, 0));
+            else
+              mbar_arrive(bar);
+          }
+          released = true;
+        }
+        if (!have) break;
         const int col = tc.n0 + c0;
-        const long long* bcol = bias64 + (c0 - col_begin);
-        if (p.splits > 1) {
-          // partial sums of this K range go to the int64 workspace
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const long long v = combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0);
-            if (row_ok && col + j < p.N && v != 0)
-              atomicAdd((unsigned long long*)(p.ws + (long long)m * p.ws_ld + col + j), (unsigned long long)v);
-          }
-        } else if (p.mode == ADAPTION_MODE_RANGE) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            long long v = combine<NACC>(a0[j], NACC >= 2 ? a1[j] : 0, NACC == 3 ? a2[j] : 0) + bcol[j];
-            if (p.rq.relu && v < 0) v = 0;
-            v = v < 0 ? -v : v;
-            if (row_ok && col + j < p.N) vmax = v > vmax ? v : vmax;
-          }
-        } else if (p.rq.relu) {
-          requant_store16<NACC, true>(a0, a1, a2, bcol, p, row_ok, m, col, cnt);
+        const long long* bcol = ctrl.colconst + c0;
+        if (!FAST && !storing) {
+          partial_or_range8<NACC>(xa, bcol, p, row_ok, m, col, vmax);
+          partial_or_range8<NACC>(xb, bcol + 8, p, row_ok, m, col + 8, vmax);
         } else {
-          requant_store16<NACC, false>(a0, a1, a2, bcol, p, row_ok, m, col, cnt);
+          uint32_t wq[8];
+          if (FAST) {
+            requant8_fast<NACC>(xa, bcol, p, row_ok && col < p.N, cnt, wq);
+            requant8_fast<NACC>(xb, bcol + 8, p, row_ok && col + 8 < p.N, cnt, wq + 4);
+          } else if (p.rq.relu) {
+            requant8<NACC, true>(xa, bcol, p, row_ok, col, cnt, wq);
+            requant8<NACC, true>(xb, bcol + 8, p, row_ok, col + 8, cnt, wq + 4);
+          } else {
+            requant8<NACC, false>(xa, bcol, p, row_ok, col, cnt, wq);
+            requant8<NACC, false>(xb, bcol + 8, p, row_ok, col + 8, cnt, wq + 4);
+          }
+          if (p.staged) {
+            const uint32_t off = staged_offset(row, c0 >> 4, p.BN);
+            st_shared_v4(stage_lo + off, plane_lo(wq));
+            if (p.rq.out_planes == 2) st_shared_v4(stage_hi + off, plane_hi(wq));
+          } else {
+            store16_global(wq, p, row_ok, m, col);
+          }
         }
       }
-      // accumulators of this buffer are in registers / memory: hand the buffer back to the leader
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
-        if (PAIR)
-          mbar_arrive_cluster(mapa_rank(bar, 0));
-        else
-          mbar_arrive(bar);
+      // staged planes complete -> one bulk-tensor store per plane (rows beyond M and columns beyond
+      // the channel pitch are clipped by the tensor map); the barrier also ends this tile's reads
+      // of the per-column constants
+      if (p.staged) fence_async_shared();
+      epi_bar_sync();
+      if (p.staged && store_leader) {
+        const int m_first = tc.m0 + (int)rank * kBM;
+        tma_store_2d(&map_y_lo, stage_lo, tc.n0, m_first);
+        if (p.rq.out_planes == 2) tma_store_2d(&map_y_hi, stage_hi, tc.n0, m_first);
+        bulk_commit();
       }
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 2);
     }
+    (void)ok;
+    if (p.staged && store_leader) bulk_wait_all();
     if (p.splits == 1) {
       if (p.mode == ADAPTION_MODE_RANGE)
         flush_max_warp(vmax, p.stats);
@@ -1037,6 +1198,8 @@ struct TcConfig {
   uint32_t kb_bytes = 0;
   bool pair = false;           // two CTAs per 256-row tile (cta_group::2)
   int tile_m = kBM;
+  bool staged = false;         // outputs staged in shared memory and written by bulk-tensor stores
+  uint32_t stage_out_bytes = 0, stage_off = 0;
   size_t smem_bytes = 0;
   size_t workspace_bytes = 0;
 };
@@ -1116,24 +1279,11 @@ TcConfig make_config(const GemmProblem& g) {
   // Large unsplit problems run as CTA pairs: 256-row tiles, each CTA stages its own 128 rows of A
   // and only half of the weight rows, which cuts the bytes (and TMA rows) per MAC by a quarter.
   const int pair_env = env_int("ADAPTION_TC_PAIR", -1);
-  // (measured: pairs win once the reduction is long, K >= 2304 bytes per plane row, and lose on
-  // short reductions where per-tile costs dominate)
+  // (measured: pairs win from K = 1152 bytes per plane row on; 256 x 64 pair tiles with two
+  // accumulator sets were tried for medium reductions and lost to these once the epilogue hands the
+  // accumulators back early)
   const bool pair_ok = c.splits == 1 && g.M >= 1024 && (sms % 2) == 0;
-  c.pair = pair_ok && c.BN == 128 && c.BK == 128 && c.num_kb >= 18;
-  // Medium reductions (1152 <= K < 4608 bytes per plane row) do better on 256 x 64 pair tiles: two
-  // accumulator sets fit in TMEM, so the epilogue of one tile overlaps the MMAs of the next, which
-  // outweighs the slower N = 64 instruction (measured +5..7% on the conv2_2 / conv3 / conv4_1 shapes).
-  const bool narrow = pair_ok && c.BN == 128 && c.BK == 128 && c.num_kb >= 9 && c.num_kb < 36 &&
-                      forced_bn == 0 && pair_env != 0;
-  if (narrow) {
-    c.pair = true;
-    c.BN = 64;
-    c.tiles_n = (int)((g.N + c.BN - 1) / c.BN);
-    c.acc_bufs = 512 / (c.nacc * c.BN);
-    if (c.acc_bufs > kMaxAccBufs) c.acc_bufs = kMaxAccBufs;
-    c.tmem_cols = 32;
-    while (c.tmem_cols < (uint32_t)(c.acc_bufs * c.nacc * c.BN)) c.tmem_cols <<= 1;
-  }
+  c.pair = pair_ok && c.BN == 128 && c.BK == 128 && c.num_kb >= 9;
   if (pair_env == 0) c.pair = false;
   if (pair_env == 1 && c.splits == 1 && (sms % 2) == 0) c.pair = true;
   if (c.pair) {
@@ -1142,7 +1292,14 @@ TcConfig make_config(const GemmProblem& g) {
   }
   c.a_bytes = (uint32_t)(kBM * c.BK);
   c.b_bytes = (uint32_t)((c.pair ? c.BN / 2 : c.BN) * c.BK);
-  const size_t budget = 232448 - sizeof(Ctrl) - 2048;
+  // Output staging: one plane of 128 rows x BN bytes per output byte plane.  Needs a tensor map over
+  // the output planes (pitch a multiple of 16 bytes and at least one tile wide) and no int16 copy.
+  const int out_planes = g.y.fmt.n_bits > 8 ? 2 : 1;
+  c.staged = g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.y.q16 == nullptr && g.y.lo != nullptr &&
+             g.y.c_stride >= c.BN && g.y.c_stride % 16 == 0 && env_int("ADAPTION_TC_STAGED", 1) != 0;
+  c.stage_out_bytes = c.staged ? (uint32_t)(kBM * c.BN * out_planes) : 0u;
+  // dynamic shared memory: everything up to the per-block limit except the control block
+  const size_t budget = 232448 - sizeof(Ctrl) - 256 - c.stage_out_bytes;
   // group short k-blocks so that a stage carries roughly 768 tensor-pipe cycles of work or more
   {
     const int products = c.nax * c.nbw;
@@ -1168,6 +1325,12 @@ TcConfig make_config(const GemmProblem& g) {
   }
   c.stage_bytes = (uint32_t)c.kps * c.kb_bytes;
   c.stages = (int)((budget - 1024 - c.b_res_bytes) / c.stage_bytes);
+  if (c.staged && c.stages < 3) {
+    // not enough room for a useful ring beside the staging planes: store directly instead
+    c.stages = (int)((budget + c.stage_out_bytes - 1024 - c.b_res_bytes) / c.stage_bytes);
+    c.staged = false;
+    c.stage_out_bytes = 0;
+  }
   if (c.stages > kMaxStages) c.stages = kMaxStages;
   const int stage_cap = env_int("ADAPTION_TC_STAGES", 0);   // experiment knob: shallower ring
   if (stage_cap >= 2 && stage_cap < c.stages) c.stages = stage_cap;
@@ -1175,7 +1338,8 @@ TcConfig make_config(const GemmProblem& g) {
   c.mma_warps = kMmaWarps;
   const int mmaw_env = env_int("ADAPTION_TC_MMAW", 0);      // experiment knob: force one issuing warp
   if (mmaw_env == 1) c.mma_warps = 1;
-  c.smem_bytes = (size_t)c.stages * c.stage_bytes + 1024 + c.b_res_bytes;
+  c.stage_off = (uint32_t)(((size_t)c.stages * c.stage_bytes + c.b_res_bytes + 1023) & ~(size_t)1023);
+  c.smem_bytes = (size_t)c.stage_off + 1024 + c.stage_out_bytes;
   c.ok = true;
   return c;
 }
@@ -1205,11 +1369,11 @@ bool encode_im2col_nhwc(CUtensorMap* map, const void* base, const adaption_conv_
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NAX, int NBW, bool PAIR, bool GROUPED>
+template <int NAX, int NBW, bool PAIR, bool GROUPED, bool FAST>
 int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem, cudaStream_t stream) {
   static size_t attr_size = 0;
   if (smem > attr_size) {
-    const cudaError_t ae = cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>,
+    const cudaError_t ae = cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, FAST>,
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (ae != cudaSuccess) return cuda_failure(ae, "lp_gemm_kernel shared-memory attribute");
     attr_size = smem;
@@ -1230,7 +1394,8 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
     cfg.numAttrs = 1;
   }
   const cudaError_t le =
-      cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED>, maps[0], maps[1], maps[2], maps[3], p);
+      cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, FAST>, maps[0], maps[1], maps[2], maps[3], maps[4],
+                         maps[5], p);
   if (le != cudaSuccess) {
     (void)cudaGetLastError();
     return cuda_failure(le, "lp_gemm_kernel launch");
@@ -1242,11 +1407,19 @@ template <int NAX, int NBW>
 int launch_either(bool pair, const CUtensorMap* maps, const TcParams& p, int grid, size_t smem,
                   cudaStream_t stream) {
   const bool grouped = p.kps > 1 || p.b_resident != 0;
-  if (pair)
-    return grouped ? launch_kernel<NAX, NBW, true, true>(maps, p, grid, smem, stream)
-                   : launch_kernel<NAX, NBW, true, false>(maps, p, grid, smem, stream);
-  return grouped ? launch_kernel<NAX, NBW, false, true>(maps, p, grid, smem, stream)
-                 : launch_kernel<NAX, NBW, false, false>(maps, p, grid, smem, stream);
+  const bool fast = p.fast_relu != 0;
+  if (pair) {
+    if (grouped)
+      return fast ? launch_kernel<NAX, NBW, true, true, true>(maps, p, grid, smem, stream)
+                  : launch_kernel<NAX, NBW, true, true, false>(maps, p, grid, smem, stream);
+    return fast ? launch_kernel<NAX, NBW, true, false, true>(maps, p, grid, smem, stream)
+                : launch_kernel<NAX, NBW, true, false, false>(maps, p, grid, smem, stream);
+  }
+  if (grouped)
+    return fast ? launch_kernel<NAX, NBW, false, true, true>(maps, p, grid, smem, stream)
+                : launch_kernel<NAX, NBW, false, true, false>(maps, p, grid, smem, stream);
+  return fast ? launch_kernel<NAX, NBW, false, false, true>(maps, p, grid, smem, stream)
+              : launch_kernel<NAX, NBW, false, false, false>(maps, p, grid, smem, stream);
 }
 
 
@@ -1377,7 +1550,7 @@ int launch_tensor(const GemmProblem& g) {
   // plane 0 is the high byte plane when there are two, else the single plane
   const void* xa[2] = {c.nax == 2 ? g.x.hi : g.x.lo, g.x.lo};
   const void* wb[2] = {c.nbw == 2 ? g.w.hi : g.w.lo, g.w.lo};
-  CUtensorMap maps[4];
+  CUtensorMap maps[6];   // activation planes, weight planes, output planes (hi, lo)
   std::memset(maps, 0, sizeof(maps));
   for (int i = 0; i < 2; ++i) {
     bool ok;
@@ -1392,6 +1565,18 @@ int launch_tensor(const GemmProblem& g) {
     if (!encode_tiled_2d(&maps[2 + i], wb[i], wk, (uint64_t)g.N, wpitch, (uint32_t)c.BK,
                          (uint32_t)(c.pair ? c.BN / 2 : c.BN), c.swizzle))
       return ADAPTION_ERR_CUDA;
+  }
+
+  if (c.staged) {
+    const CUtensorMapSwizzle yswz = c.BN == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                                : (c.BN == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    const void* planes[2] = {g.y.hi, g.y.lo};
+    for (int i = 0; i < 2; ++i) {
+      if (planes[i] == nullptr) continue;      // single-plane outputs have no high plane
+      if (!encode_tiled_2d(&maps[4 + i], planes[i], (uint64_t)g.y.c_stride, (uint64_t)g.M, (uint64_t)g.y.c_stride,
+                           (uint32_t)c.BN, (uint32_t)kBM, yswz))
+        return ADAPTION_ERR_CUDA;
+    }
   }
 
   TcParams p;
@@ -1419,6 +1604,21 @@ int launch_tensor(const GemmProblem& g) {
     p.y_hi = (int8_t*)g.y.hi; p.y_lo = (uint8_t*)g.y.lo; p.y_q16 = g.y.q16; p.y_stride = g.y.c_stride;
   } else {
     p.rq = RequantParams{0, g.relu ? 1 : 0, 0, 0, 1};
+  }
+  p.staged = c.staged ? 1 : 0;
+  p.stage_off = c.stage_off;
+  if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && p.rq.shift >= 9 && p.rq.shift <= 31 &&
+      g.N % 8 == 0 && env_int("ADAPTION_TC_FAST", 1) != 0) {
+    // 32-bit bounds of the fast epilogue (see shifted32): with a reduction of kred bytes per plane row
+    // |hh| <= kred 2^14, |mid| <= kred 65280, |ll| <= kred 65025, and |C| < 2^(15 + bias_shift) + 2^(shift-1)
+    const long long kred = (long long)c.num_kb * c.BK;
+    const long long cmax = (g.bias != nullptr ? (1ll << (15 + g.bias_shift)) : 0ll) + (1ll << (p.rq.shift - 1));
+    const long long hmax = kred * 16384 + (cmax >> 16) + 1;
+    const long long tmax = kred * 65280 + ((kred * 65025 + 65535) >> 8) + 1;
+    const long long lim = 1ll << 31;
+    bool ok32 = kred * 65025 + 65535 < lim && tmax < lim && hmax + (tmax >> 8) + 1 < lim;
+    if (p.rq.shift < 16) ok32 = ok32 && (hmax << (16 - p.rq.shift)) + (tmax >> (p.rq.shift - 8)) + 1 < lim;
+    p.fast_relu = ok32 ? 1 : 0;
   }
   p.ws = (long long*)g.workspace; p.ws_ld = g.N;
   p.stats = g.stats;

@@ -27,14 +27,17 @@ def _pick_f_out(acc, bq, fb, F, relu, n_out):
 
 
 def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, algo, with_bias=True,
-                  extreme=False, f_out=None):
+                  extreme=False, f_out=None, with_q16=True, mag_bits=None, fmts=None):
+    """`with_q16=False` leaves out the optional int16 copy of the output, which lets the tensor-core
+    kernel stage its byte planes in shared memory and write them with bulk-tensor stores.
+    `mag_bits` limits operand magnitudes (small accumulators -> short requantization shifts)."""
     cs = B.pad_to(Cin, 32)
-    xq = _rand_q(rng, (N, H, W, Cin), nx, 0.4)
-    wq = _rand_q(rng, (K, R, R, Cin), nw)
+    xq = _rand_q(rng, (N, H, W, Cin), nx if mag_bits is None else min(nx, mag_bits[0]), 0.4)
+    wq = _rand_q(rng, (K, R, R, Cin), nw if mag_bits is None else min(nw, mag_bits[1]))
     if extreme:   # drive every byte plane to its extremes
         xq[:] = np.where(rng.random(xq.shape) < 0.5, -(1 << (nx - 1)), (1 << (nx - 1)) - 1)
         wq[:] = np.where(rng.random(wq.shape) < 0.5, -(1 << (nw - 1)), (1 << (nw - 1)) - 1)
-    fx, fw = nx - 3, nw - 1
+    fx, fw = (nx - 3, nw - 1) if fmts is None else fmts
     bq = _rand_q(rng, (K,), nw) if with_bias else None
     acc = orc.conv_acc(xq, wq, (pad, pad), (stride, stride))
     F = fx + fw
@@ -46,7 +49,7 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
     x = to_qtensor(xq.reshape(-1, Cin), nx, fx, cs)
     w = to_qtensor(wq.reshape(-1, Cin), nw, fw, cs)
     ycs = B.pad_to(K, 32)
-    y = B.QTensor.empty(N * OH * OW, K, n_out, f_out, ycs, with_q16=True)
+    y = B.QTensor.empty(N * OH * OW, K, n_out, f_out, ycs, with_q16=with_q16)
     y.lo.fill_(0x3C)
     if y.hi is not None:
         y.hi.fill_(0x3C)
@@ -67,12 +70,14 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
     got = from_qtensor(y).reshape(want.shape)
     bad = np.argwhere(got != want)
     assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}: got {got[tuple(bad[0])]} want {want[tuple(bad[0])]}"
-    assert np.array_equal(q16_of(y).reshape(want.shape), want)
+    if with_q16:
+        assert np.array_equal(q16_of(y).reshape(want.shape), want)
     assert y.padding_is_zero()
     assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+    return cnt
 
 
-def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out=None):
+def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out=None, with_q16=True):
     xq = _rand_q(rng, (Bsz, K), nx, 0.4)
     wq = _rand_q(rng, (O, K), nw)
     fx, fw = nx - 2, nw - 1
@@ -84,8 +89,10 @@ def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out
     want, cnt = orc.epilogue(acc, bq, fw, F, relu, n_out, f_out)
     x = to_qtensor(xq, nx, fx)
     w = to_qtensor(wq, nw, fw)
-    y = B.QTensor.empty(Bsz, O, n_out, f_out, None, with_q16=True)
+    y = B.QTensor.empty(Bsz, O, n_out, f_out, None, with_q16=with_q16)
     y.lo.fill_(0x3C)
+    if y.hi is not None:
+        y.hi.fill_(0x3C)
     bias_dev = dev(bq) if with_bias else None
     need = B.adaption_lp_ip_workspace_bytes(Bsz, K, O, x.fmt(), w.fmt(), algo)
     ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
@@ -100,7 +107,8 @@ def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out
     got = from_qtensor(y)
     bad = np.argwhere(got != want)
     assert bad.size == 0, f"{len(bad)} mismatches, first at {bad[:5].tolist()}"
-    assert np.array_equal(q16_of(y), want)
+    if with_q16:
+        assert np.array_equal(q16_of(y), want)
     assert y.padding_is_zero()
     assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
     return need
@@ -170,6 +178,44 @@ def test_conv_tensor(case, cta_mode):
                   B.ALGO_TENSOR)
 
 
+@pytest.mark.parametrize("case", TC_CONV)
+def test_conv_tensor_staged_stores(case, cta_mode):
+    """Same cases without the int16 copy: byte planes leave through shared memory and bulk-tensor
+    stores, ReLU layers with shifts of 9 and more take the paired 16-bit epilogue."""
+    N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu = case
+    run_conv_case(np.random.default_rng(sum(case) + 1), N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu,
+                  B.ALGO_TENSOR, with_q16=False)
+
+
+@pytest.mark.parametrize("shift", [2, 8, 9, 12, 15, 16, 17, 22])
+@pytest.mark.parametrize("n_out", [16, 8])
+def test_fast_epilogue_shifts_and_saturation(shift, n_out, cta_mode):
+    """ReLU layers across the requantization shifts on both sides of the fast epilogue's limits
+    (9 <= shift: 32-bit path, its two forms split at 16), with outputs that saturate: operands of
+    reduced magnitude so that short shifts still give in-range values."""
+    nx = nw = 16
+    fmts = (4, 8) if shift <= 12 else ((8, 12) if shift <= 17 else (13, 15))
+    f_out = sum(fmts) - shift
+    if not 0 <= f_out <= n_out - 1:
+        pytest.skip("shift not reachable with this output width")
+    mag = (min(16, (shift + 8) // 2), min(16, (shift + 7) // 2))   # accumulators of about 2^(shift + 8)
+    cnt = run_conv_case(np.random.default_rng(100 + shift), 2, 24, 24, 128, 128, 3, 1, 1, nx, nw, n_out, True,
+                        B.ALGO_TENSOR, f_out=f_out, with_q16=False, mag_bits=mag, fmts=fmts)
+    assert cnt.zeros > 0
+    if n_out == 8:
+        assert cnt.sat_pos > 0   # the case does exercise saturation
+
+
+def test_epilogue_variants_agree(monkeypatch):
+    """Cross-path identity: the generic 64-bit epilogue with direct stores, the staged stores and the
+    fast paired path all give the oracle's bits on the same case."""
+    case = (2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True)
+    for fast, staged in (("0", "0"), ("0", "1"), ("1", "0"), ("1", "1")):
+        monkeypatch.setenv("ADAPTION_TC_FAST", fast)
+        monkeypatch.setenv("ADAPTION_TC_STAGED", staged)
+        run_conv_case(np.random.default_rng(5), *case, B.ALGO_TENSOR, with_q16=False, mag_bits=(10, 10))
+
+
 def test_conv_tensor_extreme_operands(cta_mode):
     # every operand at +-full scale: largest possible partial sums in all three accumulators
     run_conv_case(np.random.default_rng(1), 1, 32, 32, 256, 128, 3, 1, 1, 16, 16, 16, False, B.ALGO_TENSOR,
@@ -187,6 +233,12 @@ TC_IP = [(8, 800, 500, 16, 16, 16, True), (70, 1000, 260, 16, 16, 16, False), (2
 def test_ip_tensor(case, cta_mode):
     Bsz, K, O, nx, nw, n_out, relu = case
     run_ip_case(np.random.default_rng(sum(case)), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_TENSOR)
+
+
+@pytest.mark.parametrize("case", TC_IP)
+def test_ip_tensor_staged_stores(case, cta_mode):
+    Bsz, K, O, nx, nw, n_out, relu = case
+    run_ip_case(np.random.default_rng(sum(case) + 1), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_TENSOR, with_q16=False)
 
 
 def test_ip_tensor_split_k_paths():
