@@ -125,7 +125,9 @@ ADAPTION_API int adaption_lp_act(const float* d_x_f32, const adaption_qtensor* h
  * contribute 0, the sum is exact.  x and w must share c_stride.  bias_q (int16 [K], may be
  * NULL) has bias_frac_bits <= x.fmt.frac_bits + w.fmt.frac_bits.  In RANGE mode y is ignored.
  * The workspace query returns the bytes the call needs (possibly 0); the workspace contents
- * need no initialisation.  d_stats must not be NULL. */
+ * need no initialisation.  (Layers with at most 4 input channels whose R*S*C taps fit 32 bytes,
+ * e.g. the first 3x3 layer of an RGB network, gather their taps into packed planes there: 64 bytes
+ * per output pixel.)  d_stats must not be NULL. */
 ADAPTION_API size_t adaption_lp_conv_workspace_bytes(const adaption_conv_shape* h_shape, adaption_qfmt fx,
                                         adaption_qfmt fw, int64_t c_stride, int32_t algo);
 ADAPTION_API int adaption_lp_conv_fwd(const adaption_conv_shape* h_shape, adaption_qtensor x,

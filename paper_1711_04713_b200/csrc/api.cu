@@ -110,6 +110,12 @@ static int dispatch(const GemmProblem& g, int32_t algo) {
   if (algo != ADAPTION_ALGO_AUTO && algo != ADAPTION_ALGO_TENSOR && algo != ADAPTION_ALGO_DIRECT)
     return ADAPTION_ERR_INVALID_ARG;
   if (g.M == 0) return ADAPTION_OK;
+  if (algo != ADAPTION_ALGO_DIRECT && pack_taps_applicable(g)) {
+    const size_t need = pack_taps_workspace(g);
+    if (g.workspace == nullptr || g.workspace_bytes < need) return ADAPTION_ERR_WORKSPACE;
+    if (!aligned16(g.workspace)) return ADAPTION_ERR_ALIGNMENT;
+    return launch_pack_taps(g);
+  }
   const bool tensor_ok = tensor_path_supported(g);
   if (algo == ADAPTION_ALGO_TENSOR && !tensor_ok) return ADAPTION_ERR_UNSUPPORTED;
   if (algo != ADAPTION_ALGO_DIRECT && tensor_ok) {
@@ -167,6 +173,7 @@ size_t adaption_lp_conv_workspace_bytes(const adaption_conv_shape* h_shape, adap
   if (build_conv_problem(h_shape, x, w, nullptr, 0, 0, ADAPTION_MODE_RANGE, y, fake_stats, nullptr, 0,
                          nullptr, g) != ADAPTION_OK)
     return 0;
+  if (pack_taps_applicable(g)) return pack_taps_workspace(g);
   return tensor_path_supported(g) ? tensor_path_workspace(g) : 0;
 }
 

@@ -142,6 +142,11 @@ int launch_direct(const GemmProblem& p);
 bool tensor_path_supported(const GemmProblem& p);
 size_t tensor_path_workspace(const GemmProblem& p);
 int launch_tensor(const GemmProblem& p);
+// Convolutions with at most 4 input channels whose taps fit one 32-byte row: gather the taps into
+// packed planes in the workspace and run the layer as an inner product on the tensor-core path.
+bool pack_taps_applicable(const GemmProblem& p);
+size_t pack_taps_workspace(const GemmProblem& p);
+int launch_pack_taps(const GemmProblem& p);
 // bias/ReLU/requantize (or range) of an int64 accumulator matrix acc[M][ld] -> y
 int launch_finalize(const int64_t* acc, int64_t ld, const GemmProblem& p);
 

@@ -301,11 +301,15 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t 
         "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int32_t (&r)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr)
-               : "memory");
+// sixteen consecutive columns: the first eight into `lo`, the next eight into `hi`
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&lo)[8], int32_t (&hi)[8]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(lo[0]), "=r"(lo[1]), "=r"(lo[2]), "=r"(lo[3]), "=r"(lo[4]), "=r"(lo[5]), "=r"(lo[6]), "=r"(lo[7]),
+        "=r"(hi[0]), "=r"(hi[1]), "=r"(hi[2]), "=r"(hi[3]), "=r"(hi[4]), "=r"(hi[5]), "=r"(hi[6]), "=r"(hi[7])
+      : "r"(taddr)
+      : "memory");
 }
 // Placed after tcgen05.wait::ld: ties the loaded registers to that point so that no use of them can
 // be scheduled before the wait (the load fills them asynchronously).
@@ -478,13 +482,7 @@ __device__ __forceinline__ int32_t requant_shift_right(long long v, long long ha
 //   shift >= 16:  floor((H + floor(T / 2^8)) / 2^(shift-16))
 //   shift <  16:  H * 2^(16-shift) + floor(T / 2^(shift-8))
 // The host checks from the reduction length that none of these 32-bit quantities can overflow
-// (otherwise the layer takes the generic 64-bit epilogue).  The divisions by 2^8 are taken as the
-// high word of a product with 2^24, which runs on the multiplier beside the integer ALU.
-__device__ __forceinline__ int32_t mad_hi(int32_t a, int32_t b, int32_t c) {
-  int32_t d;
-  asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
+// (otherwise the layer takes the generic 64-bit epilogue).
 __device__ __forceinline__ int32_t mad_lo(int32_t a, int32_t b, int32_t c) {
   int32_t d;
   asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -496,9 +494,9 @@ __device__ __forceinline__ int32_t shifted32(int32_t x0, int32_t x1, int32_t x2,
   const int32_t hh = NACC == 3 ? x0 : 0;
   const int32_t mid = NACC == 3 ? x1 : (NACC == 2 ? x0 : 0);
   const int32_t ll = NACC == 3 ? x2 : (NACC == 2 ? x1 : x0);
-  const int32_t T = mad_hi(ll + c.x, 1 << 24, mid);
+  const int32_t T = mid + ((ll + c.x) >> 8);
   const int32_t H = hh + c.y;
-  if (WIDE) return mad_hi(T, 1 << 24, H) >> (shift - 16);
+  if (WIDE) return (H + (T >> 8)) >> (shift - 16);
   return mad_lo(H, 1 << (16 - shift), T >> (shift - 8));
 }
 
@@ -524,11 +522,12 @@ template <int NACC>
 struct Acc8 {
   int32_t a[3][8];
 };
+// sixteen columns as two groups of eight, one load instruction per accumulator
 template <int NACC>
-__device__ __forceinline__ void load_acc8(uint32_t taddr, int bn, Acc8<NACC>& x) {
-  tmem_ld8(taddr, x.a[0]);
-  if (NACC >= 2) tmem_ld8(taddr + (uint32_t)bn, x.a[1]);
-  if (NACC == 3) tmem_ld8(taddr + 2u * (uint32_t)bn, x.a[2]);
+__device__ __forceinline__ void load_acc16(uint32_t taddr, int bn, Acc8<NACC>& x, Acc8<NACC>& y) {
+  tmem_ld16(taddr, x.a[0], y.a[0]);
+  if (NACC >= 2) tmem_ld16(taddr + (uint32_t)bn, x.a[1], y.a[1]);
+  if (NACC == 3) tmem_ld16(taddr + 2u * (uint32_t)bn, x.a[2], y.a[2]);
 }
 template <int NACC>
 __device__ __forceinline__ void pin_acc8(Acc8<NACC>& x) {
@@ -1033,23 +1032,27 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     Counts cnt;
     long long vmax = 0;
     bool ok = true;
+    int const_n0 = -1;          // first column of the tile whose constants are staged
     for (int t = worker; t < p.total_tiles; t += workers, ++tile_iter) {
       const TileCoord tc = decode_tile(t, p);
       const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
       const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
       // per-column constants of this tile (the last barrier of the previous tile separates these
       // writes from its readers): bias aligned to the accumulator, plus the rounding half on the
-      // fast path
-      for (int c = (int)threadIdx.x - 32 * kFirstEpiWarp; c < p.BN; c += 32 * kEpiWarps) {
-        const int n = tc.n0 + c;
-        long long b = 0;
-        if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
-        if (FAST) {
-          const long long C = b + (1ll << (p.rq.shift - 1));
-          reinterpret_cast<int2*>(ctrl.colconst)[c] = make_int2((int)(C & 0xffff), (int)(C >> 16));
-        } else {
-          ctrl.colconst[c] = b;
+      // fast path.  Kept when the tile covers the same columns as the previous one.
+      if (tc.n0 != const_n0) {
+        for (int c = (int)threadIdx.x - 32 * kFirstEpiWarp; c < p.BN; c += 32 * kEpiWarps) {
+          const int n = tc.n0 + c;
+          long long b = 0;
+          if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
+          if (FAST) {
+            const long long C = b + (1ll << (p.rq.shift - 1));
+            reinterpret_cast<int2*>(ctrl.colconst)[c] = make_int2((int)(C & 0xffff), (int)(C >> 16));
+          } else {
+            ctrl.colconst[c] = b;
+          }
         }
+        const_n0 = tc.n0;
       }
       // the previous tile's bulk stores must have read the staging planes before they are reused
       if (p.staged && store_leader) bulk_wait_read_all();
@@ -1072,8 +1075,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const bool have = c0 < col_end;
         Acc8<NACC> xa, xb;
         if (have) {
-          load_acc8<NACC>(taddr + c0, p.BN, xa);
-          load_acc8<NACC>(taddr + c0 + 8, p.BN, xb);
+          load_acc16<NACC>(taddr + c0, p.BN, xa, xb);
           tmem_ld_wait();
           pin_acc8<NACC>(xa);
           pin_acc8<NACC>(xb);

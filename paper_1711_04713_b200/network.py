@@ -73,8 +73,13 @@ class LPNetwork:
         self.x_fmt_dev = torch.zeros(2, dtype=torch.int32, device=device)
         self.x_max_dev = torch.zeros(1, dtype=torch.float32, device=device)
         self.x_stats = B.new_stats(device)
-        self.xq = B.QTensor.empty(batch * self.in_h * self.in_w, in_c, n_bits, 0, act_c_stride(in_c),
-                                  keep_q16, device)
+        # A first convolution with few input channels gathers its taps into packed rows inside the
+        # library (it needs no 32-byte pitch), so the network input keeps the smallest pitch.
+        first = params[0] if params else None
+        few = (first is not None and first["type"] == "conv" and in_c <= 4
+               and first["w"].shape[1] * first["w"].shape[2] * in_c <= 32)
+        in_cs = B.pad_to(in_c, 16) if few else act_c_stride(in_c)
+        self.xq = B.QTensor.empty(batch * self.in_h * self.in_w, in_c, n_bits, 0, in_cs, keep_q16, device)
         h, w, c, cs = self.in_h, self.in_w, in_c, self.xq.c_stride
         flat = False
         for p in params:

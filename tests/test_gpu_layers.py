@@ -27,11 +27,11 @@ def _pick_f_out(acc, bq, fb, F, relu, n_out):
 
 
 def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, algo, with_bias=True,
-                  extreme=False, f_out=None, with_q16=True, mag_bits=None, fmts=None):
+                  extreme=False, f_out=None, with_q16=True, mag_bits=None, fmts=None, cs=None):
     """`with_q16=False` leaves out the optional int16 copy of the output, which lets the tensor-core
     kernel stage its byte planes in shared memory and write them with bulk-tensor stores.
     `mag_bits` limits operand magnitudes (small accumulators -> short requantization shifts)."""
-    cs = B.pad_to(Cin, 32)
+    cs = B.pad_to(Cin, 32) if cs is None else cs
     xq = _rand_q(rng, (N, H, W, Cin), nx if mag_bits is None else min(nx, mag_bits[0]), 0.4)
     wq = _rand_q(rng, (K, R, R, Cin), nw if mag_bits is None else min(nw, mag_bits[1]))
     if extreme:   # drive every byte plane to its extremes
@@ -214,6 +214,32 @@ def test_epilogue_variants_agree(monkeypatch):
         monkeypatch.setenv("ADAPTION_TC_FAST", fast)
         monkeypatch.setenv("ADAPTION_TC_STAGED", staged)
         run_conv_case(np.random.default_rng(5), *case, B.ALGO_TENSOR, with_q16=False, mag_bits=(10, 10))
+
+
+FEW_CHANNELS = [
+    # N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, channel pitch
+    (8, 32, 32, 3, 64, 3, 1, 1, 16, 16, 16, True, 16),    # RGB 3x3 (27 taps x channels), pitch 16
+    (8, 28, 28, 1, 20, 5, 0, 1, 16, 16, 16, True, 16),    # one channel, 5x5 valid (25 taps)
+    (3, 41, 37, 2, 72, 4, 2, 2, 16, 16, 16, False, 32),   # two channels, 4x4, stride 2, pad 2, ragged N
+    (4, 30, 30, 4, 128, 2, 0, 1, 8, 8, 8, True, 16),      # four channels, 2x2, single int8 pass
+    (2, 40, 24, 3, 40, 3, 1, 1, 16, 8, 12, True, 48),     # mixed widths, pitch 48
+    (16, 9, 9, 4, 16, 1, 0, 1, 12, 12, 12, False, 16),    # 1x1, M just above the threshold
+]
+
+
+@pytest.mark.parametrize("case", FEW_CHANNELS)
+@pytest.mark.parametrize("with_q16", [True, False])
+def test_conv_few_channels_packed_taps(case, with_q16):
+    """Layers with at most 4 input channels whose taps fit 32 bytes run as a packed inner product
+    (taps gathered into the workspace): image borders, strides, every channel count, both stores."""
+    N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, cs = case
+    run_conv_case(np.random.default_rng(sum(case)), N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu,
+                  B.ALGO_AUTO, with_q16=with_q16, cs=cs)
+    shp = B.conv_shape(N, H, W, Cin, K, R, R, pad, stride)
+    OH = (H + 2 * pad - R) // stride + 1
+    OW = (W + 2 * pad - R) // stride + 1
+    need = B.adaption_lp_conv_workspace_bytes(shp, B.adaption_qfmt(nx, 0), B.adaption_qfmt(nw, 0), cs, B.ALGO_AUTO)
+    assert need >= N * OH * OW * 32 * ((nx > 8) + 1)      # the packed planes are in the workspace
 
 
 def test_conv_tensor_extreme_operands(cta_mode):
