@@ -1,0 +1,84 @@
+"""CPU oracle for stochastic rounding (test infrastructure, not the product).
+
+Paper Sec. 2.4: a stochastically rounded value is one of the two nearest fixed-point values,
+drawn so that its expectation is the unrounded value.  The paper fixes neither the random
+number generator nor how a draw is compared with the fraction, so both are fixed here
+(readings S1-S3) and the CUDA path follows them bit for bit:
+
+S1  The real value y = x * 2^f is split as y = floor(y) + frac, 0 <= frac < 1, exactly (x is
+    fp32, so both parts are exact in fp64).  The result is floor(y) + 1 with probability
+    T / 2^32, T = floor(frac * 2^32), else floor(y); then it is saturated like the deterministic
+    quantizer (NaN -> 0, +-Inf saturate).  A value already on the grid never moves.
+S2  The draw for element i (index in the logical [outer][inner] order, padding excluded) is the
+    32-bit word  R_i = Philox4x32-10(counter = (i >> 2, 0, 0) as (lo32, hi32, 0, 0),
+    key = (seed lo32, seed hi32))[i & 3]  and the value moves up iff R_i < T.
+S3  Philox4x32-10 is the counter-based generator of Salmon, Moraes, Dror and Shaw, "Parallel
+    random numbers: as easy as 1, 2, 3" (SC'11), written out below from its definition: ten
+    rounds of two 32x32 -> 64-bit multiplications with the constants 0xD2511F53 and 0xCD9E8D57,
+    the key bumped by 0x9E3779B9 and 0xBB67AE85 between rounds.
+
+Plain numpy, vectorised over elements; no code is shared with the CUDA path.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+_M0 = np.uint64(0xD2511F53)
+_M1 = np.uint64(0xCD9E8D57)
+_W0 = np.uint64(0x9E3779B9)
+_W1 = np.uint64(0xBB67AE85)
+_MASK = np.uint64(0xFFFFFFFF)
+_S32 = np.uint64(32)
+
+
+def philox4x32_10(counter, key):
+    """counter: four arrays (or scalars) of 32-bit words, key: two 32-bit words -> four arrays of
+    32-bit words.  Definition: Salmon et al. 2011, Sec. 3.3 (Philox-4x32 with 10 rounds)."""
+    c0, c1, c2, c3 = (np.asarray(c, dtype=np.uint64) & _MASK for c in counter)
+    k0 = np.uint64(key[0]) & _MASK
+    k1 = np.uint64(key[1]) & _MASK
+    for rnd in range(10):
+        if rnd > 0:                       # key schedule: bumped before every round but the first
+            k0 = (k0 + _W0) & _MASK
+            k1 = (k1 + _W1) & _MASK
+        p0 = _M0 * c0                     # 32 x 32 -> 64 bit products (operands below 2^32)
+        p1 = _M1 * c2
+        hi0, lo0 = p0 >> _S32, p0 & _MASK
+        hi1, lo1 = p1 >> _S32, p1 & _MASK
+        c0, c1, c2, c3 = (hi1 ^ c1 ^ k0) & _MASK, lo1, (hi0 ^ c3 ^ k1) & _MASK, lo0
+    return c0, c1, c2, c3
+
+
+def draws(n: int, seed: int) -> np.ndarray:
+    """R_i for i in [0, n): reading S2."""
+    i = np.arange(n, dtype=np.uint64)
+    blk = i >> np.uint64(2)
+    out = philox4x32_10((blk & _MASK, blk >> _S32, np.zeros_like(blk), np.zeros_like(blk)),
+                        (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    words = np.stack(out, axis=1)                       # [n, 4]
+    return words[np.arange(n), (i & np.uint64(3)).astype(np.int64)].astype(np.uint64)
+
+
+def quantize_stochastic(x, n_bits: int, frac_bits: int, seed: int, relu: bool = False):
+    """Stochastically rounded canonical integers (int16) of a fp32 tensor, with counters
+    (zeros, sat_pos, sat_neg) like the deterministic quantizer.  Readings S1-S2."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    flat = x.reshape(-1).astype(np.float64)
+    qmin, qmax = -(1 << (n_bits - 1)), (1 << (n_bits - 1)) - 1
+    y = flat * float(2.0 ** frac_bits)                  # exact: power-of-two scaling of an fp32 value
+    nan = np.isnan(y)
+    y = np.where(nan, 0.0, y)
+    # far outside the range the fraction is irrelevant: clamp first so that floor() stays finite
+    y = np.clip(y, float(qmin) - 2.0, float(qmax) + 2.0)
+    lo = np.floor(y)
+    frac = y - lo                                       # exact
+    T = np.floor(frac * 4294967296.0).astype(np.uint64)
+    R = draws(flat.size, seed)
+    r = lo.astype(np.int64) + (R < T).astype(np.int64)
+    if relu:
+        r = np.maximum(r, 0)
+    sat_pos = int((r > qmax).sum())
+    sat_neg = int((r < qmin).sum())
+    q = np.clip(r, qmin, qmax)
+    zeros = int((q == 0).sum())
+    return q.astype(np.int16).reshape(x.shape), (zeros, sat_pos, sat_neg)

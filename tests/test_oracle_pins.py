@@ -395,3 +395,116 @@ def test_network_driver_lenet_shapes_and_formats():
     rec2 = orc.run_network(params, x, (16, 15), 16, fixed_formats=fixed)
     for a, b in zip(rec, rec2):
         assert np.array_equal(a["y"], b["y"])
+
+
+# ---------------------------------------------------------------- thresholded bit allocation (Sec. 2.3)
+def test_bit_allocation_handworked():
+    from oracle import bit_allocation as ba
+    for row in _read_rows("bit_allocation_handworked.txt"):
+        if row[0] == "bits":
+            assert int(ba.integer_bits_needed(np.array([float(row[1])]))[0]) == int(row[2]), row
+        else:
+            n, thr = int(row[1]), float(row[2])
+            hist = [int(v) for v in row[3:3 + ba.HIST_BINS]]
+            assert ba.choose_int_bits(hist, n, thr) == int(row[3 + ba.HIST_BINS]), row
+
+
+def test_bit_histogram_against_exact_integer_definition():
+    """b(x) = smallest m >= 0 with |x| < 2^m, checked with exact rationals; the histogram is its
+    count; threshold 0 reproduces the max-based rule of the range measurement."""
+    from oracle import bit_allocation as ba
+    rng = np.random.default_rng(0)
+    x = (rng.standard_normal(4000) * np.exp(rng.uniform(-3, 9, 4000))).astype(np.float32)
+    x[:8] = [0.0, -0.0, 1.0, -1.0, 2.0 ** 15, -(2.0 ** 16), 65535.9, 1e30]
+    want = []
+    for v in x.tolist():
+        fv, m = abs(Fraction(v)), 0
+        while fv >= Fraction(2) ** m:
+            m += 1
+        want.append(m)
+    got = ba.integer_bits_needed(x)
+    assert got.tolist() == want
+    hist = ba.bit_histogram(x)
+    assert int(hist.sum()) == x.size
+    for b in range(ba.HIST_BINS - 1):
+        assert int(hist[b]) == sum(1 for m in want if m == b)
+    assert int(hist[-1]) == sum(1 for m in want if m >= ba.HIST_BINS - 1)
+    for n in (4, 8, 16):
+        assert ba.choose_int_bits(hist, n, 0.0) == orc.measure_range(x, n)[1]
+    # specials: NaN skipped, Inf in the top bin
+    h2 = ba.bit_histogram(np.array([np.nan, np.inf, -np.inf, 0.5], dtype=np.float32))
+    assert int(h2.sum()) == 3 and int(h2[-1]) == 2 and int(h2[0]) == 1
+
+
+def test_bit_allocation_is_monotone_and_bounds_the_loss():
+    from oracle import bit_allocation as ba
+    rng = np.random.default_rng(1)
+    x = (rng.standard_normal(20000) * 40).astype(np.float32)
+    hist = ba.bit_histogram(x)
+    prev = None
+    for thr in (0.0, 1e-4, 1e-3, 1e-2, 0.05, 0.3, 1.0):
+        m = ba.choose_int_bits(hist, 16, thr)
+        lost = int((ba.integer_bits_needed(x) > m).sum())
+        assert lost <= thr * x.size                      # the accepted loss is within the threshold
+        if m > 0:                                        # and one bit fewer would exceed it
+            assert int((ba.integer_bits_needed(x) > m - 1).sum()) > thr * x.size
+        assert prev is None or m <= prev                 # a larger threshold never needs more bits
+        prev = m
+    # the lost values are exactly those the quantizer saturates (up to the half-LSB edge)
+    m = ba.choose_int_bits(hist, 16, 0.01)
+    _, cnt = orc.quantize(x, 16, 15 - m)
+    assert cnt.sat_pos + cnt.sat_neg >= int((ba.integer_bits_needed(x) > m).sum())
+
+
+def test_twos_complement_width():
+    from oracle import bit_allocation as ba
+    q = np.array([0, -1, 1, -2, 2, 7, 8, -8, -9, 127, 128, -128, -129, 32767, -32768])
+    assert ba.twos_complement_width(q).tolist() == [1, 1, 2, 2, 3, 4, 5, 4, 5, 8, 9, 8, 9, 16, 16]
+
+
+# ---------------------------------------------------------------- stochastic rounding (Sec. 2.4)
+def test_philox_known_answers():
+    from oracle import stochastic as st
+    for row in _read_rows("philox4x32_10_kat.txt"):
+        w = [int(v, 16) for v in row]
+        out = st.philox4x32_10(w[0:4], w[4:6])
+        assert [int(v) for v in out] == w[6:10]
+
+
+def test_philox_draws_layout_and_uniformity():
+    from oracle import stochastic as st
+    r = st.draws(10, seed=(7 << 32) | 5)
+    for i in range(10):                                  # element i uses word i & 3 of block i >> 2
+        blk = st.philox4x32_10((i >> 2, 0, 0, 0), (5, 7))
+        assert int(r[i]) == int(blk[i & 3])
+    big = st.draws(1 << 18, seed=123).astype(np.float64) / 2.0 ** 32
+    assert abs(big.mean() - 0.5) < 4e-3 and abs(big.var() - 1.0 / 12.0) < 2e-3
+    assert not np.array_equal(st.draws(64, 1), st.draws(64, 2))
+
+
+def test_stochastic_rounding_support_and_expectation():
+    """Sec. 2.4: the result is one of the two nearest fixed-point values and its expectation is the
+    unrounded value; values on the grid never move; saturation and specials as the deterministic rule."""
+    from oracle import stochastic as st
+    n, f = 16, 8
+    xs = np.array([0.3, -0.3, 1.0 / 512, -1.0 / 512, 3.14159, -2.71828, 100.123], dtype=np.float32)
+    reps = 20000
+    x = np.tile(xs, reps)
+    q, _ = st.quantize_stochastic(x, n, f, seed=99)
+    q = q.reshape(reps, xs.size).astype(np.float64)
+    y = xs.astype(np.float64) * 2.0 ** f
+    assert np.all((q == np.floor(y)) | (q == np.floor(y) + 1))
+    se = np.sqrt(0.25 / reps)
+    assert np.all(np.abs(q.mean(axis=0) - y) < 5 * se)
+    grid = (np.arange(-300, 300, dtype=np.float32) / 2.0 ** f)
+    qg, _ = st.quantize_stochastic(grid, n, f, seed=1)
+    assert np.array_equal(qg, np.arange(-300, 300).astype(np.int16))
+    sp = np.array([np.nan, np.inf, -np.inf, 1e9, -1e9, 127.999, -0.0], dtype=np.float32)
+    qs, (z, sp_, sn) = st.quantize_stochastic(sp, 16, 8, seed=3)
+    assert qs.tolist()[:5] == [0, 32767, -32768, 32767, -32768] and qs[6] == 0
+    assert qs[5] == 32767 and sp_ in (2, 3) and sn == 2    # 127.999 * 2^8 stays or saturates by one step
+    # the deterministic quantizer's result is always one of the two candidates as well
+    xr = (np.random.default_rng(4).standard_normal(5000) * 3).astype(np.float32)
+    qd, _ = orc.quantize(xr, 16, 10)
+    qs2, _ = st.quantize_stochastic(xr, 16, 10, seed=8)
+    assert np.all(np.abs(qd.astype(np.int64) - qs2.astype(np.int64)) <= 1)
