@@ -56,6 +56,9 @@ enum {
  * away from zero.  Stochastic rounding is not implemented: ADAPTION_ERR_UNSUPPORTED. */
 enum { ADAPTION_ROUND_DETERMINISTIC = 0, ADAPTION_ROUND_STOCHASTIC = 1 };
 
+/* Bins of the bit-occupancy histograms (Sec. 2.2, 2.3): 0..15 bits, and 16 or more. */
+#define ADAPTION_HIST_BINS 17
+
 /* What a layer call does with its pre-activation values v (accumulator + bias, after ReLU if
  * asked): REQUANT rounds them to the output format and stores them; RANGE only records
  * max|v| in stats.max_abs_acc (the per-layer range measurement of Sec. 2.1 / 2.3). */
@@ -112,6 +115,37 @@ ADAPTION_API int adaption_measure_range(const float* d_x, size_t numel, int32_t 
 ADAPTION_API int adaption_quantize(const float* d_x, size_t outer, size_t inner, adaption_qtensor out,
                       const adaption_qfmt* d_fmt, int32_t rounding, adaption_stats* d_stats,
                       void* stream);
+
+/* Sec. 2.4 (rounding_scheme STOCHASTIC).  As adaption_quantize (with the ReLU option of
+ * adaption_lp_act), but x * 2^frac_bits = floor + frac is rounded up with probability
+ * floor(frac * 2^32) / 2^32 and down otherwise, so that the expectation is the unrounded value and
+ * a value already on the grid never moves.  The draw of element i (row-major index over the
+ * outer*inner real elements) is word i & 3 of Philox4x32-10 with counter (i >> 2, 0, 0) and key
+ * `seed`: the result is a pure function of (x, format, seed), whatever the launch shape.
+ * adaption_quantize / adaption_lp_act themselves return ADAPTION_ERR_UNSUPPORTED for
+ * ADAPTION_ROUND_STOCHASTIC because they carry no seed. */
+ADAPTION_API int adaption_quantize_stochastic(const float* d_x, size_t outer, size_t inner, adaption_qtensor out,
+                                 const adaption_qfmt* d_fmt, int32_t relu, uint64_t seed,
+                                 adaption_stats* d_stats, void* stream);
+
+/* Sec. 2.3 (iterative, thresholded allocation of the integer bits).  Adds to d_hist[0..17) (device,
+ * uint64, caller zeroes it before the first tensor of a group) the number of elements of
+ * x[0..numel) that need b integer bits: b = 0 for |x| < 1, else floor(log2 |x|) + 1; bin 16 also
+ * takes everything larger and +-Inf; NaN is skipped. */
+ADAPTION_API int adaption_bit_histogram(const float* d_x, size_t numel, uint64_t* d_hist, void* stream);
+
+/* Sec. 2.2 (how many quantized values fit fewer bits).  Adds to d_hist[w] the number of real
+ * elements of the fixed-point tensor x ([outer][inner], pitch x.c_stride) whose two's complement
+ * width is w: the smallest w >= 1 with -2^(w-1) <= q < 2^(w-1). */
+ADAPTION_API int adaption_width_histogram(adaption_qtensor x, size_t outer, size_t inner, uint64_t* d_hist,
+                             void* stream);
+
+/* Host helper for adaption_bit_histogram.  Starts with all n_bits - 1 non-sign bits in the integer
+ * part and moves bits to the fraction while the values that would be lost (those needing more
+ * integer bits) number at most threshold * total; threshold in [0, 1], 0 gives the format of
+ * adaption_measure_range.  h_hist is a host copy of the 17 bins. */
+ADAPTION_API int adaption_choose_frac_bits_from_hist(const uint64_t* h_hist, int32_t n_bits, double threshold,
+                                        adaption_qfmt* h_out);
 
 /* Sec. 2.1 (LPAct: the activation quantizer, followed by ReLU when relu != 0).  Exactly one
  * of d_x_f32 (fp32 [outer][inner]) and h_x_q (host pointer to the descriptor of a fixed-point

@@ -48,7 +48,10 @@ EXPORTS = [
     "adaption_lp_conv_workspace_bytes", "adaption_lp_conv_fwd", "adaption_lp_ip_workspace_bytes",
     "adaption_lp_ip_fwd", "adaption_lp_ip_fwd_static_ws", "adaption_maxpool2x2", "adaption_choose_frac_bits_from_acc",
     "adaption_probe_i8_peak", "adaption_status_string",
+    "adaption_quantize_stochastic", "adaption_bit_histogram", "adaption_width_histogram",
+    "adaption_choose_frac_bits_from_hist",
 ]
+HIST_BINS = 17
 
 _lib = None
 
@@ -87,6 +90,11 @@ def load(path: str | None = None):
     lib.adaption_maxpool2x2.argtypes = [adaption_qtensor, I32, I32, I32, I32, adaption_qtensor, P]
     lib.adaption_choose_frac_bits_from_acc.argtypes = [I64, I32, I32, C.POINTER(adaption_qfmt)]
     lib.adaption_probe_i8_peak.argtypes = [I32, I32, I32, I32, P, P, P]
+    lib.adaption_quantize_stochastic.argtypes = [P, SZ, SZ, adaption_qtensor, P, I32, C.c_uint64, P, P]
+    lib.adaption_bit_histogram.argtypes = [P, SZ, P, P]
+    lib.adaption_width_histogram.argtypes = [adaption_qtensor, SZ, SZ, P, P]
+    lib.adaption_choose_frac_bits_from_hist.argtypes = [C.POINTER(C.c_uint64), I32, C.c_double,
+                                                        C.POINTER(adaption_qfmt)]
     lib.adaption_status_string.argtypes = [C.c_int]
     lib.adaption_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -193,6 +201,37 @@ def adaption_quantize(x: torch.Tensor, outer: int, inner: int, out: QTensor,
                       d_stats: torch.Tensor | None = None):
     _check(load().adaption_quantize(_ptr(x), outer, inner, out.c_struct(), _ptr(d_fmt), rounding,
                                     _ptr(d_stats), _stream()), "adaption_quantize")
+
+
+def adaption_quantize_stochastic(x: torch.Tensor, outer: int, inner: int, out: QTensor, seed: int,
+                                 relu: bool = False, d_fmt: torch.Tensor | None = None,
+                                 d_stats: torch.Tensor | None = None):
+    _check(load().adaption_quantize_stochastic(_ptr(x), outer, inner, out.c_struct(), _ptr(d_fmt), int(relu),
+                                               seed & 0xFFFFFFFFFFFFFFFF, _ptr(d_stats), _stream()),
+           "adaption_quantize_stochastic")
+
+
+def new_hist(device="cuda") -> torch.Tensor:
+    """Zeroed device histogram of HIST_BINS 64-bit counters (int64 storage, values are counts)."""
+    return torch.zeros(HIST_BINS, dtype=torch.int64, device=device)
+
+
+def adaption_bit_histogram(x: torch.Tensor, d_hist: torch.Tensor):
+    _check(load().adaption_bit_histogram(_ptr(x), x.numel(), _ptr(d_hist), _stream()), "adaption_bit_histogram")
+
+
+def adaption_width_histogram(x: QTensor, d_hist: torch.Tensor):
+    _check(load().adaption_width_histogram(x.c_struct(), x.outer, x.inner, _ptr(d_hist), _stream()),
+           "adaption_width_histogram")
+
+
+def adaption_choose_frac_bits_from_hist(hist, n_bits: int, threshold: float) -> int:
+    """hist: HIST_BINS counts on the host (sequence or CPU tensor)."""
+    arr = (C.c_uint64 * HIST_BINS)(*[int(v) for v in hist])
+    out = adaption_qfmt()
+    _check(load().adaption_choose_frac_bits_from_hist(arr, n_bits, float(threshold), C.byref(out)),
+           "adaption_choose_frac_bits_from_hist")
+    return int(out.frac_bits)
 
 
 def adaption_lp_act(x_f32: torch.Tensor | None, x_q: QTensor | None, outer: int, inner: int, relu: bool,

@@ -19,6 +19,12 @@ int measure_range_impl(const float*, size_t, int32_t, float*, adaption_qfmt*, cu
 int maxpool_impl(const adaption_qtensor&, int32_t, int32_t, int32_t, int32_t, const adaption_qtensor&,
                  cudaStream_t);
 
+int quantize_stochastic_impl(const float*, size_t, size_t, const adaption_qtensor&, const adaption_qfmt*, int32_t,
+                             uint64_t, adaption_stats*, cudaStream_t);
+int bit_histogram_impl(const float*, size_t, uint64_t*, cudaStream_t);
+int width_histogram_impl(const adaption_qtensor&, size_t, size_t, uint64_t*, cudaStream_t);
+int choose_frac_bits_from_hist(const uint64_t*, int32_t, double, adaption_qfmt*);
+
 int probe_i8_peak(int bn, int pair, int iters, int commit_every, unsigned long long* d_cycles, int* d_status,
                   cudaStream_t stream);
 int num_sms();
@@ -145,6 +151,26 @@ int adaption_quantize(const float* d_x, size_t outer, size_t inner, adaption_qte
                       void* stream) {
   return quantize_impl(d_x, outer, inner, out, d_fmt, 0, rounding, d_stats,
                        reinterpret_cast<cudaStream_t>(stream));
+}
+
+int adaption_quantize_stochastic(const float* d_x, size_t outer, size_t inner, adaption_qtensor out,
+                                 const adaption_qfmt* d_fmt, int32_t relu, uint64_t seed,
+                                 adaption_stats* d_stats, void* stream) {
+  return quantize_stochastic_impl(d_x, outer, inner, out, d_fmt, relu, seed, d_stats,
+                                  reinterpret_cast<cudaStream_t>(stream));
+}
+
+int adaption_bit_histogram(const float* d_x, size_t numel, uint64_t* d_hist, void* stream) {
+  return bit_histogram_impl(d_x, numel, d_hist, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int adaption_width_histogram(adaption_qtensor x, size_t outer, size_t inner, uint64_t* d_hist, void* stream) {
+  return width_histogram_impl(x, outer, inner, d_hist, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int adaption_choose_frac_bits_from_hist(const uint64_t* h_hist, int32_t n_bits, double threshold,
+                                        adaption_qfmt* h_out) {
+  return choose_frac_bits_from_hist(h_hist, n_bits, threshold, h_out);
 }
 
 int adaption_lp_act(const float* d_x_f32, const adaption_qtensor* h_x_q, size_t outer, size_t inner,

@@ -79,3 +79,32 @@ def test_workspace_queries(lib):
     assert B.adaption_lp_ip_workspace_bytes(64, 25088, 4096, f16, f16, B.ALGO_DIRECT) == 0
     shp = B.conv_shape(1, 8, 8, 24, 16, 3, 3, 1, 1)   # pitch 48 is not a multiple of 32 -> direct kernel
     assert B.adaption_lp_conv_workspace_bytes(shp, f16, f16, 48) == 0
+
+
+def test_threshold_allocation_host_helper_matches_oracle(lib):
+    """adaption_choose_frac_bits_from_hist is host logic: compare it with the oracle's allocation on
+    the hand-worked rows and on random histograms, thresholds included that sit exactly on a count."""
+    import numpy as np
+
+    from oracle import bit_allocation as ba
+
+    golden = os.path.join(ROOT, "tests", "golden", "bit_allocation_handworked.txt")
+    for line in open(golden):
+        row = line.split()
+        if row and row[0] == "alloc":
+            n, thr = int(row[1]), float(row[2])
+            hist = [int(v) for v in row[3:3 + ba.HIST_BINS]]
+            assert B.adaption_choose_frac_bits_from_hist(hist, n, thr) == n - 1 - int(row[3 + ba.HIST_BINS]), row
+    rng = np.random.default_rng(0)
+    for _ in range(300):
+        hist = (rng.integers(0, 1000, ba.HIST_BINS) * (rng.random(ba.HIST_BINS) < 0.5)).tolist()
+        n = int(rng.integers(1, 17))
+        total = sum(hist)
+        tail = sum(hist[int(rng.integers(0, ba.HIST_BINS)):])
+        for thr in (0.0, 0.01, float(rng.random()) * 0.2, (tail / total) if total else 0.0, 1.0):
+            assert B.adaption_choose_frac_bits_from_hist(hist, n, thr) == ba.choose_frac_bits(hist, n, thr)
+    for bad in (-0.1, 1.5, float("nan")):
+        with pytest.raises(B.AdaptionError):
+            B.adaption_choose_frac_bits_from_hist([0] * ba.HIST_BINS, 16, bad)
+    with pytest.raises(B.AdaptionError):
+        B.adaption_choose_frac_bits_from_hist([0] * ba.HIST_BINS, 17, 0.0)
