@@ -3,7 +3,7 @@
     python -m paper_1711_04713_b200.layer_bench conv --N 8 --H 28 --C 512 --K 512 --R 3 --n-bits 16
     python -m paper_1711_04713_b200.layer_bench ip --B 64 --Kin 25088 --O 4096
     python -m paper_1711_04713_b200.layer_bench quantize --numel 268435456
-    python -m paper_1711_04713_b200.layer_bench range|act|pool ...
+    python -m paper_1711_04713_b200.layer_bench range|act|pool|hist|squantize ...
 
 Prints one JSON line with the CUDA-event time per call and the achieved rate (logical TOPS for
 the layers, algorithmic GB/s for the streaming kernels).  Inputs are seeded synthetic tensors
@@ -115,6 +115,15 @@ def bench_stream(a) -> dict:
         fmt = torch.zeros(2, dtype=torch.int32, device="cuda")
         ms = _time(lambda: B.adaption_measure_range(x, a.n_bits, mx, fmt), a.iters)
         bytes_ = 4 * n
+    elif a.kind == "hist":
+        hist = B.new_hist()
+        ms = _time(lambda: B.adaption_bit_histogram(x, hist), a.iters)
+        bytes_ = 4 * n
+    elif a.kind == "squantize":
+        q = B.QTensor.empty(outer, inner, a.n_bits, a.n_bits - 3)
+        st = B.new_stats()
+        ms = _time(lambda: B.adaption_quantize_stochastic(x, outer, inner, q, 42, False, None, st), a.iters)
+        bytes_ = (4 + plane_b) * n
     elif a.kind in ("quantize", "act"):
         q = B.QTensor.empty(outer, inner, a.n_bits, a.n_bits - 3)
         st = B.new_stats()
@@ -173,7 +182,7 @@ def bench_peak(a) -> dict:
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["conv", "ip", "range", "quantize", "act", "requant", "pool", "peak"])
+    ap.add_argument("kind", choices=["conv", "ip", "range", "quantize", "act", "requant", "pool", "peak", "hist", "squantize"])
     ap.add_argument("--N", type=int, default=8)
     ap.add_argument("--H", type=int, default=28)
     ap.add_argument("--C", type=int, default=512)
