@@ -9,9 +9,9 @@
 //                     NaN is skipped
 //   fixed-point tensor: bin w = two's complement width of q, smallest w >= 1 with
 //                     -2^(w-1) <= q < 2^(w-1)
-// Lanes of a warp that hit the same bin are grouped with a match instruction and one of them adds
-// the group's size to the warp's private histogram in shared memory (no atomics there); a block
-// ends with one global atomic per non-empty bin.  HBM bound: 4 (resp. 2 or 1) bytes per element.
+// Every thread counts into a private histogram in shared memory (bin-major, so that the lanes of a
+// warp touch distinct banks and nothing is atomic); a block ends with one reduction over its
+// threads and one global atomic per non-empty bin.  HBM bound: 4 (resp. 2 or 1) bytes per element.
 #include "common.cuh"
 
 namespace adaption {
@@ -22,13 +22,6 @@ namespace {
 
 constexpr int kBins = ADAPTION_HIST_BINS;
 constexpr int kWarps = 8;
-
-__device__ __forceinline__ void warp_bin_add(uint32_t* hist, int bin, bool valid) {
-  const unsigned active = __ballot_sync(0xffffffffu, valid);
-  if (!valid) return;
-  const unsigned peers = __match_any_sync(active, bin);
-  if ((int)(threadIdx.x & 31) == __ffs(peers) - 1) hist[bin] += (uint32_t)__popc(peers);
-}
 
 __device__ __forceinline__ int bits_of_f32(float x, bool& valid) {
   const uint32_t u = __float_as_uint(x) & 0x7fffffffu;
@@ -43,59 +36,86 @@ __device__ __forceinline__ int width_of_q(int32_t q) {
   return 33 - __clz((int)mag);                               // bit length of mag, plus the sign bit
 }
 
-__device__ __forceinline__ void block_flush(uint32_t (*wh)[kBins], unsigned long long* d_hist) {
-  __syncthreads();
-  if (threadIdx.x < kBins) {
-    unsigned long long s = 0;
+constexpr int kThreadsHist = 32 * kWarps;
+
+// private counters: hist[bin][thread]
+struct PrivateHist {
+  uint32_t c[kBins][kThreadsHist];
+};
+
+__device__ __forceinline__ void hist_clear(PrivateHist& h) {
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) s += wh[w][threadIdx.x];
-    if (s) atomicAdd(d_hist + threadIdx.x, s);
+  for (int b = 0; b < kBins; ++b) h.c[b][threadIdx.x] = 0u;
+}
+
+__device__ __forceinline__ void block_flush(PrivateHist& h, unsigned long long* d_hist) {
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int b = warp; b < kBins; b += kWarps) {
+    unsigned long long s = 0;
+    for (int t = lane; t < kThreadsHist; t += 32) s += h.c[b][t];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0 && s) atomicAdd(d_hist + b, s);
   }
 }
 
-__global__ void __launch_bounds__(32 * kWarps) bit_histogram_kernel(const float* __restrict__ x, size_t numel,
-                                                                    unsigned long long* __restrict__ d_hist) {
-  __shared__ uint32_t wh[kWarps][kBins];
-  for (int i = threadIdx.x; i < kWarps * kBins; i += blockDim.x) (&wh[0][0])[i] = 0u;
-  __syncthreads();
-  uint32_t* mine = wh[threadIdx.x >> 5];
-  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-  // whole warps walk the array together (the match needs converged lanes); the tail is masked
-  const size_t rounds = (numel + nthreads - 1) / nthreads;
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  for (size_t r = 0; r < rounds; ++r, i += nthreads) {
-    bool valid = false;
-    int b = 0;
-    if (i < numel) b = bits_of_f32(__ldcs(x + i), valid);
-    warp_bin_add(mine, b, valid);
-    __syncwarp();
-  }
-  block_flush(wh, d_hist);
+__device__ __forceinline__ void count_f32(PrivateHist& h, float x) {
+  bool valid;
+  const int b = bits_of_f32(x, valid);
+  if (valid) h.c[b][threadIdx.x] += 1u;
 }
 
-__global__ void __launch_bounds__(32 * kWarps) width_histogram_kernel(const int8_t* __restrict__ hi,
-                                                                      const uint8_t* __restrict__ lo, size_t outer,
-                                                                      int64_t inner, int64_t c_stride,
-                                                                      unsigned long long* __restrict__ d_hist) {
-  __shared__ uint32_t wh[kWarps][kBins];
-  for (int i = threadIdx.x; i < kWarps * kBins; i += blockDim.x) (&wh[0][0])[i] = 0u;
-  __syncthreads();
-  uint32_t* mine = wh[threadIdx.x >> 5];
-  const size_t total = outer * (size_t)c_stride;
+// head: elements before the first 16-byte boundary, then n4 float4, then the tail
+__global__ void __launch_bounds__(kThreadsHist) bit_histogram_kernel(const float* __restrict__ x, size_t numel,
+                                                                     size_t head, size_t n4,
+                                                                     unsigned long long* __restrict__ d_hist) {
+  __shared__ PrivateHist h;
+  hist_clear(h);
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-  const size_t rounds = (total + nthreads - 1) / nthreads;
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  for (size_t r = 0; r < rounds; ++r, i += nthreads) {
-    bool valid = false;
-    int w = 0;
-    if (i < total && (int64_t)(i % (size_t)c_stride) < inner) {     // padding channels are not counted
-      valid = true;
-      w = width_of_q(load_q(hi, lo, i));
+  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const float4* __restrict__ x4 = reinterpret_cast<const float4*>(x + head);
+  size_t i = tid;
+  for (; i + nthreads < n4; i += 2 * nthreads) {
+    const float4 a = __ldcs(x4 + i), b = __ldcs(x4 + i + nthreads);
+    count_f32(h, a.x); count_f32(h, a.y); count_f32(h, a.z); count_f32(h, a.w);
+    count_f32(h, b.x); count_f32(h, b.y); count_f32(h, b.z); count_f32(h, b.w);
+  }
+  for (; i < n4; i += nthreads) {
+    const float4 a = __ldcs(x4 + i);
+    count_f32(h, a.x); count_f32(h, a.y); count_f32(h, a.z); count_f32(h, a.w);
+  }
+  const size_t tail0 = head + 4 * n4;
+  for (size_t j = tid; j < head + (numel - tail0); j += nthreads)
+    count_f32(h, x[j < head ? j : tail0 + (j - head)]);
+  block_flush(h, d_hist);
+}
+
+// sixteen stored elements (one 16-byte vector per plane) per thread and step
+__global__ void __launch_bounds__(kThreadsHist) width_histogram_kernel(const uint4* __restrict__ hi,
+                                                                       const uint4* __restrict__ lo, size_t outer,
+                                                                       int64_t inner, int64_t c_stride,
+                                                                       unsigned long long* __restrict__ d_hist) {
+  __shared__ PrivateHist h;
+  hist_clear(h);
+  const int64_t groups_per_row = c_stride / 16;
+  const size_t total = outer * (size_t)groups_per_row;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += nthreads) {
+    const int64_t c0 = (int64_t)(g % (size_t)groups_per_row) * 16;
+    const int nreal = (int)min((int64_t)16, max((int64_t)0, inner - c0));     // padding channels are not counted
+    const uint4 l = __ldcs(lo + g);
+    const uint4 u = hi != nullptr ? __ldcs(hi + g) : make_uint4(0, 0, 0, 0);
+    const uint32_t lw[4] = {l.x, l.y, l.z, l.w}, hw[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const int32_t l8 = (lw[e >> 2] >> (8 * (e & 3))) & 255;
+      const int32_t q = hi != nullptr ? ((int32_t)(int8_t)((hw[e >> 2] >> (8 * (e & 3))) & 255)) * 256 + l8
+                                      : (int32_t)(int8_t)l8;
+      if (e < nreal) h.c[width_of_q(q)][threadIdx.x] += 1u;
     }
-    warp_bin_add(mine, w, valid);
-    __syncwarp();
   }
-  block_flush(wh, d_hist);
+  block_flush(h, d_hist);
 }
 
 int grid_for(size_t items) {
@@ -112,8 +132,11 @@ int bit_histogram_impl(const float* d_x, size_t numel, uint64_t* d_hist, cudaStr
   if ((reinterpret_cast<uintptr_t>(d_x) & 3u) != 0 || (reinterpret_cast<uintptr_t>(d_hist) & 7u) != 0)
     return ADAPTION_ERR_ALIGNMENT;
   if (numel == 0) return ADAPTION_OK;
-  bit_histogram_kernel<<<grid_for(numel), 32 * kWarps, 0, stream>>>(
-      d_x, numel, reinterpret_cast<unsigned long long*>(d_hist));
+  size_t head = ((16 - (reinterpret_cast<uintptr_t>(d_x) & 15u)) & 15u) / 4;
+  if (head > numel) head = numel;
+  const size_t n4 = (numel - head) / 4;
+  bit_histogram_kernel<<<grid_for(n4 / 2 + 64), 32 * kWarps, 0, stream>>>(
+      d_x, numel, head, n4, reinterpret_cast<unsigned long long*>(d_hist));
   return cuda_status(cudaGetLastError(), "bit_histogram_kernel launch");
 }
 
@@ -124,8 +147,8 @@ int width_histogram_impl(const adaption_qtensor& x, size_t outer, size_t inner, 
   if (rc != ADAPTION_OK) return rc;
   if ((reinterpret_cast<uintptr_t>(d_hist) & 7u) != 0) return ADAPTION_ERR_ALIGNMENT;
   if (outer == 0 || inner == 0) return ADAPTION_OK;
-  width_histogram_kernel<<<grid_for(outer * (size_t)x.c_stride), 32 * kWarps, 0, stream>>>(
-      x.fmt.n_bits > 8 ? static_cast<const int8_t*>(x.hi) : nullptr, static_cast<const uint8_t*>(x.lo), outer,
+  width_histogram_kernel<<<grid_for(outer * (size_t)(x.c_stride / 16)), 32 * kWarps, 0, stream>>>(
+      x.fmt.n_bits > 8 ? static_cast<const uint4*>(x.hi) : nullptr, static_cast<const uint4*>(x.lo), outer,
       (int64_t)inner, x.c_stride, reinterpret_cast<unsigned long long*>(d_hist));
   return cuda_status(cudaGetLastError(), "width_histogram_kernel launch");
 }

@@ -190,8 +190,9 @@ __global__ void __launch_bounds__(256) quantize_flat_kernel(const float4* __rest
   if (stats != nullptr) flush_counts_warp(c, stats);
 }
 
-// Rows with channel padding (inner < c_stride) or unaligned input: one thread per group of four
-// stored channels; padding channels receive zeros and are not counted.
+// Rows with channel padding (inner < c_stride) or unaligned input: one thread per group of sixteen
+// stored channels (one 16-byte vector per plane); padding channels receive zeros and are not
+// counted.
 __global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restrict__ x, size_t outer,
                                                             int64_t inner, int64_t c_stride,
                                                             QuantOut out, int32_t frac_bits,
@@ -201,20 +202,38 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restr
   if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
   const float scale = scale_of(frac_bits);
   Counts c;
-  const int64_t groups_per_row = c_stride / 4;
+  const int64_t groups_per_row = c_stride / 16;
   const size_t total = outer * (size_t)groups_per_row;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
   for (size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += nthreads) {
     const size_t row = g / groups_per_row;
-    const int64_t c0 = (int64_t)(g - row * groups_per_row) * 4;
-    int32_t q[4];
+    const int64_t c0 = (int64_t)(g - row * groups_per_row) * 16;
+    const float* __restrict__ src = x + row * (size_t)inner + c0;
+    const int nreal = (int)min((int64_t)16, max((int64_t)0, inner - c0));
+    uint32_t lo[4], hi[4], h16[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const bool real = c0 + u < inner;
-      const float v = real ? __ldg(x + row * inner + c0 + u) : 0.0f;
-      q[u] = quantize_f32(v, scale, relu, qmin, qmax, real, c);
+    for (int w = 0; w < 4; ++w) {
+      int32_t q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool real = 4 * w + u < nreal;
+        const float v = real ? __ldg(src + 4 * w + u) : 0.0f;
+        q[u] = quantize_f32(v, scale, relu, qmin, qmax, real, c);
+      }
+      lo[w] = (uint32_t)(q[0] & 255) | ((uint32_t)(q[1] & 255) << 8) | ((uint32_t)(q[2] & 255) << 16) |
+              ((uint32_t)(q[3] & 255) << 24);
+      hi[w] = (uint32_t)((q[0] >> 8) & 255) | ((uint32_t)((q[1] >> 8) & 255) << 8) |
+              ((uint32_t)((q[2] >> 8) & 255) << 16) | ((uint32_t)((q[3] >> 8) & 255) << 24);
+      h16[2 * w] = (uint32_t)(q[0] & 0xffff) | ((uint32_t)(q[1] & 0xffff) << 16);
+      h16[2 * w + 1] = (uint32_t)(q[2] & 0xffff) | ((uint32_t)(q[3] & 0xffff) << 16);
     }
-    store4(out, g, q[0], q[1], q[2], q[3]);
+    reinterpret_cast<uint4*>(out.lo)[g] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    if (out.planes == 2) reinterpret_cast<uint4*>(out.hi)[g] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    if (out.q16 != nullptr) {
+      uint4* d = reinterpret_cast<uint4*>(out.q16) + 2 * g;
+      d[0] = make_uint4(h16[0], h16[1], h16[2], h16[3]);
+      d[1] = make_uint4(h16[4], h16[5], h16[6], h16[7]);
+    }
   }
   if (stats != nullptr) flush_counts_warp(c, stats);
 }
@@ -444,7 +463,7 @@ int quantize_impl(const float* d_x, size_t outer, size_t inner, const adaption_q
     quantize_flat_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const float4*>(d_x), n4, qo,
                                                    out.fmt.frac_bits, d_fmt, relu, qmin, qmax, d_stats);
   } else {
-    const size_t groups = outer * (size_t)(out.c_stride / 4);
+    const size_t groups = outer * (size_t)(out.c_stride / 16);
     const int grid = stream_grid(groups, 256, 8);
     quantize_rows_kernel<<<grid, 256, 0, stream>>>(d_x, outer, (int64_t)inner, out.c_stride, qo,
                                                    out.fmt.frac_bits, d_fmt, relu, qmin, qmax, d_stats);

@@ -3,8 +3,8 @@
 //
 // For y = x * 2^f = floor(y) + frac the result is floor(y) + 1 with probability T / 2^32,
 // T = floor(frac * 2^32), else floor(y); then ReLU (if asked) and saturation as in the
-// deterministic quantizer (NaN -> 0, +-Inf saturate).  Both parts of y are exact in double
-// precision because x is fp32.  The draw of element i (index in the logical [outer][inner] order)
+// deterministic quantizer (NaN -> 0, +-Inf saturate).  y * 2^32 is exact in double precision
+// because x is fp32, and floor(y * 2^32) = floor(y) * 2^32 + T.  The draw of element i (index in the logical [outer][inner] order)
 // is word i & 3 of Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) with counter
 // (i >> 2 as two 32-bit words, 0, 0) and the caller's 64-bit seed as key; the value moves up iff
 // draw < T.  A counter-based generator makes the result a pure function of (seed, index), so it
@@ -43,13 +43,16 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
 }
 
 struct Out {
-  int8_t* hi;
-  uint8_t* lo;
-  int16_t* q16;
+  uint4* hi;      // sixteen bytes per group of sixteen stored channels
+  uint4* lo;
+  uint4* q16;     // two vectors per group
+  int planes;
 };
 
-// One thread per group of four stored channels of one row (padding channels receive zeros and
-// are neither drawn for nor counted).
+// One thread per group of sixteen stored channels of one row (padding channels receive zeros and
+// are neither drawn for nor counted).  floor(y * 2^32), clamped a little outside the output range
+// (beyond it only saturation matters), is taken with one rounding-down conversion of an exact
+// double product: its high word is floor(y), its low word is T.
 __global__ void __launch_bounds__(256) quantize_stochastic_kernel(const float* __restrict__ x, size_t outer,
                                                                   int64_t inner, int64_t c_stride, Out out,
                                                                   int32_t frac_bits,
@@ -57,48 +60,105 @@ __global__ void __launch_bounds__(256) quantize_stochastic_kernel(const float* _
                                                                   int32_t qmin, int32_t qmax, uint32_t key0,
                                                                   uint32_t key1, adaption_stats* __restrict__ stats) {
   if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
-  const double scale = __longlong_as_double((long long)(1023 + frac_bits) << 52);   // 2^frac_bits
+  const double scale = __longlong_as_double((long long)(1023 + 32 + frac_bits) << 52);   // 2^(frac_bits + 32)
+  const double y_lo = ((double)qmin - 2.0) * 4294967296.0, y_hi = ((double)qmax + 2.0) * 4294967296.0;
   Counts c;
-  const int64_t groups_per_row = c_stride / 4;
+  const int64_t groups_per_row = c_stride / 16;
   const size_t total = outer * (size_t)groups_per_row;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
   for (size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += nthreads) {
     const size_t row = g / groups_per_row;
-    const int64_t c0 = (int64_t)(g - row * groups_per_row) * 4;
+    const int64_t c0 = (int64_t)(g - row * groups_per_row) * 16;
+    const int nreal = (int)min((int64_t)16, max((int64_t)0, inner - c0));
+    const unsigned long long i0 = (unsigned long long)row * (unsigned long long)inner + (unsigned long long)c0;
     unsigned long long have_block = ~0ull;
     Philox4 rnd{};
+    uint32_t lo[4], hi[4], h16[8];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      int32_t q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = 4 * w + u;
+        const bool real = e < nreal;
+        int32_t r = 0;
+        if (real) {
+          const unsigned long long i = i0 + (unsigned long long)e;
+          const unsigned long long blk = i >> 2;
+          if (blk != have_block) {
+            rnd = philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), 0u, 0u, key0, key1);
+            have_block = blk;
+          }
+          const uint32_t sel = (uint32_t)(i & 3ull);
+          const uint32_t draw = sel == 0 ? rnd.w[0] : (sel == 1 ? rnd.w[1] : (sel == 2 ? rnd.w[2] : rnd.w[3]));
+          const float xv = __ldg(x + i);
+          const double y = (xv != xv) ? 0.0 : fmin(fmax((double)xv * scale, y_lo), y_hi);
+          const long long Y = __double2ll_rd(y);
+          r = (int32_t)(Y >> 32) + (draw < (uint32_t)Y ? 1 : 0);
+          if (relu) r = max(r, 0);
+        }
+        const int32_t qq = min(max(r, qmin), qmax);
+        c.sat_pos += (real && r > qmax);
+        c.sat_neg += (real && r < qmin);
+        c.zeros += (real && qq == 0);
+        q[u] = qq;
+      }
+      lo[w] = (uint32_t)(q[0] & 255) | ((uint32_t)(q[1] & 255) << 8) | ((uint32_t)(q[2] & 255) << 16) |
+              ((uint32_t)(q[3] & 255) << 24);
+      hi[w] = (uint32_t)((q[0] >> 8) & 255) | ((uint32_t)((q[1] >> 8) & 255) << 8) |
+              ((uint32_t)((q[2] >> 8) & 255) << 16) | ((uint32_t)((q[3] >> 8) & 255) << 24);
+      h16[2 * w] = (uint32_t)(q[0] & 0xffff) | ((uint32_t)(q[1] & 0xffff) << 16);
+      h16[2 * w + 1] = (uint32_t)(q[2] & 0xffff) | ((uint32_t)(q[3] & 0xffff) << 16);
+    }
+    out.lo[g] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    if (out.planes == 2) out.hi[g] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    if (out.q16 != nullptr) {
+      out.q16[2 * g] = make_uint4(h16[0], h16[1], h16[2], h16[3]);
+      out.q16[2 * g + 1] = make_uint4(h16[4], h16[5], h16[6], h16[7]);
+    }
+  }
+  if (stats != nullptr) flush_counts_warp(c, stats);
+}
+
+// Dense rows (inner == c_stride, 16-byte aligned input): the tensor is one flat array; a thread
+// takes one float4 = the four elements of one generator block, and writes one 4-byte word per plane.
+__global__ void __launch_bounds__(256) quantize_stochastic_flat_kernel(const float4* __restrict__ x, size_t n4,
+                                                                       uint32_t* __restrict__ out_hi,
+                                                                       uint32_t* __restrict__ out_lo,
+                                                                       uint2* __restrict__ out_q16, int32_t frac_bits,
+                                                                       const adaption_qfmt* __restrict__ d_fmt,
+                                                                       int relu, int32_t qmin, int32_t qmax,
+                                                                       uint32_t key0, uint32_t key1,
+                                                                       adaption_stats* __restrict__ stats) {
+  if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
+  const double scale = __longlong_as_double((long long)(1023 + 32 + frac_bits) << 52);   // 2^(frac_bits + 32)
+  const double y_lo = ((double)qmin - 2.0) * 4294967296.0, y_hi = ((double)qmax + 2.0) * 4294967296.0;
+  Counts c;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += nthreads) {
+    const float4 v = __ldcs(x + i);
+    const Philox4 rnd = philox4x32_10((uint32_t)i, (uint32_t)((unsigned long long)i >> 32), 0u, 0u, key0, key1);
+    const float xs[4] = {v.x, v.y, v.z, v.w};
     int32_t q[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const bool real = c0 + u < inner;
-      int32_t r = 0;
-      if (real) {
-        const unsigned long long i = (unsigned long long)row * (unsigned long long)inner + (unsigned long long)(c0 + u);
-        const unsigned long long blk = i >> 2;
-        if (blk != have_block) {
-          rnd = philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), 0u, 0u, key0, key1);
-          have_block = blk;
-        }
-        const uint32_t sel = (uint32_t)(i & 3ull);
-        const uint32_t draw = sel == 0 ? rnd.w[0] : (sel == 1 ? rnd.w[1] : (sel == 2 ? rnd.w[2] : rnd.w[3]));
-        const float xv = __ldg(x + i);
-        double y = (xv != xv) ? 0.0 : (double)xv * scale;
-        // far outside the range only saturation matters: clamp so that the integer parts stay small
-        y = fmin(fmax(y, (double)qmin - 2.0), (double)qmax + 2.0);
-        const double fl = floor(y);
-        const uint32_t T = (uint32_t)(unsigned long long)((y - fl) * 4294967296.0);
-        r = (int32_t)fl + (draw < T ? 1 : 0);
-        if (relu) r = max(r, 0);
-      }
-      const int32_t qq = min(max(r, qmin), qmax);
-      c.sat_pos += (real && r > qmax);
-      c.sat_neg += (real && r < qmin);
-      c.zeros += (real && qq == 0);
-      q[u] = qq;
+      const double y = (xs[u] != xs[u]) ? 0.0 : fmin(fmax((double)xs[u] * scale, y_lo), y_hi);
+      const long long Y = __double2ll_rd(y);
+      int32_t r = (int32_t)(Y >> 32) + (rnd.w[u] < (uint32_t)Y ? 1 : 0);
+      if (relu) r = max(r, 0);
+      q[u] = min(max(r, qmin), qmax);
+      c.sat_pos += (r > qmax);
+      c.sat_neg += (r < qmin);
+      c.zeros += (q[u] == 0);
     }
-    const size_t e0 = g * 4;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) store_q(out.hi, out.lo, out.q16, e0 + u, q[u]);
+    out_lo[i] = (uint32_t)(q[0] & 255) | ((uint32_t)(q[1] & 255) << 8) | ((uint32_t)(q[2] & 255) << 16) |
+                ((uint32_t)(q[3] & 255) << 24);
+    if (out_hi != nullptr)
+      out_hi[i] = (uint32_t)((q[0] >> 8) & 255) | ((uint32_t)((q[1] >> 8) & 255) << 8) |
+                  ((uint32_t)((q[2] >> 8) & 255) << 16) | ((uint32_t)((q[3] >> 8) & 255) << 24);
+    if (out_q16 != nullptr)
+      out_q16[i] = make_uint2((uint32_t)(q[0] & 0xffff) | ((uint32_t)(q[1] & 0xffff) << 16),
+                              (uint32_t)(q[2] & 0xffff) | ((uint32_t)(q[3] & 0xffff) << 16));
   }
   if (stats != nullptr) flush_counts_warp(c, stats);
 }
@@ -115,13 +175,22 @@ int quantize_stochastic_impl(const float* d_x, size_t outer, size_t inner, const
   if ((reinterpret_cast<uintptr_t>(d_x) & 3u) != 0) return ADAPTION_ERR_ALIGNMENT;
   const int32_t qmin = -(1 << (out.fmt.n_bits - 1)), qmax = (1 << (out.fmt.n_bits - 1)) - 1;
   Out o;
-  o.hi = out.fmt.n_bits > 8 ? static_cast<int8_t*>(out.hi) : nullptr;
-  o.lo = static_cast<uint8_t*>(out.lo);
-  o.q16 = out.q16;
-  const size_t groups = outer * (size_t)(out.c_stride / 4);
+  o.planes = out.fmt.n_bits > 8 ? 2 : 1;
+  o.hi = o.planes == 2 ? static_cast<uint4*>(out.hi) : nullptr;
+  o.lo = static_cast<uint4*>(out.lo);
+  o.q16 = reinterpret_cast<uint4*>(out.q16);
+  const bool flat = (int64_t)inner == out.c_stride && aligned16(d_x);
+  const size_t groups = flat ? outer * inner / 4 : outer * (size_t)(out.c_stride / 16);
   size_t want = (groups + 255) / 256;
   const size_t cap = (size_t)num_sms() * 8;
   const int grid = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+  if (flat) {
+    quantize_stochastic_flat_kernel<<<grid, 256, 0, stream>>>(
+        reinterpret_cast<const float4*>(d_x), groups, reinterpret_cast<uint32_t*>(o.hi),
+        reinterpret_cast<uint32_t*>(o.lo), reinterpret_cast<uint2*>(o.q16), out.fmt.frac_bits, d_fmt, relu ? 1 : 0,
+        qmin, qmax, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), d_stats);
+    return cuda_status(cudaGetLastError(), "quantize_stochastic_flat_kernel launch");
+  }
   quantize_stochastic_kernel<<<grid, 256, 0, stream>>>(d_x, outer, (int64_t)inner, out.c_stride, o,
                                                         out.fmt.frac_bits, d_fmt, relu ? 1 : 0, qmin, qmax,
                                                         (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), d_stats);

@@ -229,6 +229,18 @@ class LPNetwork:
         self.calibrated = True
         return rec
 
+    def set_formats(self, x_frac_bits: int, layer_frac_bits: list[int]):
+        """Fix the decimal points without a calibration run (formats chosen elsewhere, e.g. on another
+        batch): ``x_frac_bits`` for the network input, one entry per conv / inner-product layer for
+        its output.  Weight formats still come from max|w| on the device."""
+        self.quantize_params(measure=True)
+        self.xq.frac_bits = x_frac_bits
+        it = iter(layer_frac_bits)
+        for L in self.layers:
+            if L.type in ("conv", "ip"):
+                L.y.frac_bits = int(next(it))
+        self.calibrated = True
+
     # ------------------------------------------------------------------ inference
     def forward(self, x_f32: torch.Tensor, requantize_params: bool = True, measure_input: bool = True):
         """One forward pass with the calibrated formats; enqueues work only (no host sync).

@@ -130,3 +130,88 @@ def test_vgg16_conv3_2_batch32_sampled():
 def test_vgg16_conv4_1_precision_sweep_sampled():
     for n_bits, seed in [(4, 0), (8, 1), (12, 2), (16, 3)]:
         _sampled_conv_check(16, 28, 256, 512, n_bits, seed, samples=300)
+
+
+@pytest.mark.parametrize("n_bits,batch", [(16, 64), (8, 128)])
+def test_vgg16_full_batch_in_the_benchmark_configuration(n_bits, batch):
+    """The whole VGG16 stack at the benchmark's batch size and launch configuration (same network
+    object, same forward call).  The oracle runs the first two images of the batch, with decimal
+    points it chose itself on those two images; the GPU gets these formats and must reproduce every
+    layer's output for the two images bit for bit (images are independent).  Counters and padding are
+    checked on the full batch through properties that hold at any size."""
+    specs = wl.vgg16_specs()
+    params = wl.make_params(specs, seed=0)
+    x = wl.vgg16_input(batch, seed=0)
+    sub = 2
+    rec = orc.run_network(params, x[:sub], None, n_bits)
+    net = LPNetwork(params, batch, (224, 224), 3, n_bits)
+    xd = dev(x.reshape(-1, 3))
+    net.set_formats(rec[0]["frac_bits"], [r["frac_bits"] for r in rec[1:] if r["type"] in ("conv", "ip")])
+    net.zero_stats()
+    out, _ = net.forward(xd)
+    torch.cuda.synchronize()
+    got_in = from_qtensor(net.xq)
+    assert np.array_equal(got_in[:sub * 224 * 224].reshape(rec[0]["y"].shape), rec[0]["y"])
+    for L, r in zip(net.layers, rec[1:]):
+        full = from_qtensor(L.y)
+        rows = full.shape[0] // batch * sub
+        assert np.array_equal(full[:rows].reshape(r["y"].shape), r["y"]), L.name
+        assert L.y.padding_is_zero(), L.name
+        if r["type"] in ("conv", "ip"):
+            assert L.w.frac_bits == r["w_frac_bits"], L.name
+            st = B.read_stats(L.stats)
+            assert int(st.status) == 0
+            assert int(st.zeros) == int((full == 0).sum()), L.name
+            qmax, qmin = (1 << (n_bits - 1)) - 1, -(1 << (n_bits - 1))
+            assert int(st.sat_pos) <= int((full == qmax).sum()) and int(st.sat_neg) <= int((full == qmin).sum())
+            if L.relu:
+                assert int(full.min()) >= 0 and int(st.sat_neg) == 0
+        del full
+
+
+@pytest.mark.parametrize("n_bits,seed", [(4, 0), (8, 1), (12, 2), (16, 3)])
+def test_fc6_batch256_precision_sweep(n_bits, seed):
+    """The inner-product half of the precision sweep at full size: 25088 -> 4096 at batch 256,
+    ReLU'd N(0,1) inputs, He-normal weights, formats from range measurement; every output compared."""
+    Bsz, K, O = 256, 25088, 4096
+    x = wl.relu_normal((Bsz, K), seed)
+    w = wl.he_ip_weight(O, K, seed + 1)
+    b = wl.bias(O, seed + 2)
+    fx = orc.measure_range(x, n_bits)[2]
+    xq, _ = orc.quantize(x, n_bits, fx)
+    wq, fw = orc.quantize_param(w, n_bits)
+    bq, _ = orc.quantize(b, n_bits, fw)
+    acc = orc.ip_acc(xq, wq)
+    F = fx + fw
+    A = orc.epilogue_range(acc, bq, fw, F, True)
+    f_out = n_bits - 1 - orc.int_bits_from_acc(A, F, n_bits)
+    want, cnt = orc.epilogue(acc, bq, fw, F, True, n_bits, f_out)
+
+    # the GPU measures the same formats itself
+    mx = torch.zeros(1, dtype=torch.float32, device="cuda")
+    fmt = torch.zeros(2, dtype=torch.int32, device="cuda")
+    xd, wd = dev(x), dev(w)
+    B.adaption_measure_range(xd, n_bits, mx, fmt)
+    assert int(fmt.cpu()[1]) == fx
+    xg = B.QTensor.empty(Bsz, K, n_bits, fx, K)
+    B.adaption_quantize(xd, Bsz, K, xg)
+    mx.zero_()
+    B.adaption_measure_range(wd, n_bits, mx, fmt)
+    assert int(fmt.cpu()[1]) == fw
+    wg = B.QTensor.empty(O, K, n_bits, fw, K)
+    B.adaption_quantize(wd, O, K, wg)
+    bg = B.QTensor.empty(1, O, n_bits, fw, None, with_q16=True)
+    B.adaption_quantize(dev(b), 1, O, bg)
+    need = B.adaption_lp_ip_workspace_bytes(Bsz, K, O, xg.fmt(), wg.fmt(), B.ALGO_AUTO)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+    st = B.new_stats()
+    B.adaption_lp_ip_fwd(Bsz, K, O, xg, wg, bg.q16, fw, True, B.MODE_RANGE, B.ALGO_AUTO, None, st, ws)
+    assert int(B.read_stats(st).max_abs_acc) == A
+    assert B.adaption_choose_frac_bits_from_acc(A, F, n_bits) == f_out
+    y = B.QTensor.empty(Bsz, O, n_bits, f_out, O)
+    st = B.new_stats()
+    B.adaption_lp_ip_fwd(Bsz, K, O, xg, wg, bg.q16, fw, True, B.MODE_REQUANT, B.ALGO_AUTO, y, st, ws)
+    s = B.read_stats(st)
+    assert s.status == 0
+    assert np.array_equal(from_qtensor(y), want)
+    assert (int(s.zeros), int(s.sat_pos), int(s.sat_neg)) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
