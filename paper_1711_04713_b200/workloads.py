@@ -59,6 +59,38 @@ def vgg16_specs() -> list[LayerSpec]:
     return specs
 
 
+# Giga1Net (paper, "New Benchmark Networks", Table 1): (Cin, Cout, kernel, input H=W, pool after, pad).
+# The table lists no paddings; these are the ones that reproduce its input sizes (112 -> 7x7 ->
+# pool gives the listed 54 only with pad 1; the 18x18 maps are kept through the 3x3 layers by pad 1)
+# and its cost of about 1 GOp per frame (567 MMAC with the first inner product fed by 9 x 9 x 128).
+GIGA1NET_CONV = [
+    (3, 16, 1, 224, True, 0), (16, 16, 7, 112, True, 1), (16, 32, 7, 54, True, 0),
+    (32, 64, 5, 24, False, 1), (64, 64, 5, 22, False, 1), (64, 64, 5, 20, False, 1),
+    (64, 128, 3, 18, False, 1), (128, 128, 3, 18, False, 1), (128, 128, 3, 18, False, 1),
+    (128, 128, 3, 18, False, 1), (128, 128, 3, 18, True, 1),
+]
+GIGA1NET_FC = [("fc12", 9 * 9 * 128, 4096, True), ("fc13", 4096, 1000, False)]
+
+
+def giga1net_specs() -> list[LayerSpec]:
+    specs: list[LayerSpec] = []
+    for i, (cin, cout, k, _, pool, pad) in enumerate(GIGA1NET_CONV, start=1):
+        specs.append(LayerSpec("conv", f"conv{i}", cin, cout, k, pad, 1, True))
+        if pool:
+            specs.append(LayerSpec("pool", f"pool{i}"))
+    for name, k, o, relu in GIGA1NET_FC:
+        specs.append(LayerSpec("ip", name, k, o, relu=relu))
+    return specs
+
+
+def giga1net_macs_per_image() -> int:
+    macs = 0
+    for cin, cout, k, h, _, pad in GIGA1NET_CONV:
+        oh = h + 2 * pad - k + 1
+        macs += oh * oh * cout * k * k * cin
+    return macs + sum(k * o for _, k, o, _ in GIGA1NET_FC)
+
+
 def lenet_specs() -> list[LayerSpec]:
     return [
         LayerSpec("conv", "conv1", 1, 20, 5, 0, 1, True), LayerSpec("pool", "pool1"),

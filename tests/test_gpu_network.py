@@ -76,6 +76,16 @@ def test_small_vgg_like_stack_tensor_path():
     _compare_stack(params, x, None, 16, (32, 32), 3, B.ALGO_AUTO)
 
 
+def test_giga1net_stack():
+    """Giga1Net (paper Table 1): kernels of 1, 7, 5 and 3, 3 to 128 channels, four pools, two inner
+    products; every tensor, decimal point and counter against the oracle on a small batch."""
+    specs = wl.giga1net_specs()
+    assert abs(wl.giga1net_macs_per_image() * 2 / 1e9 - 1.0) < 0.2      # "1 GOp/frame"
+    params = wl.make_params(specs, seed=5)
+    x = wl.vgg16_input(3, seed=5)
+    _compare_stack(params, x, None, 16, (224, 224), 3, B.ALGO_AUTO)
+
+
 def _sampled_conv_check(N, H, Cin, K, n_bits, seed, samples=1500):
     rng = np.random.default_rng(seed)
     x = wl.relu_normal((N, H, H, Cin), seed)
