@@ -147,6 +147,13 @@ ADAPTION_API int adaption_width_histogram(adaption_qtensor x, size_t outer, size
 ADAPTION_API int adaption_choose_frac_bits_from_hist(const uint64_t* h_hist, int32_t n_bits, double threshold,
                                         adaption_qfmt* h_out);
 
+/* The same allocation for a tensor that is already stored with frac_bits fractional bits (e.g. a
+ * layer output quantized with the max-based format, so that nothing was clipped), from the
+ * histogram of adaption_width_histogram: a value keeps its bits with m integer bits iff its width
+ * is at most m + frac_bits + 1. */
+ADAPTION_API int adaption_choose_frac_bits_from_widths(const uint64_t* h_hist, int32_t frac_bits, int32_t n_bits,
+                                          double threshold, adaption_qfmt* h_out);
+
 /* Sec. 2.1 (LPAct: the activation quantizer, followed by ReLU when relu != 0).  Exactly one
  * of d_x_f32 (fp32 [outer][inner]) and h_x_q (host pointer to the descriptor of a fixed-point
  * tensor, whose format is converted) is given.  Otherwise as adaption_quantize. */

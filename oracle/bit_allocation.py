@@ -72,12 +72,32 @@ def choose_frac_bits(hist, n_bits: int, threshold: float) -> int:
     return n_bits - 1 - choose_int_bits(hist, n_bits, threshold)
 
 
+def width_histogram(q) -> np.ndarray:
+    """Histogram over w = 1..16 of the two's complement widths of a quantized tensor (bin 0 stays 0)."""
+    return np.bincount(twos_complement_width(q), minlength=HIST_BINS).astype(np.uint64)
+
+
+def choose_int_bits_from_widths(width_hist, frac_bits: int, n_bits: int, threshold: float) -> int:
+    """Reading B3 for a tensor already stored with ``frac_bits`` fractional bits (the layer output
+    quantized with the max-based format, so that nothing was clipped): q keeps its value with m
+    integer bits iff its width is at most m + frac_bits + 1.  Same order as the paper: start with
+    all n - 1 non-sign bits in the integer part, give bits away while the loss stays within the
+    threshold."""
+    hist = [int(v) for v in width_hist]
+    total = sum(hist)
+
+    def lost(m: int) -> int:
+        return sum(hist[w] for w in range(len(hist)) if w > m + frac_bits + 1)
+
+    m = n_bits - 1
+    while m > 0 and lost(m - 1) <= threshold * total:
+        m -= 1
+    return m
+
+
 def twos_complement_width(q) -> np.ndarray:
     """Reading B4: smallest w >= 1 with -2^(w-1) <= q < 2^(w-1)."""
     q = np.asarray(q, dtype=np.int64).reshape(-1)
-    out = np.empty(q.shape, dtype=np.int64)
-    for i, v in enumerate(q):
-        v = int(v)
-        mag = v if v >= 0 else -v - 1          # q >= 0: q < 2^(w-1);  q < 0: -q - 1 < 2^(w-1)
-        out[i] = mag.bit_length() + 1
-    return out
+    mag = np.where(q >= 0, q, -q - 1)          # q >= 0: q < 2^(w-1);  q < 0: -q - 1 < 2^(w-1)
+    _, e = np.frexp(mag.astype(np.float64))    # exact below 2^53: mag in [2^(e-1), 2^e), e = 0 for 0
+    return e.astype(np.int64) + 1              # bit length of mag, plus the sign bit

@@ -269,8 +269,20 @@ def quantize_param(w, n_bits: int):
     return q, f
 
 
-def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None):
+def _thresholded_fmt(t, n_bits: int, threshold: float) -> int:
+    """Fractional bits of an fp32 tensor by the thresholded allocation of Sec. 2.3."""
+    from . import bit_allocation as ba
+    return ba.choose_frac_bits(ba.bit_histogram(t), n_bits, threshold)
+
+
+def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None, threshold: float = 0.0):
     """Forward pass of a stack of LP layers on a batch.
+
+    ``threshold`` > 0 (only without ``fixed_formats``): decimal points by the thresholded allocation
+    of Sec. 2.3 instead of the maximum: fp32 tensors (input, weights) from their bit-occupancy
+    histogram; a layer output is first quantized with the max-based format (nothing clipped), the
+    widths of those integers decide how many integer bits may go, and the layer is requantized
+    from its exact accumulators with the final format.
 
     ``layers``: list of dicts, each one of
         {"type": "conv", "w": fp32 [K][R][S][C], "b": fp32 [K], "pad": p, "stride": s, "relu": bool}
@@ -282,7 +294,7 @@ def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None):
     """
     records = []
     if x_fmt is None:
-        _, _, fx = measure_range(x, n_bits)
+        fx = _thresholded_fmt(x, n_bits, threshold) if threshold > 0 else measure_range(x, n_bits)[2]
         nx = n_bits
     else:
         nx, fx = x_fmt
@@ -294,7 +306,11 @@ def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None):
             a = maxpool2x2(a)
             records.append({"type": "pool", "y": a, "n_bits": nx, "frac_bits": fx})
             continue
-        wq, fw = quantize_param(L["w"], n_bits)
+        if threshold > 0 and fixed_formats is None:
+            fw = _thresholded_fmt(L["w"], n_bits, threshold)
+            wq, _ = quantize(L["w"], n_bits, fw)
+        else:
+            wq, fw = quantize_param(L["w"], n_bits)
         bq, _ = quantize(L["b"], n_bits, fw)
         if L["type"] == "conv":
             p, s = L["pad"], L["stride"]
@@ -303,6 +319,11 @@ def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None):
             acc = ip_acc(a.reshape(a.shape[0], -1), wq)
         f_out = None if fixed_formats is None else fixed_formats[li]
         res = lp_layer(acc, fx, fw, bq, fw, L["relu"], n_bits, f_out)
+        if threshold > 0 and fixed_formats is None:
+            from . import bit_allocation as ba
+            m = ba.choose_int_bits_from_widths(ba.width_histogram(res.y), res.frac_bits, n_bits, threshold)
+            if n_bits - 1 - m != res.frac_bits:
+                res = lp_layer(acc, fx, fw, bq, fw, L["relu"], n_bits, n_bits - 1 - m)
         records.append({"type": L["type"], "y": res.y, "n_bits": n_bits, "frac_bits": res.frac_bits,
                         "w_frac_bits": fw, "wq": wq, "bq": bq, "counters": res.counters,
                         "max_abs_acc": res.max_abs_acc, "acc_frac_bits": res.acc_frac_bits})

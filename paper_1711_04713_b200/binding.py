@@ -49,7 +49,7 @@ EXPORTS = [
     "adaption_lp_ip_fwd", "adaption_lp_ip_fwd_static_ws", "adaption_maxpool2x2", "adaption_choose_frac_bits_from_acc",
     "adaption_probe_i8_peak", "adaption_status_string",
     "adaption_quantize_stochastic", "adaption_bit_histogram", "adaption_width_histogram",
-    "adaption_choose_frac_bits_from_hist",
+    "adaption_choose_frac_bits_from_hist", "adaption_choose_frac_bits_from_widths",
 ]
 HIST_BINS = 17
 
@@ -95,6 +95,8 @@ def load(path: str | None = None):
     lib.adaption_width_histogram.argtypes = [adaption_qtensor, SZ, SZ, P, P]
     lib.adaption_choose_frac_bits_from_hist.argtypes = [C.POINTER(C.c_uint64), I32, C.c_double,
                                                         C.POINTER(adaption_qfmt)]
+    lib.adaption_choose_frac_bits_from_widths.argtypes = [C.POINTER(C.c_uint64), I32, I32, C.c_double,
+                                                          C.POINTER(adaption_qfmt)]
     lib.adaption_status_string.argtypes = [C.c_int]
     lib.adaption_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -231,6 +233,15 @@ def adaption_choose_frac_bits_from_hist(hist, n_bits: int, threshold: float) -> 
     out = adaption_qfmt()
     _check(load().adaption_choose_frac_bits_from_hist(arr, n_bits, float(threshold), C.byref(out)),
            "adaption_choose_frac_bits_from_hist")
+    return int(out.frac_bits)
+
+
+def adaption_choose_frac_bits_from_widths(hist, frac_bits: int, n_bits: int, threshold: float) -> int:
+    """hist: HIST_BINS width counts on the host of a tensor stored with ``frac_bits`` fractional bits."""
+    arr = (C.c_uint64 * HIST_BINS)(*[int(v) for v in hist])
+    out = adaption_qfmt()
+    _check(load().adaption_choose_frac_bits_from_widths(arr, frac_bits, n_bits, float(threshold), C.byref(out)),
+           "adaption_choose_frac_bits_from_widths")
     return int(out.frac_bits)
 
 

@@ -24,6 +24,7 @@ int quantize_stochastic_impl(const float*, size_t, size_t, const adaption_qtenso
 int bit_histogram_impl(const float*, size_t, uint64_t*, cudaStream_t);
 int width_histogram_impl(const adaption_qtensor&, size_t, size_t, uint64_t*, cudaStream_t);
 int choose_frac_bits_from_hist(const uint64_t*, int32_t, double, adaption_qfmt*);
+int choose_frac_bits_from_widths(const uint64_t*, int32_t, int32_t, double, adaption_qfmt*);
 
 int probe_i8_peak(int bn, int pair, int iters, int commit_every, unsigned long long* d_cycles, int* d_status,
                   cudaStream_t stream);
@@ -171,6 +172,11 @@ int adaption_width_histogram(adaption_qtensor x, size_t outer, size_t inner, uin
 int adaption_choose_frac_bits_from_hist(const uint64_t* h_hist, int32_t n_bits, double threshold,
                                         adaption_qfmt* h_out) {
   return choose_frac_bits_from_hist(h_hist, n_bits, threshold, h_out);
+}
+
+int adaption_choose_frac_bits_from_widths(const uint64_t* h_hist, int32_t frac_bits, int32_t n_bits,
+                                          double threshold, adaption_qfmt* h_out) {
+  return choose_frac_bits_from_widths(h_hist, frac_bits, n_bits, threshold, h_out);
 }
 
 int adaption_lp_act(const float* d_x_f32, const adaption_qtensor* h_x_q, size_t outer, size_t inner,

@@ -174,4 +174,20 @@ int choose_frac_bits_from_hist(const uint64_t* h_hist, int32_t n_bits, double th
   return ADAPTION_OK;
 }
 
+// Host: the same allocation for a tensor already stored with `frac_bits` fractional bits, from the
+// histogram of its two's complement widths: q keeps its value with m integer bits iff its width is
+// at most m + frac_bits + 1.
+int choose_frac_bits_from_widths(const uint64_t* h_hist, int32_t frac_bits, int32_t n_bits, double threshold,
+                                 adaption_qfmt* h_out) {
+  if (h_hist == nullptr || frac_bits < 0 || frac_bits > 15) return ADAPTION_ERR_INVALID_ARG;
+  uint64_t need[kBins];                 // need[b]: values that need b integer bits
+  for (int b = 0; b < kBins; ++b) need[b] = 0;
+  for (int w = 0; w < kBins; ++w) {
+    int b = w - 1 - frac_bits;
+    if (b < 0) b = 0;
+    need[b] += h_hist[w];
+  }
+  return choose_frac_bits_from_hist(need, n_bits, threshold, h_out);
+}
+
 }  // namespace adaption

@@ -39,18 +39,30 @@ __global__ void __launch_bounds__(256) pack_taps_kernel(const PackParams p) {
   const int taps = p.R * p.S;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
-    const int plane = (int)(i / p.rows);
-    const long long m = i - (long long)plane * p.rows;
+    // (there are at most two planes: no division)
+    const int plane = i >= p.rows ? 1 : 0;
+    const long long m = plane ? i - p.rows : i;
     const uint8_t* __restrict__ src = p.src[plane];
     long long base;            // element offset of tap (0, 0), channel 0
     int ih0 = 0, iw0 = 0;
     if (p.is_weight) {
       base = m * (long long)taps * p.c_stride;
     } else {
-      const int ow = (int)(m % p.OW);
-      const long long rest = m / p.OW;
-      const int oh = (int)(rest % p.OH);
-      const long long img = rest / p.OH;
+      // pixel index -> (image, row, column); 32-bit arithmetic whenever the index fits
+      int ow, oh;
+      long long img;
+      if (p.rows <= 0x7fffffffll) {
+        const unsigned mu = (unsigned)m, rest = mu / (unsigned)p.OW;
+        ow = (int)(mu - rest * (unsigned)p.OW);
+        const unsigned im = rest / (unsigned)p.OH;
+        oh = (int)(rest - im * (unsigned)p.OH);
+        img = im;
+      } else {
+        ow = (int)(m % p.OW);
+        const long long rest = m / p.OW;
+        oh = (int)(rest % p.OH);
+        img = rest / p.OH;
+      }
       ih0 = oh * p.stride_h - p.pad_h;
       iw0 = ow * p.stride_w - p.pad_w;
       base = ((img * p.H + ih0) * (long long)p.W + iw0) * p.c_stride;

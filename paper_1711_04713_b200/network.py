@@ -137,13 +137,25 @@ class LPNetwork:
         self.total_macs = sum(L.macs for L in self.layers)
 
     # ------------------------------------------------------------------ parameters
-    def quantize_params(self, measure: bool = True):
+    def _fp32_fmt_by_threshold(self, t: torch.Tensor, threshold: float) -> int:
+        """Fractional bits of an fp32 device tensor by the thresholded allocation (Sec. 2.3)."""
+        hist = B.new_hist(self.device)
+        B.adaption_bit_histogram(t, hist)
+        return B.adaption_choose_frac_bits_from_hist(hist.cpu().tolist(), self.n_bits, threshold)
+
+    def quantize_params(self, measure: bool = True, threshold: float = 0.0):
         """Weights and biases -> fixed point (paper Sec. 2.1: quantized in the forward pass).  With
-        ``measure`` the decimal point of each layer's weights is taken from max|w| on the device."""
+        ``measure`` the decimal point of each layer's weights is taken from max|w| on the device, or,
+        with ``threshold`` > 0, from the thresholded allocation of Sec. 2.3."""
         for L in self.layers:
             if L.type not in ("conv", "ip"):
                 continue
-            if measure:
+            if measure and threshold > 0:
+                L.w.frac_bits = L.b.frac_bits = self._fp32_fmt_by_threshold(L.w_f32, threshold)
+                L.w_fmt_dev.copy_(torch.tensor([self.n_bits, L.w.frac_bits], dtype=torch.int32))
+                B.adaption_quantize(L.w_f32, L.w.outer, L.w.inner, L.w)
+                B.adaption_quantize(L.b_f32, 1, L.K, L.b)
+            elif measure:
                 L.w_max_dev.zero_()
                 B.adaption_measure_range(L.w_f32, self.n_bits, L.w_max_dev, L.w_fmt_dev)
                 B.adaption_quantize(L.w_f32, L.w.outer, L.w.inner, L.w, L.w_fmt_dev)
@@ -189,13 +201,18 @@ class LPNetwork:
         return L.y
 
     # ------------------------------------------------------------------ calibration
-    def calibrate(self, x_f32: torch.Tensor, x_fmt: tuple[int, int] | None = None):
+    def calibrate(self, x_f32: torch.Tensor, x_fmt: tuple[int, int] | None = None, threshold: float = 0.0):
         """Run one batch layer by layer, measuring each layer's range on it and fixing its decimal
-        point (paper Sec. 2.1, 2.3).  Returns the per-layer records (formats, counters, ranges)."""
-        self.quantize_params(measure=True)
+        point (paper Sec. 2.1, 2.3).  Returns the per-layer records (formats, counters, ranges).
+        ``threshold`` > 0: thresholded allocation of the integer bits instead of the maximum (fp32
+        tensors from their bit-occupancy histogram; a layer output is first stored with the
+        max-based format, the widths of those integers decide, then the layer is run again)."""
+        self.quantize_params(measure=True, threshold=threshold)
         rec = []
         self.x_stats.zero_()
-        if x_fmt is None:
+        if x_fmt is None and threshold > 0:
+            self.xq.frac_bits = self._fp32_fmt_by_threshold(x_f32, threshold)
+        elif x_fmt is None:
             self.x_max_dev.zero_()
             B.adaption_measure_range(x_f32, self.n_bits, self.x_max_dev, self.x_fmt_dev)
             self.xq.frac_bits = int(self.x_fmt_dev.cpu()[1])
@@ -219,7 +236,17 @@ class LPNetwork:
             F = a.frac_bits + L.w.frac_bits
             L.y.frac_bits = B.adaption_choose_frac_bits_from_acc(int(st.max_abs_acc), F, self.n_bits)
             L.stats.zero_()
-            a = self._run_layer(L, a, B.MODE_REQUANT)
+            a_in = a
+            a = self._run_layer(L, a_in, B.MODE_REQUANT)
+            if threshold > 0:
+                hist = B.new_hist(self.device)
+                B.adaption_width_histogram(L.y, hist)
+                f = B.adaption_choose_frac_bits_from_widths(hist.cpu().tolist(), L.y.frac_bits, self.n_bits,
+                                                            threshold)
+                if f != L.y.frac_bits:
+                    L.y.frac_bits = f
+                    L.stats.zero_()
+                    a = self._run_layer(L, a_in, B.MODE_REQUANT)
             st2 = B.read_stats(L.stats)
             if st2.status != 0:
                 raise B.AdaptionError(st2.status, f"layer {L.name}")

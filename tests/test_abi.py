@@ -103,6 +103,12 @@ def test_threshold_allocation_host_helper_matches_oracle(lib):
         tail = sum(hist[int(rng.integers(0, ba.HIST_BINS)):])
         for thr in (0.0, 0.01, float(rng.random()) * 0.2, (tail / total) if total else 0.0, 1.0):
             assert B.adaption_choose_frac_bits_from_hist(hist, n, thr) == ba.choose_frac_bits(hist, n, thr)
+    for _ in range(200):
+        hist = [0] + (rng.integers(0, 500, ba.HIST_BINS - 1) * (rng.random(ba.HIST_BINS - 1) < 0.6)).tolist()
+        n, f = int(rng.integers(2, 17)), int(rng.integers(0, 16))
+        for thr in (0.0, 0.01, 0.1):
+            want = n - 1 - ba.choose_int_bits_from_widths(hist, f, n, thr)
+            assert B.adaption_choose_frac_bits_from_widths(hist, f, n, thr) == want
     for bad in (-0.1, 1.5, float("nan")):
         with pytest.raises(B.AdaptionError):
             B.adaption_choose_frac_bits_from_hist([0] * ba.HIST_BINS, 16, bad)

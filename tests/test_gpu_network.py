@@ -13,11 +13,11 @@ from tests.util import dev, from_qtensor
 pytestmark = pytest.mark.gpu
 
 
-def _compare_stack(params, x, x_fmt, n_bits, in_hw, in_c, algo):
-    rec = orc.run_network(params, x, x_fmt, n_bits)
+def _compare_stack(params, x, x_fmt, n_bits, in_hw, in_c, algo, threshold=0.0):
+    rec = orc.run_network(params, x, x_fmt, n_bits, threshold=threshold)
     net = LPNetwork(params, x.shape[0], in_hw, in_c, n_bits, algo=algo)
     xd = dev(x.reshape(-1, in_c))
-    grec = net.calibrate(xd, x_fmt)
+    grec = net.calibrate(xd, x_fmt, threshold=threshold)
     assert len(grec) == len(rec)
     assert grec[0]["frac_bits"] == rec[0]["frac_bits"]
     assert np.array_equal(from_qtensor(net.xq).reshape(rec[0]["y"].shape), rec[0]["y"])
@@ -74,6 +74,27 @@ def test_small_vgg_like_stack_tensor_path():
     params = wl.make_params(specs, seed=3)
     x = wl.vgg16_input(8, seed=3, hw=32)
     _compare_stack(params, x, None, 16, (32, 32), 3, B.ALGO_AUTO)
+
+
+@pytest.mark.parametrize("threshold", [0.002, 0.02])
+def test_stacks_with_thresholded_bit_allocation(threshold):
+    """Sec. 2.3: decimal points by the thresholded allocation instead of the maximum.  Formats differ
+    from the max-based ones (more fractional bits, some values saturate) and every tensor, format
+    and counter still matches the oracle."""
+    params = wl.make_params(wl.lenet_specs(), seed=0)
+    x = wl.lenet_input(8, seed=0)
+    rec = _compare_stack(params, x, None, 16, (28, 28), 1, B.ALGO_AUTO, threshold=threshold)
+    base = orc.run_network(params, x, None, 16)
+    assert all(r["frac_bits"] >= b["frac_bits"] for r, b in zip(rec, base))
+    if threshold >= 0.02:     # large enough to move decimal points on this stack
+        assert any(r["frac_bits"] > b["frac_bits"] for r, b in zip(rec, base))
+        assert sum(r["counters"].sat_pos for r in rec if "counters" in r) > 0
+    specs = [wl.LayerSpec("conv", "c1", 3, 64, 3, 1, 1, True), wl.LayerSpec("conv", "c2", 64, 64, 3, 1, 1, True),
+             wl.LayerSpec("pool", "p1"), wl.LayerSpec("conv", "c3", 64, 128, 3, 1, 1, True),
+             wl.LayerSpec("pool", "p2"), wl.LayerSpec("ip", "f1", 8 * 8 * 128, 256, relu=True),
+             wl.LayerSpec("ip", "f2", 256, 10, relu=False)]
+    _compare_stack(wl.make_params(specs, seed=4), wl.vgg16_input(8, seed=4, hw=32), None, 8, (32, 32), 3,
+                   B.ALGO_AUTO, threshold=threshold)
 
 
 def test_giga1net_stack():
