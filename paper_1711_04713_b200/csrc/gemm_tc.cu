@@ -82,6 +82,7 @@ struct TcParams {
   unsigned long long timeout_ns;
   // epilogue variants chosen on the host
   int fast_relu;              // launch the FAST kernel variant (paired 16-bit epilogue)
+  int epi_groups;             // 1, or 2: the epilogue warps form two groups that take alternate tiles
   int staged;                 // outputs leave through shared memory and bulk-tensor stores
   uint32_t stage_off;         // offset of the staging planes from the ring base
 };
@@ -680,22 +681,23 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void fence_async_shared() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
-// Barrier among the epilogue warps only (barrier 0 belongs to __syncthreads).
-__device__ __forceinline__ void epi_bar_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+// Barriers among the warps of one epilogue group only (barrier 0 belongs to __syncthreads; group g
+// uses barriers 1 + 2g and 2 + 2g).
+__device__ __forceinline__ void epi_bar_sync(int group, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + 2 * group), "r"(threads) : "memory");
 }
 // ... that also returns the conjunction of every thread's predicate
-__device__ __forceinline__ bool epi_bar_all(bool pred) {
+__device__ __forceinline__ bool epi_bar_all(int group, int threads, bool pred) {
   uint32_t r;
   asm volatile(
       "{\n"
       ".reg .pred p, q;\n"
       "setp.ne.b32 p, %1, 0;\n"
-      "bar.red.and.pred q, 2, %2, p;\n"
+      "bar.red.and.pred q, %2, %3, p;\n"
       "selp.u32 %0, 1, 0, q;\n"
       "}\n"
       : "=r"(r)
-      : "r"((uint32_t)pred), "n"(32 * kEpiWarps)
+      : "r"((uint32_t)pred), "r"(2 + 2 * group), "r"(threads)
       : "memory");
   return r != 0;
 }
@@ -717,7 +719,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   __shared__ Ctrl ctrl;
 
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const int warp = threadIdx.x >> 5;
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform for the compiler too
   const int lane = threadIdx.x & 31;
   // PAIR: two CTAs (a cluster of two) share every tile of 256 rows.  Rank 0 is the leader: it owns
   // the "full" and "tmem_empty" barriers that are in use and issues the MMAs for both.
@@ -735,7 +737,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     for (int b = 0; b < p.acc_bufs; ++b) {
       mbar_init(smem_u32(&ctrl.tmem_full[b]), (uint32_t)p.mma_warps);
       mbar_init(smem_u32(&ctrl.first_issued[b]), 1);
-      mbar_init(smem_u32(&ctrl.tmem_empty[b]), PAIR ? 2 * kEpiWarps : kEpiWarps);
+      mbar_init(smem_u32(&ctrl.tmem_empty[b]), (uint32_t)((PAIR ? 2 : 1) * (kEpiWarps / p.epi_groups)));
     }
     for (int w = 0; w < kMmaWarps; ++w) mbar_init(smem_u32(&ctrl.drain[w]), 1);
     mbar_init(smem_u32(&ctrl.b_ready), 1);
@@ -1019,21 +1021,29 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;          // TMEM lanes 32*quarter .. 32*quarter+31
-    const int ew = warp - kFirstEpiWarp;
+    // With two accumulator sets and narrow tiles the warps form two groups that take alternate
+    // tiles (and accumulator sets), so that one group's TMEM loads overlap the other's arithmetic;
+    // each group has its own barriers, constants and staging planes.
+    const int groups = p.epi_groups;
+    const int gwarps = kEpiWarps / groups, gthreads = 32 * gwarps;
+    const int group = (warp - kFirstEpiWarp) / gwarps;
+    const int ew = (warp - kFirstEpiWarp) - group * gwarps;      // warp index within its group
     // the warps of a lane quarter split the columns of the tile
-    const int cols_per_warp = max(16, p.BN / (kEpiWarps / 4));
+    const int cols_per_warp = max(16, p.BN / (gwarps / 4));
     const int col_begin = min(p.BN, (ew >> 2) * cols_per_warp);
     const int col_end = min(p.BN, col_begin + cols_per_warp);
     const int row = quarter * 32 + lane;   // row of the tile (and of this CTA's staging planes)
-    const uint32_t stage_lo = ring + p.stage_off;
+    const int planes_bytes = kBM * p.BN * p.rq.out_planes;
+    const uint32_t stage_lo = ring + p.stage_off + (uint32_t)(group * planes_bytes);
     const uint32_t stage_hi = stage_lo + (uint32_t)(kBM * p.BN);
+    long long* colconst = ctrl.colconst + group * (kMaxBN / 2);
     const bool store_leader = ew == 0 && lane == 0;
-    uint32_t tile_iter = 0;
+    uint32_t tile_iter = (uint32_t)group;
     Counts cnt;
     long long vmax = 0;
     bool ok = true;
     int const_n0 = -1;          // first column of the tile whose constants are staged
-    for (int t = worker; t < p.total_tiles; t += workers, ++tile_iter) {
+    for (int t = worker + group * workers; t < p.total_tiles; t += groups * workers, tile_iter += (uint32_t)groups) {
       const TileCoord tc = decode_tile(t, p);
       const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
       const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
@@ -1041,15 +1051,15 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       // writes from its readers): bias aligned to the accumulator, plus the rounding half on the
       // fast path.  Kept when the tile covers the same columns as the previous one.
       if (tc.n0 != const_n0) {
-        for (int c = (int)threadIdx.x - 32 * kFirstEpiWarp; c < p.BN; c += 32 * kEpiWarps) {
+        for (int c = 32 * ew + lane; c < p.BN; c += gthreads) {
           const int n = tc.n0 + c;
           long long b = 0;
           if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
           if (FAST) {
             const long long C = b + (1ll << (p.rq.shift - 1));
-            reinterpret_cast<int2*>(ctrl.colconst)[c] = make_int2((int)(C & 0xffff), (int)(C >> 16));
+            reinterpret_cast<int2*>(colconst)[c] = make_int2((int)(C & 0xffff), (int)(C >> 16));
           } else {
-            ctrl.colconst[c] = b;
+            colconst[c] = b;
           }
         }
         const_n0 = tc.n0;
@@ -1060,7 +1070,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       bool w = wait_bar(smem_u32(&ctrl.tmem_full[buf]), bph, &ctrl, p);
       // one decision for all epilogue warps (they meet at barriers below), which also publishes the
       // constants and the free staging planes
-      w = epi_bar_all(w);
+      w = epi_bar_all(group, gthreads, w);
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 1);
       if (!w) { ok = false; break; }
       tc_fence_after();
@@ -1094,7 +1104,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         }
         if (!have) break;
         const int col = tc.n0 + c0;
-        const long long* bcol = ctrl.colconst + c0;
+        const long long* bcol = colconst + c0;
         if (!FAST && !storing) {
           partial_or_range8<NACC>(xa, bcol, p, row_ok, m, col, vmax);
           partial_or_range8<NACC>(xb, bcol + 8, p, row_ok, m, col + 8, vmax);
@@ -1123,7 +1133,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       // the channel pitch are clipped by the tensor map); the barrier also ends this tile's reads
       // of the per-column constants
       if (p.staged) fence_async_shared();
-      epi_bar_sync();
+      epi_bar_sync(group, gthreads);
       if (p.staged && store_leader) {
         const int m_first = tc.m0 + (int)rank * kBM;
         tma_store_2d(&map_y_lo, stage_lo, tc.n0, m_first);
@@ -1200,6 +1210,7 @@ struct TcConfig {
   uint32_t kb_bytes = 0;
   bool pair = false;           // two CTAs per 256-row tile (cta_group::2)
   int tile_m = kBM;
+  int epi_groups = 1;
   bool staged = false;         // outputs staged in shared memory and written by bulk-tensor stores
   uint32_t stage_out_bytes = 0, stage_off = 0;
   size_t smem_bytes = 0;
@@ -1299,7 +1310,11 @@ TcConfig make_config(const GemmProblem& g) {
   const int out_planes = g.y.fmt.n_bits > 8 ? 2 : 1;
   c.staged = g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.y.q16 == nullptr && g.y.lo != nullptr &&
              g.y.c_stride >= c.BN && g.y.c_stride % 16 == 0 && env_int("ADAPTION_TC_STAGED", 1) != 0;
-  c.stage_out_bytes = c.staged ? (uint32_t)(kBM * c.BN * out_planes) : 0u;
+  // two epilogue groups when two tiles can be in flight in TMEM and their constants fit the halves
+  // of the per-column array
+  c.epi_groups = (c.acc_bufs >= 2 && c.acc_bufs % 2 == 0 && c.BN <= kMaxBN / 2 &&
+                  env_int("ADAPTION_TC_EPIGROUPS", 2) == 2) ? 2 : 1;
+  c.stage_out_bytes = c.staged ? (uint32_t)(kBM * c.BN * out_planes * c.epi_groups) : 0u;
   // dynamic shared memory: everything up to the per-block limit except the control block
   const size_t budget = 232448 - sizeof(Ctrl) - 256 - c.stage_out_bytes;
   // group short k-blocks so that a stage carries roughly 768 tensor-pipe cycles of work or more
@@ -1607,6 +1622,7 @@ int launch_tensor(const GemmProblem& g) {
   } else {
     p.rq = RequantParams{0, g.relu ? 1 : 0, 0, 0, 1};
   }
+  p.epi_groups = c.epi_groups;
   p.staged = c.staged ? 1 : 0;
   p.stage_off = c.stage_off;
   if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && p.rq.shift >= 9 && p.rq.shift <= 31 &&

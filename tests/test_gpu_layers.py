@@ -261,6 +261,19 @@ def test_ip_tensor(case, cta_mode):
     run_ip_case(np.random.default_rng(sum(case)), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_TENSOR)
 
 
+@pytest.mark.parametrize("groups", ["1", "2"])
+@pytest.mark.parametrize("with_q16", [False, True])
+def test_epilogue_groups_agree(groups, with_q16, monkeypatch):
+    """Narrow tiles (two accumulator sets in TMEM): one group of epilogue warps, or two groups taking
+    alternate tiles, give the same bits; odd and even tile counts per CTA, ReLU and signed outputs."""
+    monkeypatch.setenv("ADAPTION_TC_EPIGROUPS", groups)
+    for case in [(5, 40, 40, 64, 64, 3, 1, 1, 16, 16, 16, True),       # 63 tiles of 128 x 64
+                 (2, 30, 30, 256, 48, 3, 1, 1, 16, 16, 16, False),     # signed outputs, ragged N
+                 (37, 64, 64, 32, 32, 3, 1, 1, 16, 16, 8, True),       # BN = 32, more tiles than CTAs
+                 (37, 64, 64, 3, 64, 3, 1, 1, 16, 16, 16, True)]:      # packed taps, K = 32, 1184 tiles
+        run_conv_case(np.random.default_rng(sum(case)), *case, B.ALGO_AUTO, with_q16=with_q16)
+
+
 @pytest.mark.parametrize("case", TC_IP)
 def test_ip_tensor_staged_stores(case, cta_mode):
     Bsz, K, O, nx, nw, n_out, relu = case
