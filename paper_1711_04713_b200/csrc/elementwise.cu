@@ -213,6 +213,10 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restr
     uint32_t lo[4], hi[4], h16[8];
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
+      if (4 * w >= nreal) {               // only padding from here on: zeros, nothing to compute
+        lo[w] = hi[w] = h16[2 * w] = h16[2 * w + 1] = 0u;
+        continue;
+      }
       int32_t q[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
