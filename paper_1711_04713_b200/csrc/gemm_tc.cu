@@ -138,6 +138,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same test, but the hardware may keep the thread suspended for up to `hint_ns` while the phase
+// is incomplete (it resumes as soon as the phase completes): far fewer polling instructions.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
 // True in exactly one lane of a converged warp.  Code guarded by it still has its operands computed
 // warp-uniformly outside the guard, which lets the compiler keep them in uniform registers (the
 // tensor-core and bulk-copy instructions take uniform-register operands).
@@ -398,15 +413,15 @@ __device__ __forceinline__ uint32_t make_idesc(bool a_signed, bool b_signed, int
 
 // Bounded wait on an mbarrier phase.  Returns false once the time limit is hit (or another
 // role already gave up); the caller then leaves its loop.
-// `relaxed` waiters (producers, epilogue) sleep between polls so that their spinning does not take
-// issue slots from the MMA-issuing thread, whose instruction stream is the critical path.
+// `relaxed` waiters (producers, epilogue) let the hardware suspend them while the phase is
+// incomplete, so that their polling neither takes issue slots from the MMA-issuing thread, whose
+// instruction stream is the critical path, nor burns power during the long mainloops.
 __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, Ctrl* ctrl, const TcParams& p,
                                        bool relaxed) {
   const unsigned long long t0 = global_ns();
   uint32_t spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if (relaxed) __nanosleep(40);
-    if ((++spins & 127u) == 0) {
+  while (!(relaxed ? mbar_try_wait_suspend(bar, parity, 1000u) : mbar_try_wait(bar, parity))) {
+    if (relaxed || (++spins & 127u) == 0) {
       if (ctrl->abort) return false;
       if (global_ns() - t0 > p.timeout_ns) {
         ctrl->abort = 1;
