@@ -42,7 +42,6 @@ constexpr int kMmaWarps = 1;
 constexpr int kMmaWarp = kProducerWarps;
 constexpr int kFirstEpiWarp = kProducerWarps + kMmaWarps;
 constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
-constexpr int kMaxBN = 128;
 // int32 accumulators: the shared middle accumulator takes two products of magnitude
 // <= 128*255 per k, so a reduction of up to 32768 stays below 2^31.
 constexpr int64_t kMaxKPerAccumulation = 32768;
@@ -85,6 +84,7 @@ struct TcParams {
   int epi_groups;             // 1, or 2: the epilogue warps form two groups that take alternate tiles
   int staged;                 // outputs leave through shared memory and bulk-tensor stores
   uint32_t stage_off;         // offset of the staging planes from the ring base
+  uint32_t const_off;         // offset of the per-column epilogue constants (8 bytes per column and group)
 };
 
 // Optional per-role time stamps of CTA 0 (development builds only: -DADAPTION_TIMELINE).
@@ -108,7 +108,6 @@ struct Ctrl {
   unsigned long long b_ready;   // resident weights have landed
   uint32_t tmem_base;
   volatile uint32_t abort;
-  long long colconst[kMaxBN];   // per-column epilogue constants of the current tile
 };
 
 // ---------------------------------------------------------------------------------- PTX
@@ -673,9 +672,13 @@ __device__ __forceinline__ void store16_global(const uint32_t (&w)[8], const TcP
 // Staged stores: the tile's byte planes are assembled in shared memory (rows of BN bytes, 16-byte
 // chunks swizzled the way the bulk-tensor store expects for that row length, which also keeps the
 // 16-byte writes of a quarter warp on distinct banks) and leave as one bulk-tensor store per plane.
+// (Rows longer than the 128-byte swizzle span are kept as sub-planes of 128 columns, one store each.)
 __device__ __forceinline__ uint32_t staged_offset(int row, int chunk, int bn) {
-  uint32_t off = (uint32_t)row * (uint32_t)bn + (uint32_t)chunk * 16u;
-  return off ^ (((off >> 7) & (uint32_t)((bn >> 4) - 1) & 7u) << 4);
+  const int sub = chunk >> 3;
+  const int w = bn < 128 ? bn : 128;                       // row length of a (sub-)plane
+  uint32_t off = (uint32_t)row * (uint32_t)w + (uint32_t)(chunk & 7) * 16u;
+  off ^= ((off >> 7) & (uint32_t)((w >> 4) - 1) & 7u) << 4;
+  return off + (uint32_t)sub * (uint32_t)(kBM * 128);
 }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
@@ -1051,7 +1054,9 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     const int planes_bytes = kBM * p.BN * p.rq.out_planes;
     const uint32_t stage_lo = ring + p.stage_off + (uint32_t)(group * planes_bytes);
     const uint32_t stage_hi = stage_lo + (uint32_t)(kBM * p.BN);
-    long long* colconst = ctrl.colconst + group * (kMaxBN / 2);
+    // per-column epilogue constants of the current tile, one array per group, behind the staging planes
+    long long* colconst = reinterpret_cast<long long*>(smem_raw + (ring - smem_u32(smem_raw)) + p.const_off) +
+                          group * p.BN;
     const bool store_leader = ew == 0 && lane == 0;
     uint32_t tile_iter = (uint32_t)group;
     Counts cnt;
@@ -1151,8 +1156,11 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       epi_bar_sync(group, gthreads);
       if (p.staged && store_leader) {
         const int m_first = tc.m0 + (int)rank * kBM;
-        tma_store_2d(&map_y_lo, stage_lo, tc.n0, m_first);
-        if (p.rq.out_planes == 2) tma_store_2d(&map_y_hi, stage_hi, tc.n0, m_first);
+        for (int sub = 0; sub * 128 < p.BN; ++sub) {
+          const uint32_t so = (uint32_t)sub * (uint32_t)(kBM * 128);
+          tma_store_2d(&map_y_lo, stage_lo + so, tc.n0 + sub * 128, m_first);
+          if (p.rq.out_planes == 2) tma_store_2d(&map_y_hi, stage_hi + so, tc.n0 + sub * 128, m_first);
+        }
         bulk_commit();
       }
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 2);
@@ -1227,7 +1235,7 @@ struct TcConfig {
   int tile_m = kBM;
   int epi_groups = 1;
   bool staged = false;         // outputs staged in shared memory and written by bulk-tensor stores
-  uint32_t stage_out_bytes = 0, stage_off = 0;
+  uint32_t stage_out_bytes = 0, stage_off = 0, const_bytes = 0;
   size_t smem_bytes = 0;
   size_t workspace_bytes = 0;
 };
@@ -1238,7 +1246,17 @@ int env_int(const char* name, int dflt) {
   return std::atoi(v);
 }
 
+TcConfig make_config_impl(const GemmProblem& g, bool allow_wide);
+
+// 256-column tiles only exist as CTA pairs: if the wide attempt does not end up paired (the
+// reduction gets split, say), the ordinary configuration is taken.
 TcConfig make_config(const GemmProblem& g) {
+  TcConfig c = make_config_impl(g, true);
+  if (c.BN == 256 && !(c.ok && c.pair)) c = make_config_impl(g, false);
+  return c;
+}
+
+TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   TcConfig c;
   if (g.M <= 0 || g.N <= 0 || g.M > (int64_t)1 << 30 || g.N > (int64_t)1 << 24) return c;
   c.nax = g.x.fmt.n_bits > 8 ? 2 : 1;
@@ -1275,6 +1293,13 @@ TcConfig make_config(const GemmProblem& g) {
   c.BN = g.N <= 32 ? 32 : (g.N <= 64 ? 64 : 128);
   const int forced_bn = env_int("ADAPTION_TC_BN", 0);    // experiment knob: narrower tiles
   if ((forced_bn == 32 || forced_bn == 64) && forced_bn < c.BN) c.BN = forced_bn;
+  // Single-pass (8-bit) layers with many output channels take 256-column pair tiles: one int32
+  // accumulator per tile leaves room for two sets of 256 columns, and a 256 x 256 tile halves the
+  // operand bytes per MMA cycle, which is what limits the int8 rate (see make_config's pair notes).
+  const bool wide = allow_wide && c.nacc == 1 && c.BK == 128 && g.N >= 256 && c.num_kb >= 9 && g.M >= 1024 &&
+                    (num_sms() % 2) == 0 && forced_bn == 0 && env_int("ADAPTION_TC_PAIR", -1) != 0 &&
+                    env_int("ADAPTION_TC_WIDE", 1) != 0;
+  if (wide) c.BN = 256;
   c.tiles_m = (int)((g.M + kBM - 1) / kBM);
   c.tiles_n = (int)((g.N + c.BN - 1) / c.BN);
   c.acc_bufs = 512 / (c.nacc * c.BN);
@@ -1311,7 +1336,7 @@ TcConfig make_config(const GemmProblem& g) {
   // accumulator sets were tried for medium reductions and lost to these once the epilogue hands the
   // accumulators back early)
   const bool pair_ok = c.splits == 1 && g.M >= 1024 && (sms % 2) == 0;
-  c.pair = pair_ok && c.BN == 128 && c.BK == 128 && c.num_kb >= 9;
+  c.pair = pair_ok && c.BN >= 128 && c.BK == 128 && c.num_kb >= 9;
   if (pair_env == 0) c.pair = false;
   if (pair_env == 1 && c.splits == 1 && (sms % 2) == 0) c.pair = true;
   if (c.pair) {
@@ -1327,15 +1352,16 @@ TcConfig make_config(const GemmProblem& g) {
              g.y.c_stride >= c.BN && g.y.c_stride % 16 == 0 && env_int("ADAPTION_TC_STAGED", 1) != 0;
   // two epilogue groups when two tiles can be in flight in TMEM and their constants fit the halves
   // of the per-column array
-  c.epi_groups = (c.acc_bufs >= 2 && c.acc_bufs % 2 == 0 && c.BN <= kMaxBN / 2 &&
+  c.epi_groups = (c.acc_bufs >= 2 && c.acc_bufs % 2 == 0 && c.BN <= 64 &&
                   env_int("ADAPTION_TC_EPIGROUPS", 2) == 2) ? 2 : 1;
   c.stage_out_bytes = c.staged ? (uint32_t)(kBM * c.BN * out_planes * c.epi_groups) : 0u;
   // dynamic shared memory: everything up to the per-block limit except the control block
-  const size_t budget = 232448 - sizeof(Ctrl) - 256 - c.stage_out_bytes;
+  c.const_bytes = (uint32_t)(c.BN * c.epi_groups * sizeof(long long));
+  const size_t budget = 232448 - sizeof(Ctrl) - 256 - c.stage_out_bytes - c.const_bytes;
   // group short k-blocks so that a stage carries roughly 768 tensor-pipe cycles of work or more
   {
     const int products = c.nax * c.nbw;
-    const int cyc_per_kb = (c.BK / 32) * products * (c.BN >= 128 ? 64 : 48);
+    const int cyc_per_kb = (c.BK / 32) * products * (c.BN >= 128 ? c.BN / 2 : 48);
     int kps = (768 + cyc_per_kb - 1) / cyc_per_kb;
     if (kps > 4) kps = 4;
     const int kps_env = env_int("ADAPTION_TC_KPS", 0);
@@ -1371,7 +1397,7 @@ TcConfig make_config(const GemmProblem& g) {
   const int mmaw_env = env_int("ADAPTION_TC_MMAW", 0);      // experiment knob: force one issuing warp
   if (mmaw_env == 1) c.mma_warps = 1;
   c.stage_off = (uint32_t)(((size_t)c.stages * c.stage_bytes + c.b_res_bytes + 1023) & ~(size_t)1023);
-  c.smem_bytes = (size_t)c.stage_off + 1024 + c.stage_out_bytes;
+  c.smem_bytes = (size_t)c.stage_off + 1024 + c.stage_out_bytes + c.const_bytes;
   c.ok = true;
   return c;
 }
@@ -1600,13 +1626,14 @@ int launch_tensor(const GemmProblem& g) {
   }
 
   if (c.staged) {
-    const CUtensorMapSwizzle yswz = c.BN == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                                : (c.BN == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    const int ybox = c.BN < 128 ? c.BN : 128;       // wider tiles leave as several stores of 128 columns
+    const CUtensorMapSwizzle yswz = ybox == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                                : (ybox == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
     const void* planes[2] = {g.y.hi, g.y.lo};
     for (int i = 0; i < 2; ++i) {
       if (planes[i] == nullptr) continue;      // single-plane outputs have no high plane
       if (!encode_tiled_2d(&maps[4 + i], planes[i], (uint64_t)g.y.c_stride, (uint64_t)g.M, (uint64_t)g.y.c_stride,
-                           (uint32_t)c.BN, (uint32_t)kBM, yswz))
+                           (uint32_t)ybox, (uint32_t)kBM, yswz))
         return ADAPTION_ERR_CUDA;
     }
   }
@@ -1640,6 +1667,7 @@ int launch_tensor(const GemmProblem& g) {
   p.epi_groups = c.epi_groups;
   p.staged = c.staged ? 1 : 0;
   p.stage_off = c.stage_off;
+  p.const_off = c.stage_off + c.stage_out_bytes;
   if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && p.rq.shift >= 9 && p.rq.shift <= 31 &&
       g.N % 8 == 0 && env_int("ADAPTION_TC_FAST", 1) != 0) {
     // 32-bit bounds of the fast epilogue (see shifted32): with a reduction of kred bytes per plane row

@@ -261,6 +261,29 @@ def test_ip_tensor(case, cta_mode):
     run_ip_case(np.random.default_rng(sum(case)), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_TENSOR)
 
 
+WIDE_CONV = [
+    # single-pass layers with 256 and more output channels: 256-column pair tiles
+    (2, 24, 24, 128, 256, 3, 1, 1, 8, 8, 8, True),        # one column tile, 5 row tiles (ragged)
+    (3, 28, 28, 256, 512, 3, 1, 1, 8, 8, 8, True),        # two column tiles, two channel blocks per tap
+    (2, 24, 24, 128, 320, 3, 1, 1, 8, 8, 8, False),       # ragged N (320 = 256 + 64), signed outputs
+    (2, 24, 24, 128, 256, 3, 1, 1, 8, 8, 16, True),       # 8-bit operands, 16-bit outputs (two planes)
+    (2, 24, 24, 128, 264, 3, 1, 1, 4, 4, 4, True),        # 4-bit, N = 264
+]
+
+
+@pytest.mark.parametrize("case", WIDE_CONV)
+@pytest.mark.parametrize("with_q16", [False, True])
+@pytest.mark.parametrize("wide", ["1", "0"])
+def test_conv_single_pass_wide_tiles(case, with_q16, wide, monkeypatch):
+    monkeypatch.setenv("ADAPTION_TC_WIDE", wide)
+    run_conv_case(np.random.default_rng(sum(case)), *case, B.ALGO_TENSOR, with_q16=with_q16)
+
+
+def test_ip_single_pass_wide_tiles():
+    run_ip_case(np.random.default_rng(77), 1100, 1152, 384, 8, 8, 8, True, B.ALGO_TENSOR, with_q16=False)
+    run_ip_case(np.random.default_rng(78), 2048, 2304, 256, 8, 8, 8, False, B.ALGO_TENSOR, with_q16=True)
+
+
 @pytest.mark.parametrize("groups", ["1", "2"])
 @pytest.mark.parametrize("with_q16", [False, True])
 def test_epilogue_groups_agree(groups, with_q16, monkeypatch):
