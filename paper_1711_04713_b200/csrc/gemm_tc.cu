@@ -7,7 +7,7 @@
 // unsigned); the product of two such numbers is four int8 products
 //   q_a*q_b = 2^16 hi_a*hi_b + 2^8 (hi_a*lo_b + lo_a*hi_b) + lo_a*lo_b
 // each accumulated exactly in int32 by tcgen05.mma kind::i8 into its own TMEM accumulator
-// (the two middle terms share one) and recombined in int64 in the epilogue.  8-bit operands
+// (the two middle terms share one) and recombined exactly in the epilogue.  8-bit operands
 // take a single product.
 //
 // One persistent CTA per SM walks over output tiles (128 rows x BN columns):
@@ -54,7 +54,6 @@ struct TcParams {
   int BN, BK, ksteps;
   uint32_t sbo, layout_type;
   int stages;
-  int mma_warps;              // 1, or 2 (then ring slot s belongs to issuing warp s & 1)
   uint32_t a_bytes, b_bytes, stage_bytes;
   // a stage holds `kps` consecutive k-blocks of `kb_bytes` each (short k-blocks are grouped so
   // that the per-stage hand-shake is amortised over enough MMAs)
@@ -103,8 +102,7 @@ struct Ctrl {
   unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[kMaxAccBufs];
   unsigned long long tmem_empty[kMaxAccBufs];
-  unsigned long long first_issued[kMaxAccBufs];   // first stage of a tile is in the pipe
-  unsigned long long drain[kMmaWarps];
+  unsigned long long drain;     // the issuing warp's last commit before an early exit
   unsigned long long b_ready;   // resident weights have landed
   uint32_t tmem_base;
   volatile uint32_t abort;
@@ -265,19 +263,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
         "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
             bar),
         "h"((uint16_t)3)
-        : "memory");
-  else
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-                 : "memory");
-}
-// Same, but only the issuing (leader) CTA's barrier is signalled.
-template <bool PAIR>
-__device__ __forceinline__ void tc_commit_leader(uint32_t bar) {
-  if (PAIR)
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
-            bar),
-        "h"((uint16_t)1)
         : "memory");
   else
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
@@ -753,11 +738,10 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       mbar_init(smem_u32(&ctrl.empty[s]), 1);
     }
     for (int b = 0; b < p.acc_bufs; ++b) {
-      mbar_init(smem_u32(&ctrl.tmem_full[b]), (uint32_t)p.mma_warps);
-      mbar_init(smem_u32(&ctrl.first_issued[b]), 1);
+      mbar_init(smem_u32(&ctrl.tmem_full[b]), 1);
       mbar_init(smem_u32(&ctrl.tmem_empty[b]), (uint32_t)((PAIR ? 2 : 1) * (kEpiWarps / p.epi_groups)));
     }
-    for (int w = 0; w < kMmaWarps; ++w) mbar_init(smem_u32(&ctrl.drain[w]), 1);
+    mbar_init(smem_u32(&ctrl.drain), 1);
     mbar_init(smem_u32(&ctrl.b_ready), 1);
     ctrl.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -905,17 +889,9 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     }
     __syncwarp();
   } else if (warp < kFirstEpiWarp) {
-    // ------------------------------------------------------------------ MMA issuers (leader only)
-    // One warp, or two that walk the same loop (uniform control flow and operands) and own the
-    // ring slots of their parity: a slot's "full" barrier is then only ever waited on by the warp
-    // that also releases the slot, so no phase of it can pass unseen.
-    // In each warp one elected lane issues.  The accumulators are overwritten by a tile's first
-    // stage; the other warp may add to them only after that stage has retired, which its owner
-    // reports through a commit on `first_issued` (instructions of different threads are not
-    // ordered otherwise; integer additions commute, so nothing else needs an order).
-    const int mw = warp - kMmaWarp;
-    if (rank == 0 && mw < p.mma_warps) {
-      const bool solo = p.mma_warps == 1;
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    // The warp walks the stages in uniform control flow; one elected lane issues.
+    if (rank == 0) {
       const int tile_rows = PAIR ? 2 * kBM : kBM;
       const uint32_t id_ss = make_idesc(true, true, p.BN, tile_rows);
       const uint32_t id_su = make_idesc(true, false, p.BN, tile_rows);
@@ -943,33 +919,26 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const TileCoord tc = decode_tile(t, p);
         const uint32_t buf = tile_iter % (uint32_t)p.acc_bufs;
         const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
-        if (lane == 0 && mw == 0) TL_STAMP(1, tile_iter, 0);
+        if (lane == 0) TL_STAMP(1, tile_iter, 0);
         ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p, false));
         if (!ok) break;
         tc_fence_after();
-        if (lane == 0 && mw == 0) TL_STAMP(1, tile_iter, 1);
+        if (lane == 0) TL_STAMP(1, tile_iter, 1);
         const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
         const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
         uint32_t bres = bres_lo + (uint32_t)tc.kb_begin * bres_u;   // resident weights of this k-block
-        bool after_first = solo || (s & 1) == mw;     // the first stage's owner needs no hand-shake
         for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps) {
           const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;
-          const bool mine = solo || (s & 1) == mw;
-          if (mine) {
+          {
 #ifdef ADAPTION_TIMELINE
           const long long tw0 = clock64();
 #endif
           ok = __all_sync(0xffffffffu, wait_bar(full_bar, ph, &ctrl, p, false));
 #ifdef ADAPTION_TIMELINE
           if (lane == 0 && blockIdx.x == 0 && tile_iter < 32u)
-            g_timeline[((1 + mw * 3) * 32 + tile_iter) * 8 + 3] += clock64() - tw0;   // time waiting for data
+            g_timeline[(1 * 32 + tile_iter) * 8 + 3] += clock64() - tw0;   // time waiting for data
 #endif
           if (!ok) break;
-          if (!after_first) {
-            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.first_issued[buf]), bph, &ctrl, p, false));
-            if (!ok) break;
-            after_first = true;
-          }
           tc_fence_after();
           const uint32_t acc = kb == tc.kb_begin ? 0u : 1u;
           if (elect_one()) {
@@ -1008,7 +977,6 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
               }
             }
             tc_commit<PAIR>(empty_bar);                        // stage reusable once these MMAs retire
-            if (!solo && kb == tc.kb_begin) tc_commit_leader<PAIR>(smem_u32(&ctrl.first_issued[buf]));
           }
           }
           if (GROUPED) bres += (uint32_t)nkb * bres_u;
@@ -1025,13 +993,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         }
         if (ok && elect_one()) tc_commit<PAIR>(smem_u32(&ctrl.tmem_full[buf]));   // tile complete
         __syncwarp();
-        if (lane == 0 && mw == 0) TL_STAMP(1, tile_iter, 2);
+        if (lane == 0) TL_STAMP(1, tile_iter, 2);
       }
       if ((!ok || ctrl.abort) && lane == 0) {
         // make sure no MMA still reads shared memory or writes TMEM when the CTAs tear down
-        tc_commit<false>(smem_u32(&ctrl.drain[mw]));
+        tc_commit<false>(smem_u32(&ctrl.drain));
         const unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(smem_u32(&ctrl.drain[mw]), 0) && global_ns() - t0 < 50000000ull) {
+        while (!mbar_try_wait(smem_u32(&ctrl.drain), 0) && global_ns() - t0 < 50000000ull) {
         }
       }
     }
@@ -1220,7 +1188,6 @@ struct TcConfig {
   uint32_t layout_type = 0;
   int nax = 1, nbw = 1, nacc = 1;
   int stages = 0;
-  int mma_warps = 1;
   uint32_t a_bytes = 0, b_bytes = 0, stage_bytes = 0;
   int acc_bufs = 1;
   uint32_t tmem_cols = 32;
@@ -1393,9 +1360,6 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   const int stage_cap = env_int("ADAPTION_TC_STAGES", 0);   // experiment knob: shallower ring
   if (stage_cap >= 2 && stage_cap < c.stages) c.stages = stage_cap;
   if (c.stages < 2) return c;
-  c.mma_warps = kMmaWarps;
-  const int mmaw_env = env_int("ADAPTION_TC_MMAW", 0);      // experiment knob: force one issuing warp
-  if (mmaw_env == 1) c.mma_warps = 1;
   c.stage_off = (uint32_t)(((size_t)c.stages * c.stage_bytes + c.b_res_bytes + 1023) & ~(size_t)1023);
   c.smem_bytes = (size_t)c.stage_off + 1024 + c.stage_out_bytes + c.const_bytes;
   c.ok = true;
@@ -1646,7 +1610,7 @@ int launch_tensor(const GemmProblem& g) {
   p.num_kb = c.num_kb; p.kb_per_split = c.kb_per_split;
   p.BN = c.BN; p.BK = c.BK; p.ksteps = c.BK / 32;
   p.sbo = (uint32_t)(8 * c.BK); p.layout_type = c.layout_type;
-  p.stages = c.stages; p.mma_warps = c.mma_warps; p.a_bytes = c.a_bytes; p.b_bytes = c.b_bytes; p.stage_bytes = c.stage_bytes;
+  p.stages = c.stages; p.a_bytes = c.a_bytes; p.b_bytes = c.b_bytes; p.stage_bytes = c.stage_bytes;
   p.kps = c.kps; p.kb_bytes = c.kb_bytes;
   p.b_resident = c.b_resident ? 1 : 0;
   p.b_res_off = (uint32_t)c.stages * c.stage_bytes;
