@@ -128,6 +128,15 @@ ADAPTION_API int adaption_quantize_stochastic(const float* d_x, size_t outer, si
                                  const adaption_qfmt* d_fmt, int32_t relu, uint64_t seed,
                                  adaption_stats* d_stats, void* stream);
 
+/* Sec. 2.1 + 2.4 (LPAct with rounding_scheme STOCHASTIC).  As adaption_lp_act.  fp32 input:
+ * adaption_quantize_stochastic.  Fixed-point input (format change f_in -> f_out, s = f_in - f_out):
+ * for s > 0 the stored integer v (after ReLU) gives v / 2^s = floor + rem / 2^s and moves up with
+ * probability rem / 2^s (threshold rem * 2^(32 - s) against the same per-element draw); for
+ * s <= 0 the shift is exact and nothing is drawn. */
+ADAPTION_API int adaption_lp_act_stochastic(const float* d_x_f32, const adaption_qtensor* h_x_q, size_t outer,
+                               size_t inner, int32_t relu, adaption_qtensor out, const adaption_qfmt* d_fmt,
+                               uint64_t seed, adaption_stats* d_stats, void* stream);
+
 /* Sec. 2.3 (iterative, thresholded allocation of the integer bits).  Adds to d_hist[0..17) (device,
  * uint64, caller zeroes it before the first tensor of a group) the number of elements of
  * x[0..numel) that need b integer bits: b = 0 for |x| < 1, else floor(log2 |x|) + 1; bin 16 also

@@ -82,3 +82,28 @@ def quantize_stochastic(x, n_bits: int, frac_bits: int, seed: int, relu: bool = 
     q = np.clip(r, qmin, qmax)
     zeros = int((q == 0).sum())
     return q.astype(np.int16).reshape(x.shape), (zeros, sat_pos, sat_neg)
+
+
+def requantize_stochastic(xq, in_frac_bits: int, relu: bool, out_n_bits: int, out_frac_bits: int, seed: int):
+    """LPAct on an already quantized tensor with stochastic rounding: format change f_in -> f_out.
+    The stored integer v (after the optional ReLU) stands for v * 2^-f_in; with s = f_in - f_out > 0
+    the exact quotient v / 2^s = floor + rem / 2^s moves up with probability rem / 2^s, taken as
+    T = rem * 2^(32 - s) against the same 32-bit draw as in S2 (exact: s <= 15); s <= 0 is an exact
+    left shift.  Saturation and counters as in the deterministic requantizer."""
+    q = np.ascontiguousarray(xq, dtype=np.int16)
+    v = q.reshape(-1).astype(np.int64)
+    if relu:
+        v = np.maximum(v, 0)
+    s = in_frac_bits - out_frac_bits
+    qmin, qmax = -(1 << (out_n_bits - 1)), (1 << (out_n_bits - 1)) - 1
+    if s > 0:
+        lo = v >> s                                   # floor division by 2^s (arithmetic shift)
+        rem = v - (lo << s)                           # 0 <= rem < 2^s
+        T = (rem << (32 - s)).astype(np.uint64)
+        r = lo + (draws(v.size, seed) < T).astype(np.int64)
+    else:
+        r = v << (-s)
+    sat_pos = int((r > qmax).sum())
+    sat_neg = int((r < qmin).sum())
+    y = np.clip(r, qmin, qmax)
+    return y.astype(np.int16).reshape(q.shape), (int((y == 0).sum()), sat_pos, sat_neg)

@@ -50,6 +50,7 @@ EXPORTS = [
     "adaption_probe_i8_peak", "adaption_status_string",
     "adaption_quantize_stochastic", "adaption_bit_histogram", "adaption_width_histogram",
     "adaption_choose_frac_bits_from_hist", "adaption_choose_frac_bits_from_widths",
+    "adaption_lp_act_stochastic",
 ]
 HIST_BINS = 17
 
@@ -91,6 +92,8 @@ def load(path: str | None = None):
     lib.adaption_choose_frac_bits_from_acc.argtypes = [I64, I32, I32, C.POINTER(adaption_qfmt)]
     lib.adaption_probe_i8_peak.argtypes = [I32, I32, I32, I32, P, P, P]
     lib.adaption_quantize_stochastic.argtypes = [P, SZ, SZ, adaption_qtensor, P, I32, C.c_uint64, P, P]
+    lib.adaption_lp_act_stochastic.argtypes = [P, C.POINTER(adaption_qtensor), SZ, SZ, I32, adaption_qtensor, P,
+                                               C.c_uint64, P, P]
     lib.adaption_bit_histogram.argtypes = [P, SZ, P, P]
     lib.adaption_width_histogram.argtypes = [adaption_qtensor, SZ, SZ, P, P]
     lib.adaption_choose_frac_bits_from_hist.argtypes = [C.POINTER(C.c_uint64), I32, C.c_double,
@@ -211,6 +214,15 @@ def adaption_quantize_stochastic(x: torch.Tensor, outer: int, inner: int, out: Q
     _check(load().adaption_quantize_stochastic(_ptr(x), outer, inner, out.c_struct(), _ptr(d_fmt), int(relu),
                                                seed & 0xFFFFFFFFFFFFFFFF, _ptr(d_stats), _stream()),
            "adaption_quantize_stochastic")
+
+
+def adaption_lp_act_stochastic(x_f32: torch.Tensor | None, x_q: QTensor | None, outer: int, inner: int, relu: bool,
+                               out: QTensor, seed: int, d_fmt: torch.Tensor | None = None,
+                               d_stats: torch.Tensor | None = None):
+    xq = None if x_q is None else C.byref(x_q.c_struct())
+    _check(load().adaption_lp_act_stochastic(_ptr(x_f32), xq, outer, inner, int(relu), out.c_struct(), _ptr(d_fmt),
+                                             seed & 0xFFFFFFFFFFFFFFFF, _ptr(d_stats), _stream()),
+           "adaption_lp_act_stochastic")
 
 
 def new_hist(device="cuda") -> torch.Tensor:

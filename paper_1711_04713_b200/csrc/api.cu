@@ -21,6 +21,8 @@ int maxpool_impl(const adaption_qtensor&, int32_t, int32_t, int32_t, int32_t, co
 
 int quantize_stochastic_impl(const float*, size_t, size_t, const adaption_qtensor&, const adaption_qfmt*, int32_t,
                              uint64_t, adaption_stats*, cudaStream_t);
+int requant_stochastic_impl(const adaption_qtensor&, size_t, size_t, int32_t, const adaption_qtensor&,
+                            const adaption_qfmt*, uint64_t, adaption_stats*, cudaStream_t);
 int bit_histogram_impl(const float*, size_t, uint64_t*, cudaStream_t);
 int width_histogram_impl(const adaption_qtensor&, size_t, size_t, uint64_t*, cudaStream_t);
 int choose_frac_bits_from_hist(const uint64_t*, int32_t, double, adaption_qfmt*);
@@ -159,6 +161,20 @@ int adaption_quantize_stochastic(const float* d_x, size_t outer, size_t inner, a
                                  adaption_stats* d_stats, void* stream) {
   return quantize_stochastic_impl(d_x, outer, inner, out, d_fmt, relu, seed, d_stats,
                                   reinterpret_cast<cudaStream_t>(stream));
+}
+
+int adaption_lp_act_stochastic(const float* d_x_f32, const adaption_qtensor* h_x_q, size_t outer, size_t inner,
+                               int32_t relu, adaption_qtensor out, const adaption_qfmt* d_fmt, uint64_t seed,
+                               adaption_stats* d_stats, void* stream) {
+  if ((d_x_f32 == nullptr) == (h_x_q == nullptr)) {
+    if (outer == 0 || inner == 0) return ADAPTION_OK;
+    return ADAPTION_ERR_INVALID_ARG;
+  }
+  if (d_x_f32 != nullptr)
+    return quantize_stochastic_impl(d_x_f32, outer, inner, out, d_fmt, relu, seed, d_stats,
+                                    reinterpret_cast<cudaStream_t>(stream));
+  return requant_stochastic_impl(*h_x_q, outer, inner, relu, out, d_fmt, seed, d_stats,
+                                 reinterpret_cast<cudaStream_t>(stream));
 }
 
 int adaption_bit_histogram(const float* d_x, size_t numel, uint64_t* d_hist, void* stream) {

@@ -116,3 +116,31 @@ def test_quantize_stochastic_properties_at_size():
     with pytest.raises(B.AdaptionError) as e:
         B.adaption_quantize(xd, 1, x.size, out, None, B.ROUND_STOCHASTIC)
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("n_in,f_in,n_out,f_out,relu", [
+    (16, 12, 16, 6, False), (16, 12, 8, 3, True), (16, 10, 16, 10, False), (16, 4, 16, 9, True),
+    (8, 6, 8, 2, False), (12, 8, 4, 1, True), (8, 3, 16, 0, False)])
+@pytest.mark.parametrize("shape", [(1000, 64), (37, 3), (129, 20)])
+def test_lp_act_stochastic_format_change(n_in, f_in, n_out, f_out, relu, shape):
+    rng = np.random.default_rng(n_in + f_in + n_out + shape[0])
+    q = rng.integers(-(1 << (n_in - 1)), 1 << (n_in - 1), shape).astype(np.int16)
+    q.flat[:3] = [-(1 << (n_in - 1)), (1 << (n_in - 1)) - 1, 0]
+    seed = 0xC0FFEE00 + shape[1]
+    want, (z, sp, sn) = st.requantize_stochastic(q, f_in, relu, n_out, f_out, seed)
+    xin = to_qtensor(q, n_in, f_in)
+    out = B.QTensor.empty(shape[0], shape[1], n_out, f_out, None, with_q16=True)
+    stats = B.new_stats()
+    B.adaption_lp_act_stochastic(None, xin, shape[0], shape[1], relu, out, seed, None, stats)
+    assert np.array_equal(from_qtensor(out), want)
+    assert np.array_equal(q16_of(out), want)
+    assert out.padding_is_zero()
+    assert stats_tuple(stats) == (z, sp, sn)
+
+
+def test_lp_act_stochastic_fp32_is_the_stochastic_quantizer_with_relu():
+    x = (np.random.default_rng(9).standard_normal((300, 48)) * 3).astype(np.float32)
+    want, _ = st.quantize_stochastic(x, 16, 9, 77, relu=True)
+    out = B.QTensor.empty(300, 48, 16, 9)
+    B.adaption_lp_act_stochastic(dev(x), None, 300, 48, True, out, 77)
+    assert np.array_equal(from_qtensor(out), want)

@@ -508,3 +508,28 @@ def test_stochastic_rounding_support_and_expectation():
     qd, _ = orc.quantize(xr, 16, 10)
     qs2, _ = st.quantize_stochastic(xr, 16, 10, seed=8)
     assert np.all(np.abs(qd.astype(np.int64) - qs2.astype(np.int64)) <= 1)
+
+
+def test_stochastic_requantization_support_expectation_and_exact_cases():
+    """Format change of stored integers with stochastic rounding: one of the two neighbours of
+    v / 2^s, mean equal to it, exact when v is a multiple of 2^s or when the shift is to the left,
+    and never further than one step from the deterministic requantizer."""
+    from oracle import stochastic as st
+    vals = np.array([5, -5, 1, -1, 1023, -1023, 12345, -12345, 7, 64], dtype=np.int16)
+    reps = 20000
+    y, _ = st.requantize_stochastic(np.tile(vals, reps), 10, False, 16, 4, seed=11)      # s = 6
+    y = y.reshape(reps, vals.size).astype(np.float64)
+    exact = vals.astype(np.float64) / 64.0
+    assert np.all((y == np.floor(exact)) | (y == np.floor(exact) + 1))
+    assert np.all(np.abs(y.mean(axis=0) - exact) < 5 * np.sqrt(0.25 / reps))
+    assert np.all(y[:, 9] == 1.0)                                                         # 64 / 64 exactly
+    up, _ = st.requantize_stochastic(vals, 4, False, 16, 6, seed=1)                       # left shift by 2
+    assert np.array_equal(up[:6], vals[:6] * 4) and up[6] == 32767 and up[7] == -32768     # 12345 * 4 saturates
+    rng = np.random.default_rng(2)
+    q = rng.integers(-32768, 32768, 5000).astype(np.int16)
+    for relu in (False, True):
+        ys, (z, sp, sn) = st.requantize_stochastic(q, 12, relu, 8, 3, seed=5)            # s = 9, saturating
+        yd, cd = orc.requantize(q, 12, relu, 8, 3)
+        assert np.all(np.abs(ys.astype(np.int64) - yd.astype(np.int64)) <= 1)
+        assert z == int((ys == 0).sum()) and sn == (0 if relu else sn)
+        assert abs(sp - cd.sat_pos) <= int((np.abs(q.astype(np.int64) - 127 * 512) < 512).sum()) + 1
