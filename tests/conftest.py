@@ -27,3 +27,11 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _cuda_library_is_current():
+    """Build the CUDA library in-tree if it is missing or older than its sources (a no-op otherwise),
+    so that a fresh checkout runs the tests against the code it contains."""
+    from paper_1711_04713_b200 import build
+    build.build_library()
