@@ -145,11 +145,11 @@ __device__ __forceinline__ void store4(const QuantOut& o, size_t word, int32_t q
                                        int32_t q2, int32_t q3) {
   const uint32_t lo = (uint32_t)(q0 & 255) | ((uint32_t)(q1 & 255) << 8) |
                       ((uint32_t)(q2 & 255) << 16) | ((uint32_t)(q3 & 255) << 24);
-  o.lo[word] = lo;
+  __stcs(o.lo + word, lo);                    // streaming stores: the planes are read much later
   if (o.planes == 2) {
     const uint32_t hi = (uint32_t)((q0 >> 8) & 255) | ((uint32_t)((q1 >> 8) & 255) << 8) |
                         ((uint32_t)((q2 >> 8) & 255) << 16) | ((uint32_t)((q3 >> 8) & 255) << 24);
-    o.hi[word] = hi;
+    __stcs(o.hi + word, hi);
   }
   if (o.q16 != nullptr) {
     uint2 v;

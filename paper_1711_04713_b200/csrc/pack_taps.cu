@@ -28,77 +28,90 @@ struct PackParams {
   int H, W, OH, OW, R, S, pad_h, pad_w, stride_h, stride_w;
 };
 
-// One thread gathers one packed row of one plane.  C is a template parameter so that every byte
-// position t*C + c is known at compile time and the eight output words stay in registers.
-// Each tap is read as one aligned 32-bit word (the channel pitch is a multiple of 16 bytes and
-// C <= 4), of which the low C bytes are used.
+// One thread gathers the packed rows of one output pixel (or weight row) in every plane, so that
+// the index arithmetic is done once.  C is a template parameter so that every byte position
+// t*C + c is known at compile time and the eight output words stay in registers.  Each tap is read
+// as one aligned 32-bit word (the channel pitch is a multiple of 16 bytes and C <= 4), of which the
+// low C bytes are used.  Pixels whose whole window lies inside the image skip the bounds tests.
+template <int C, bool CHECKED>
+__device__ __forceinline__ void pack_row(const uint8_t* __restrict__ src, long long base, long long tap_pitch,
+                                         long long row_pitch, int taps, int S, int ih0, int iw0, int H, int W,
+                                         uint8_t* __restrict__ dst) {
+  constexpr int kMaxTaps = kPackK / C;
+  uint32_t out[kPackK / 4];
+#pragma unroll
+  for (int j = 0; j < kPackK / 4; ++j) out[j] = 0u;
+  int r = 0, s = 0;
+  long long off = base;                 // element offset of the current tap
+#pragma unroll
+  for (int t = 0; t < kMaxTaps; ++t) {
+    uint32_t v = 0u;
+    if (t < taps) {
+      bool inside = true;
+      if (CHECKED) {
+        const int ih = ih0 + r, iw = iw0 + s;
+        inside = ih >= 0 && ih < H && iw >= 0 && iw < W;
+      }
+      if (inside) v = __ldg(reinterpret_cast<const unsigned int*>(src + off));
+    }
+    v &= 0xffffffffu >> (32 - 8 * C);
+    // bytes t*C .. t*C + C - 1 of the packed row (may straddle two words)
+    const int k0 = t * C;
+    const int w0 = k0 >> 2, sh = (k0 & 3) * 8;
+    out[w0] |= v << sh;
+    if (sh + 8 * C > 32) out[w0 + 1] |= v >> (32 - sh);
+    off += tap_pitch;
+    if (++s == S) { s = 0; ++r; off += row_pitch - (long long)S * tap_pitch; }
+  }
+  uint4* d = reinterpret_cast<uint4*>(dst);
+  d[0] = make_uint4(out[0], out[1], out[2], out[3]);
+  d[1] = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
 template <int C>
 __global__ void __launch_bounds__(256) pack_taps_kernel(const PackParams p) {
-  constexpr int kMaxTaps = kPackK / C;
-  const long long total = p.rows * p.planes;
   const int taps = p.R * p.S;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-       i += (long long)gridDim.x * blockDim.x) {
-    // (there are at most two planes: no division)
-    const int plane = i >= p.rows ? 1 : 0;
-    const long long m = plane ? i - p.rows : i;
-    const uint8_t* __restrict__ src = p.src[plane];
-    long long base;            // element offset of tap (0, 0), channel 0
-    int ih0 = 0, iw0 = 0;
+  for (long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x; m < p.rows;
+       m += (long long)gridDim.x * blockDim.x) {
     if (p.is_weight) {
-      base = m * (long long)taps * p.c_stride;
+      // [rows][R*S][c_stride]: consecutive taps are one pitch apart, always in bounds
+      for (int plane = 0; plane < p.planes; ++plane)
+        pack_row<C, false>(p.src[plane], m * (long long)taps * p.c_stride, p.c_stride, (long long)p.S * p.c_stride,
+                           taps, p.S, 0, 0, 0, 0, p.dst[plane] + m * kPackK);
+      continue;
+    }
+    // pixel index -> (image, row, column); 32-bit arithmetic whenever the index fits
+    int ow, oh;
+    long long img;
+    if (p.rows <= 0x7fffffffll) {
+      const unsigned mu = (unsigned)m, rest = mu / (unsigned)p.OW;
+      ow = (int)(mu - rest * (unsigned)p.OW);
+      const unsigned im = rest / (unsigned)p.OH;
+      oh = (int)(rest - im * (unsigned)p.OH);
+      img = im;
     } else {
-      // pixel index -> (image, row, column); 32-bit arithmetic whenever the index fits
-      int ow, oh;
-      long long img;
-      if (p.rows <= 0x7fffffffll) {
-        const unsigned mu = (unsigned)m, rest = mu / (unsigned)p.OW;
-        ow = (int)(mu - rest * (unsigned)p.OW);
-        const unsigned im = rest / (unsigned)p.OH;
-        oh = (int)(rest - im * (unsigned)p.OH);
-        img = im;
-      } else {
-        ow = (int)(m % p.OW);
-        const long long rest = m / p.OW;
-        oh = (int)(rest % p.OH);
-        img = rest / p.OH;
-      }
-      ih0 = oh * p.stride_h - p.pad_h;
-      iw0 = ow * p.stride_w - p.pad_w;
-      base = ((img * p.H + ih0) * (long long)p.W + iw0) * p.c_stride;
+      ow = (int)(m % p.OW);
+      const long long rest = m / p.OW;
+      oh = (int)(rest % p.OH);
+      img = rest / p.OH;
     }
-    uint32_t out[kPackK / 4];
-#pragma unroll
-    for (int j = 0; j < kPackK / 4; ++j) out[j] = 0u;
-    int r = 0, s = 0;
-#pragma unroll
-    for (int t = 0; t < kMaxTaps; ++t) {
-      uint32_t v = 0u;
-      if (t < taps) {
-        if (p.is_weight) {
-          v = *reinterpret_cast<const uint32_t*>(src + base + (long long)t * p.c_stride);
-        } else {
-          const int ih = ih0 + r, iw = iw0 + s;
-          if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
-            v = *reinterpret_cast<const uint32_t*>(src + base + ((long long)r * p.W + s) * p.c_stride);
-        }
-      }
-      v &= 0xffffffffu >> (32 - 8 * C);
-      // bytes t*C .. t*C + C - 1 of the packed row (may straddle two words)
-      const int k0 = t * C;
-      const int w0 = k0 >> 2, sh = (k0 & 3) * 8;
-      out[w0] |= v << sh;
-      if (sh + 8 * C > 32) out[w0 + 1] |= v >> (32 - sh);
-      if (++s == p.S) { s = 0; ++r; }
+    const int ih0 = oh * p.stride_h - p.pad_h, iw0 = ow * p.stride_w - p.pad_w;
+    const long long base = ((img * p.H + ih0) * (long long)p.W + iw0) * p.c_stride;
+    const long long row_pitch = (long long)p.W * p.c_stride;
+    const bool interior = ih0 >= 0 && ih0 + p.R <= p.H && iw0 >= 0 && iw0 + p.S <= p.W;
+    for (int plane = 0; plane < p.planes; ++plane) {
+      if (interior)
+        pack_row<C, false>(p.src[plane], base, p.c_stride, row_pitch, taps, p.S, ih0, iw0, p.H, p.W,
+                           p.dst[plane] + m * kPackK);
+      else
+        pack_row<C, true>(p.src[plane], base, p.c_stride, row_pitch, taps, p.S, ih0, iw0, p.H, p.W,
+                          p.dst[plane] + m * kPackK);
     }
-    uint4* dst = reinterpret_cast<uint4*>(p.dst[plane] + m * kPackK);
-    dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
-    dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
   }
 }
 
 int launch_pack(const PackParams& p, int C, cudaStream_t stream) {
-  const long long total = p.rows * p.planes;
+  const long long total = p.rows;
   if (total == 0) return ADAPTION_OK;
   long long blocks = (total + 255) / 256;
   const long long cap = (long long)num_sms() * 16;
