@@ -186,6 +186,28 @@ ADAPTION_API int adaption_lp_conv_fwd(const adaption_conv_shape* h_shape, adapti
                          adaption_stats* d_stats, void* d_workspace, size_t workspace_bytes,
                          void* stream);
 
+/* Sec. 2 + Table 1 "Pooling" (LPConvolution followed by the 2x2 / stride-2 max-pool of its output,
+ * as in VGG16 and Giga1Net).  y is the pooled tensor [N, OH/2, OW/2, K] in the layer's output format;
+ * OH and OW must be even.  The result equals adaption_lp_conv_fwd followed by adaption_maxpool2x2
+ * (the quantizer is monotone, so pooling the stored integers is exact); d_stats counts the
+ * convolution's own outputs, before pooling.  Requantizing mode only.  The convolution's output
+ * lives in the workspace: where the tensor-core path can, only the maxima of horizontal pixel
+ * pairs are stored there (half the bytes written and read back), otherwise all of it.
+ * phases: ADAPTION_PHASE_CONV | ADAPTION_PHASE_POOL runs the whole layer pair; the two phases may
+ * also be issued by two calls with otherwise identical arguments (convolution first, same stream
+ * order, workspace untouched in between), e.g. to time them apart.
+ * y_c_stride in the query is the pitch of y. */
+#define ADAPTION_PHASE_CONV 1
+#define ADAPTION_PHASE_POOL 2
+ADAPTION_API size_t adaption_lp_conv_pool_workspace_bytes(const adaption_conv_shape* h_shape, adaption_qfmt fx,
+                                             adaption_qfmt fw, adaption_qfmt fy, int64_t c_stride,
+                                             int64_t y_c_stride, int32_t algo);
+ADAPTION_API int adaption_lp_conv_pool_fwd(const adaption_conv_shape* h_shape, adaption_qtensor x,
+                              adaption_qtensor w, const int16_t* d_bias_q, int32_t bias_frac_bits,
+                              int32_t relu, int32_t algo, int32_t phases, adaption_qtensor y,
+                              adaption_stats* d_stats, void* d_workspace, size_t workspace_bytes,
+                              void* stream);
+
 /* Sec. 2 (LPInnerProduct forward).  y[b,o] = requant(relu(sum_k x[b,k] * w[o,k] + bias[o])).
  * x is [B][K], w is [O][K], y is [B][O]. */
 ADAPTION_API size_t adaption_lp_ip_workspace_bytes(int64_t B, int64_t K, int64_t O, adaption_qfmt fx,

@@ -21,6 +21,7 @@ ERR_K_TOO_LARGE, ERR_CUDA, ERR_TIMEOUT = 5, 6, 7
 ROUND_DETERMINISTIC, ROUND_STOCHASTIC = 0, 1
 MODE_REQUANT, MODE_RANGE = 0, 1
 ALGO_AUTO, ALGO_TENSOR, ALGO_DIRECT = 0, 1, 2
+PHASE_CONV, PHASE_POOL = 1, 2
 
 
 class adaption_qfmt(C.Structure):
@@ -50,7 +51,7 @@ EXPORTS = [
     "adaption_probe_i8_peak", "adaption_status_string",
     "adaption_quantize_stochastic", "adaption_bit_histogram", "adaption_width_histogram",
     "adaption_choose_frac_bits_from_hist", "adaption_choose_frac_bits_from_widths",
-    "adaption_lp_act_stochastic",
+    "adaption_lp_act_stochastic", "adaption_lp_conv_pool_workspace_bytes", "adaption_lp_conv_pool_fwd",
 ]
 HIST_BINS = 17
 
@@ -82,6 +83,11 @@ def load(path: str | None = None):
     lib.adaption_lp_conv_workspace_bytes.restype = SZ
     lib.adaption_lp_conv_fwd.argtypes = [C.POINTER(adaption_conv_shape), adaption_qtensor, adaption_qtensor,
                                          P, I32, I32, I32, I32, adaption_qtensor, P, P, SZ, P]
+    lib.adaption_lp_conv_pool_workspace_bytes.argtypes = [C.POINTER(adaption_conv_shape), adaption_qfmt,
+                                                          adaption_qfmt, adaption_qfmt, I64, I64, I32]
+    lib.adaption_lp_conv_pool_workspace_bytes.restype = SZ
+    lib.adaption_lp_conv_pool_fwd.argtypes = [C.POINTER(adaption_conv_shape), adaption_qtensor, adaption_qtensor,
+                                              P, I32, I32, I32, I32, adaption_qtensor, P, P, SZ, P]
     lib.adaption_lp_ip_workspace_bytes.argtypes = [I64, I64, I64, adaption_qfmt, adaption_qfmt, I32]
     lib.adaption_lp_ip_workspace_bytes.restype = SZ
     lib.adaption_lp_ip_fwd.argtypes = [I64, I64, I64, adaption_qtensor, adaption_qtensor, P, I32, I32, I32,
@@ -104,7 +110,7 @@ def load(path: str | None = None):
     lib.adaption_status_string.restype = C.c_char_p
     for name in EXPORTS:
         if name not in ("adaption_lp_conv_workspace_bytes", "adaption_lp_ip_workspace_bytes",
-                        "adaption_status_string"):
+                        "adaption_lp_conv_pool_workspace_bytes", "adaption_status_string"):
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -282,6 +288,21 @@ def adaption_lp_conv_fwd(shape: adaption_conv_shape, x: QTensor, w: QTensor, bia
     _check(load().adaption_lp_conv_fwd(C.byref(shape), x.c_struct(), w.c_struct(), _ptr(bias_q),
                                        bias_frac_bits, int(relu), mode, algo, ys, _ptr(d_stats),
                                        _ptr(workspace), wsb, _stream()), "adaption_lp_conv_fwd")
+
+
+def adaption_lp_conv_pool_workspace_bytes(shape: adaption_conv_shape, fx: adaption_qfmt, fw: adaption_qfmt,
+                                          fy: adaption_qfmt, c_stride: int, y_c_stride: int,
+                                          algo: int = ALGO_AUTO) -> int:
+    return int(load().adaption_lp_conv_pool_workspace_bytes(C.byref(shape), fx, fw, fy, c_stride, y_c_stride, algo))
+
+
+def adaption_lp_conv_pool_fwd(shape: adaption_conv_shape, x: QTensor, w: QTensor, bias_q: torch.Tensor | None,
+                              bias_frac_bits: int, relu: bool, algo: int, y: QTensor, d_stats: torch.Tensor,
+                              workspace: torch.Tensor | None, phases: int = 3):
+    wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().adaption_lp_conv_pool_fwd(C.byref(shape), x.c_struct(), w.c_struct(), _ptr(bias_q), bias_frac_bits,
+                                            int(relu), algo, phases, y.c_struct(), _ptr(d_stats), _ptr(workspace),
+                                            wsb, _stream()), "adaption_lp_conv_pool_fwd")
 
 
 def adaption_lp_ip_workspace_bytes(B: int, K: int, O: int, fx: adaption_qfmt, fw: adaption_qfmt,

@@ -17,7 +17,7 @@ int requant_impl(const adaption_qtensor&, size_t, size_t, int32_t, const adaptio
                  const adaption_qfmt*, int32_t, adaption_stats*, cudaStream_t);
 int measure_range_impl(const float*, size_t, int32_t, float*, adaption_qfmt*, cudaStream_t);
 int maxpool_impl(const adaption_qtensor&, int32_t, int32_t, int32_t, int32_t, const adaption_qtensor&,
-                 cudaStream_t);
+                 cudaStream_t, bool half_pooled = false);
 
 int quantize_stochastic_impl(const float*, size_t, size_t, const adaption_qtensor&, const adaption_qfmt*, int32_t,
                              uint64_t, adaption_stats*, cudaStream_t);
@@ -138,6 +138,41 @@ static int dispatch(const GemmProblem& g, int32_t algo) {
   return launch_direct(g);
 }
 
+// ---- LPConvolution followed by the 2x2 max-pool of its output -------------------------------
+// The convolution's own output goes to temporary planes in the workspace (behind whatever the
+// convolution itself needs there): only its horizontal pair maxima when the tensor-core path can
+// store those (half the bytes), else all of it; a pooling pass then writes y.
+struct ConvPoolPlan {
+  bool fused = false;        // the layer kernel stores horizontal maxima
+  size_t conv_ws = 0;        // bytes the convolution needs at the start of the workspace
+  size_t plane = 0;          // bytes of one temporary plane
+  size_t total = 0;
+};
+
+static ConvPoolPlan plan_conv_pool(GemmProblem g, int32_t algo) {
+  ConvPoolPlan pl;
+  const int planes = g.y.fmt.n_bits > 8 ? 2 : 1;
+  // a stand-in output of the right shape decides whether the staged (pool-capable) stores apply
+  g.y.lo = reinterpret_cast<void*>(uintptr_t(256));
+  g.y.hi = planes == 2 ? reinterpret_cast<void*>(uintptr_t(256)) : nullptr;
+  g.y.q16 = nullptr;
+  const bool packs = algo != ADAPTION_ALGO_DIRECT && pack_taps_applicable(g);
+  if (algo != ADAPTION_ALGO_DIRECT) {
+    if (packs) {
+      pl.conv_ws = pack_taps_workspace(g);
+      pl.fused = pack_taps_can_pool(g);
+    } else if (tensor_path_supported(g)) {
+      pl.conv_ws = tensor_path_workspace(g);
+      pl.fused = tensor_path_can_pool(g);
+    }
+  }
+  pl.conv_ws = (pl.conv_ws + 255) & ~(size_t)255;
+  const size_t rows = pl.fused ? (size_t)g.M / 2 : (size_t)g.M;
+  pl.plane = (rows * (size_t)g.y.c_stride + 255) & ~(size_t)255;
+  pl.total = pl.conv_ws + (size_t)planes * pl.plane;
+  return pl;
+}
+
 }  // namespace adaption
 
 using namespace adaption;
@@ -234,6 +269,57 @@ int adaption_lp_conv_fwd(const adaption_conv_shape* h_shape, adaption_qtensor x,
                               d_workspace, workspace_bytes, stream, g);
   if (rc != ADAPTION_OK) return rc;
   return dispatch(g, algo);
+}
+
+size_t adaption_lp_conv_pool_workspace_bytes(const adaption_conv_shape* h_shape, adaption_qfmt fx, adaption_qfmt fw,
+                                             adaption_qfmt fy, int64_t c_stride, int64_t y_c_stride, int32_t algo) {
+  if (h_shape == nullptr) return 0;
+  GemmProblem g;
+  adaption_qtensor x{}, w{}, y{};
+  x.fmt = fx; w.fmt = fw; y.fmt = fy;
+  x.c_stride = w.c_stride = c_stride;
+  y.c_stride = y_c_stride;
+  x.lo = w.lo = x.hi = w.hi = y.lo = reinterpret_cast<void*>(uintptr_t(256));
+  y.hi = fy.n_bits > 8 ? reinterpret_cast<void*>(uintptr_t(256)) : nullptr;
+  adaption_stats* fake_stats = reinterpret_cast<adaption_stats*>(uintptr_t(256));
+  if (build_conv_problem(h_shape, x, w, nullptr, 0, 0, ADAPTION_MODE_REQUANT, y, fake_stats, nullptr, 0, nullptr,
+                         g) != ADAPTION_OK)
+    return 0;
+  return plan_conv_pool(g, algo).total;
+}
+
+int adaption_lp_conv_pool_fwd(const adaption_conv_shape* h_shape, adaption_qtensor x, adaption_qtensor w,
+                              const int16_t* d_bias_q, int32_t bias_frac_bits, int32_t relu, int32_t algo,
+                              int32_t phases, adaption_qtensor y, adaption_stats* d_stats, void* d_workspace,
+                              size_t workspace_bytes, void* stream) {
+  GemmProblem g;
+  int rc = build_conv_problem(h_shape, x, w, d_bias_q, bias_frac_bits, relu, ADAPTION_MODE_REQUANT, y, d_stats,
+                              d_workspace, workspace_bytes, stream, g);
+  if (rc != ADAPTION_OK) return rc;
+  if (phases < 1 || phases > (ADAPTION_PHASE_CONV | ADAPTION_PHASE_POOL)) return ADAPTION_ERR_INVALID_ARG;
+  if (algo != ADAPTION_ALGO_AUTO && algo != ADAPTION_ALGO_TENSOR && algo != ADAPTION_ALGO_DIRECT)
+    return ADAPTION_ERR_INVALID_ARG;
+  if ((g.OH & 1) || (g.OW & 1)) return ADAPTION_ERR_INVALID_ARG;      // 2x2 windows need even sizes
+  if (g.M == 0) return ADAPTION_OK;
+  const ConvPoolPlan pl = plan_conv_pool(g, algo);
+  if (d_workspace == nullptr || workspace_bytes < pl.total) return ADAPTION_ERR_WORKSPACE;
+  if (!aligned16(d_workspace)) return ADAPTION_ERR_ALIGNMENT;
+  // temporary planes for the convolution's own (or half-pooled) output
+  uint8_t* ws = static_cast<uint8_t*>(d_workspace);
+  adaption_qtensor t = y;
+  t.q16 = nullptr;
+  t.lo = ws + pl.conv_ws;
+  t.hi = y.fmt.n_bits > 8 ? ws + pl.conv_ws + pl.plane : nullptr;
+  g.y = t;
+  g.workspace = ws;
+  g.workspace_bytes = pl.conv_ws;
+  g.pool_w = pl.fused;
+  if (phases & ADAPTION_PHASE_CONV) {
+    rc = dispatch(g, algo);
+    if (rc != ADAPTION_OK) return rc;
+  }
+  if (!(phases & ADAPTION_PHASE_POOL)) return ADAPTION_OK;
+  return maxpool_impl(t, h_shape->N, g.OH, g.OW, h_shape->K, y, reinterpret_cast<cudaStream_t>(stream), pl.fused);
 }
 
 size_t adaption_lp_ip_workspace_bytes(int64_t B, int64_t K, int64_t O, adaption_qfmt fx,

@@ -136,17 +136,22 @@ struct GemmProblem {
   void* workspace = nullptr;
   size_t workspace_bytes = 0;
   cudaStream_t stream = nullptr;
+  // Tensor-core path only: y receives max(row 2j, row 2j+1) of the layer's output as its row j (the
+  // horizontal half of a 2x2 max-pool; y then has M / 2 rows).  Counters still refer to all M rows.
+  bool pool_w = false;
 };
 
 int launch_direct(const GemmProblem& p);
 bool tensor_path_supported(const GemmProblem& p);
 size_t tensor_path_workspace(const GemmProblem& p);
 int launch_tensor(const GemmProblem& p);
+bool tensor_path_can_pool(const GemmProblem& p);   // whether launch_tensor takes `p` with pool_w set
 // Convolutions with at most 4 input channels whose taps fit one 32-byte row: gather the taps into
 // packed planes in the workspace and run the layer as an inner product on the tensor-core path.
 bool pack_taps_applicable(const GemmProblem& p);
 size_t pack_taps_workspace(const GemmProblem& p);
 int launch_pack_taps(const GemmProblem& p);
+bool pack_taps_can_pool(const GemmProblem& p);
 // bias/ReLU/requantize (or range) of an int64 accumulator matrix acc[M][ld] -> y
 int launch_finalize(const int64_t* acc, int64_t ld, const GemmProblem& p);
 

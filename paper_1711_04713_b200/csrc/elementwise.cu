@@ -375,9 +375,10 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const uint4* __restrict
                                                          uint4* __restrict__ out_hi,
                                                          uint4* __restrict__ out_lo,
                                                          int16_t* __restrict__ out_q16, int N, int H,
-                                                         int W, int64_t in_vecs, int64_t out_vecs) {
-  // in_vecs / out_vecs: 16-byte vectors per pixel (c_stride / 16)
-  const int OH = H / 2, OW = W / 2;
+                                                         int W, int kw, int64_t in_vecs, int64_t out_vecs) {
+  // in_vecs / out_vecs: 16-byte vectors per pixel (c_stride / 16).  kw = 2: 2x2 windows; kw = 1: the
+  // input is already the horizontal maximum of pixel pairs (W columns), only rows are paired.
+  const int OH = H / 2, OW = W / kw;
   const int64_t vecs = in_vecs < out_vecs ? in_vecs : out_vecs;
   const size_t total = (size_t)N * OH * OW * (size_t)out_vecs;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
@@ -391,19 +392,23 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const uint4* __restrict
     const int n = (int)(pix / OH);
     uint4 bh = make_uint4(0, 0, 0, 0), bl = make_uint4(0, 0, 0, 0);
     if (v < vecs) {
-      const size_t p00 = (((size_t)n * H + 2 * oh) * W + 2 * ow) * (size_t)in_vecs + (size_t)v;
-      const size_t offs[4] = {p00, p00 + (size_t)in_vecs, p00 + (size_t)W * in_vecs,
+      const size_t p00 = (((size_t)n * H + 2 * oh) * W + (size_t)kw * ow) * (size_t)in_vecs + (size_t)v;
+      const size_t offs[4] = {p00, p00 + (size_t)W * in_vecs, p00 + (size_t)in_vecs,
                               p00 + (size_t)W * in_vecs + (size_t)in_vecs};
+      const int ncand = 2 * kw;          // the two rows first, then (2x2 only) their right neighbours
       uint4 h[4], l[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        l[k] = __ldg(in_lo + offs[k]);
-        h[k] = two ? __ldg(in_hi + offs[k]) : make_uint4(0, 0, 0, 0);
+        if (k < ncand) {
+          l[k] = __ldg(in_lo + offs[k]);
+          h[k] = two ? __ldg(in_hi + offs[k]) : make_uint4(0, 0, 0, 0);
+        }
       }
       bh = h[0];
       bl = l[0];
 #pragma unroll
-      for (int k = 1; k < 4; ++k) max16(bh, bl, h[k], l[k], two);
+      for (int k = 1; k < 4; ++k)
+        if (k < ncand) max16(bh, bl, h[k], l[k], two);
     }
     out_lo[t] = bl;
     if (two) out_hi[t] = bh;
@@ -522,8 +527,9 @@ int measure_range_impl(const float* d_x, size_t numel, int32_t n_bits, float* d_
   return cuda_status(cudaGetLastError());
 }
 
+// half_pooled: x already holds the horizontal maxima (N x H x W/2 pixels); only rows are paired.
 int maxpool_impl(const adaption_qtensor& x, int32_t N, int32_t H, int32_t W, int32_t C,
-                 const adaption_qtensor& y, cudaStream_t stream) {
+                 const adaption_qtensor& y, cudaStream_t stream, bool half_pooled) {
   if (N < 0 || H < 0 || W < 0 || C < 0 || (H & 1) || (W & 1)) return ADAPTION_ERR_INVALID_ARG;
   int rc = check_qtensor_in(x, C);
   if (rc != ADAPTION_OK) return rc;
@@ -536,8 +542,8 @@ int maxpool_impl(const adaption_qtensor& x, int32_t N, int32_t H, int32_t W, int
   const int grid = stream_grid(total, 256, 8);
   maxpool2x2_kernel<<<grid, 256, 0, stream>>>(
       two ? reinterpret_cast<const uint4*>(x.hi) : nullptr, reinterpret_cast<const uint4*>(x.lo),
-      two ? reinterpret_cast<uint4*>(y.hi) : nullptr, reinterpret_cast<uint4*>(y.lo), y.q16, N, H, W,
-      x.c_stride / 16, y.c_stride / 16);
+      two ? reinterpret_cast<uint4*>(y.hi) : nullptr, reinterpret_cast<uint4*>(y.lo), y.q16, N, H,
+      half_pooled ? W / 2 : W, half_pooled ? 1 : 2, x.c_stride / 16, y.c_stride / 16);
   return cuda_status(cudaGetLastError());
 }
 

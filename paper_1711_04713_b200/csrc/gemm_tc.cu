@@ -80,6 +80,7 @@ struct TcParams {
   unsigned long long timeout_ns;
   // epilogue variants chosen on the host
   int fast_relu;              // launch the FAST kernel variant (paired 16-bit epilogue)
+  int pool_w;                 // store max(row 2j, row 2j+1) of the tile: half of a 2x2 max-pool (staged only)
   int epi_groups;             // 1, or 2: the epilogue warps form two groups that take alternate tiles
   int staged;                 // outputs leave through shared memory and bulk-tensor stores
   uint32_t stage_off;         // offset of the staging planes from the ring base
@@ -1108,7 +1109,18 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             requant8<NACC, false>(xa, bcol, p, row_ok, col, cnt, wq);
             requant8<NACC, false>(xb, bcol + 8, p, row_ok, col + 8, cnt, wq + 4);
           }
-          if (p.staged) {
+          if (p.staged && p.pool_w) {
+            // Horizontal half of a 2x2 max-pool: rows 2j and 2j+1 of the tile are neighbouring
+            // pixels of one image row (even width, tiles start at even rows) and sit in neighbouring
+            // lanes; the maximum of the packed 16-bit values is stored once, as row j.
+#pragma unroll
+            for (int j = 0; j < 8; ++j) wq[j] = max_s16x2(wq[j], __shfl_xor_sync(0xffffffffu, wq[j], 1));
+            if ((lane & 1) == 0) {
+              const uint32_t off = staged_offset(row >> 1, c0 >> 4, p.BN);
+              st_shared_v4(stage_lo + off, plane_lo(wq));
+              if (p.rq.out_planes == 2) st_shared_v4(stage_hi + off, plane_hi(wq));
+            }
+          } else if (p.staged) {
             const uint32_t off = staged_offset(row, c0 >> 4, p.BN);
             st_shared_v4(stage_lo + off, plane_lo(wq));
             if (p.rq.out_planes == 2) st_shared_v4(stage_hi + off, plane_hi(wq));
@@ -1123,7 +1135,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       if (p.staged) fence_async_shared();
       epi_bar_sync(group, gthreads);
       if (p.staged && store_leader) {
-        const int m_first = tc.m0 + (int)rank * kBM;
+        const int m_first = (tc.m0 + (int)rank * kBM) >> (p.pool_w ? 1 : 0);     // row of the stored tensor
         for (int sub = 0; sub * 128 < p.BN; ++sub) {
           const uint32_t so = (uint32_t)sub * (uint32_t)(kBM * 128);
           tma_store_2d(&map_y_lo, stage_lo + so, tc.n0 + sub * 128, m_first);
@@ -1562,6 +1574,12 @@ extern "C" __attribute__((visibility("default"))) int adaption_debug_timeline(lo
 
 bool tensor_path_supported(const GemmProblem& g) { return make_config(g).ok; }
 
+// The horizontal half of a 2x2 max-pool can ride on the staged stores of a requantizing layer.
+bool tensor_path_can_pool(const GemmProblem& g) {
+  const TcConfig c = make_config(g);
+  return c.ok && c.staged && g.M % 2 == 0;
+}
+
 size_t tensor_path_workspace(const GemmProblem& g) { return make_config(g).workspace_bytes; }
 
 int launch_tensor(const GemmProblem& g) {
@@ -1596,8 +1614,8 @@ int launch_tensor(const GemmProblem& g) {
     const void* planes[2] = {g.y.hi, g.y.lo};
     for (int i = 0; i < 2; ++i) {
       if (planes[i] == nullptr) continue;      // single-plane outputs have no high plane
-      if (!encode_tiled_2d(&maps[4 + i], planes[i], (uint64_t)g.y.c_stride, (uint64_t)g.M, (uint64_t)g.y.c_stride,
-                           (uint32_t)ybox, (uint32_t)kBM, yswz))
+      if (!encode_tiled_2d(&maps[4 + i], planes[i], (uint64_t)g.y.c_stride, (uint64_t)(g.pool_w ? g.M / 2 : g.M),
+                           (uint64_t)g.y.c_stride, (uint32_t)ybox, (uint32_t)(g.pool_w ? kBM / 2 : kBM), yswz))
         return ADAPTION_ERR_CUDA;
     }
   }
@@ -1628,6 +1646,8 @@ int launch_tensor(const GemmProblem& g) {
   } else {
     p.rq = RequantParams{0, g.relu ? 1 : 0, 0, 0, 1};
   }
+  if (g.pool_w && !(c.staged && g.M % 2 == 0)) return ADAPTION_ERR_UNSUPPORTED;
+  p.pool_w = g.pool_w ? 1 : 0;
   p.epi_groups = c.epi_groups;
   p.staged = c.staged ? 1 : 0;
   p.stage_off = c.stage_off;

@@ -174,6 +174,12 @@ bool pack_taps_applicable(const GemmProblem& g) {
 
 size_t pack_taps_workspace(const GemmProblem& g) { return layout_of(g).total; }
 
+// whether the packed inner product can store horizontal pair maxima (GemmProblem::pool_w)
+bool pack_taps_can_pool(const GemmProblem& g) {
+  uint8_t* fake = reinterpret_cast<uint8_t*>(uintptr_t(256));
+  return (g.OW & 1) == 0 && tensor_path_can_pool(packed_problem(g, fake));
+}
+
 int launch_pack_taps(const GemmProblem& g) {
   uint8_t* ws = static_cast<uint8_t*>(g.workspace);
   const GemmProblem q = packed_problem(g, ws);

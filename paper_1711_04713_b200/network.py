@@ -58,8 +58,9 @@ class _Layer:
 
 class LPNetwork:
     def __init__(self, params: list[dict], batch: int, in_hw: tuple[int, int], in_c: int, n_bits: int,
-                 algo: int = B.ALGO_AUTO, keep_q16: bool = False, device="cuda"):
+                 algo: int = B.ALGO_AUTO, keep_q16: bool = False, device="cuda", fuse_pool: bool = True):
         self.n_bits = n_bits
+        self.fuse_pool = fuse_pool
         self.algo = algo
         self.device = device
         self.batch = batch
@@ -182,6 +183,25 @@ class LPNetwork:
             L.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         return L.workspace
 
+    def fused_pool_after(self, i: int) -> bool:
+        """True where layer i is a convolution whose output only feeds the 2x2 max-pool after it, so
+        that inference may run the pair as one library call (the convolution's own output is then not
+        materialised in ``layers[i].y``)."""
+        if not self.fuse_pool or self.keep_q16 or i + 1 >= len(self.layers):
+            return False
+        L, P = self.layers[i], self.layers[i + 1]
+        return L.type == "conv" and P.type == "pool" and L.OH % 2 == 0 and L.OW % 2 == 0
+
+    def _run_conv_pool(self, L: _Layer, P: _Layer, x: B.QTensor, phases: int = 3) -> B.QTensor:
+        P.y.frac_bits = L.y.frac_bits
+        need = B.adaption_lp_conv_pool_workspace_bytes(L.shape, x.fmt(), L.w.fmt(), P.y.fmt(), x.c_stride,
+                                                       P.y.c_stride, self.algo)
+        if P.workspace is None or P.workspace.numel() < need:
+            P.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        B.adaption_lp_conv_pool_fwd(L.shape, x, L.w, L.b.q16, L.b.frac_bits, L.relu, self.algo, P.y, L.stats,
+                                    P.workspace, phases)
+        return P.y
+
     def _run_layer(self, L: _Layer, x: B.QTensor, mode: int) -> B.QTensor:
         if L.type == "pool":
             L.y.frac_bits = x.frac_bits
@@ -285,11 +305,19 @@ class LPNetwork:
             self.quantize_params(measure=False)
             launches += 2 * sum(1 for L in self.layers if L.type in ("conv", "ip"))
         a = self.xq
-        for L in self.layers:
-            a = self._run_layer(L, a, B.MODE_REQUANT)
+        i = 0
+        while i < len(self.layers):
+            L = self.layers[i]
+            if self.fused_pool_after(i):
+                a = self._run_conv_pool(L, self.layers[i + 1], a)
+                launches += 1
+                i += 1
+            else:
+                a = self._run_layer(L, a, B.MODE_REQUANT)
             launches += 1
             if L.workspace is not None and L.type != "pool":
-                launches += 1  # split-K finalize
+                launches += 1  # split-K finalize or tap packing
+            i += 1
         self.launches_per_forward = launches
         return a, launches
 

@@ -375,3 +375,54 @@ def test_auto_falls_back_to_direct_for_small_or_odd_pitch():
         B.adaption_lp_conv_fwd(B.conv_shape(1, 4, 4, 8, 4, 3, 3, 1, 1), x, w, None, 0, False, B.MODE_RANGE,
                                B.ALGO_TENSOR, None, B.new_stats(), None)
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ convolution + 2x2 max-pool
+POOL_CONV = [
+    # N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu
+    (2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True),     # pair tiles, fused horizontal maxima
+    (6, 20, 20, 64, 96, 3, 1, 1, 16, 16, 16, True),       # BK = 64, ragged N tile and M tail
+    (2, 30, 30, 256, 64, 3, 1, 1, 16, 16, 16, False),     # signed outputs (generic epilogue), BN = 64
+    (8, 32, 32, 3, 64, 3, 1, 1, 16, 16, 16, True),        # packed taps
+    (2, 24, 24, 128, 256, 3, 1, 1, 8, 8, 8, True),        # single pass, 256-column tiles
+    (1, 64, 64, 32, 16, 3, 1, 1, 16, 16, 8, True),        # BN = 32 > output pitch 16: direct stores, full temp
+    (2, 12, 12, 20, 50, 5, 2, 1, 16, 16, 16, True),       # plain integer kernel (odd pitch), full temp
+]
+
+
+@pytest.mark.parametrize("case", POOL_CONV)
+@pytest.mark.parametrize("with_q16", [False, True])
+def test_conv_with_fused_pool(case, with_q16):
+    """adaption_lp_conv_pool_fwd equals convolution, epilogue and 2x2 max-pool of the oracle; its
+    counters are those of the convolution's own output."""
+    N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu = case
+    rng = np.random.default_rng(sum(case))
+    cs = B.pad_to(Cin, 32) if Cin != 20 else 48
+    xq = _rand_q(rng, (N, H, W, Cin), nx, 0.4)
+    wq = _rand_q(rng, (K, R, R, Cin), nw)
+    bq = _rand_q(rng, (K,), nw)
+    fx, fw = nx - 3, nw - 1
+    acc = orc.conv_acc(xq, wq, (pad, pad), (stride, stride))
+    F = fx + fw
+    _, f_out = _pick_f_out(acc, bq, fw, F, relu, n_out)
+    conv_y, cnt = orc.epilogue(acc, bq, fw, F, relu, n_out, f_out)
+    want = orc.maxpool2x2(conv_y)
+    OH, OW = acc.shape[1], acc.shape[2]
+    x = to_qtensor(xq.reshape(-1, Cin), nx, fx, cs)
+    w = to_qtensor(wq.reshape(-1, Cin), nw, fw, cs)
+    y = B.QTensor.empty(N * (OH // 2) * (OW // 2), K, n_out, f_out, B.pad_to(K, 16), with_q16=with_q16)
+    y.lo.fill_(0x3C)
+    shp = B.conv_shape(N, H, W, Cin, K, R, R, pad, stride)
+    need = B.adaption_lp_conv_pool_workspace_bytes(shp, x.fmt(), w.fmt(), y.fmt(), cs, y.c_stride, B.ALGO_AUTO)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    st = B.new_stats()
+    B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st, ws)
+    assert B.read_stats(st).status == 0
+    assert np.array_equal(from_qtensor(y).reshape(want.shape), want)
+    if with_q16:
+        assert np.array_equal(q16_of(y).reshape(want.shape), want)
+    assert y.padding_is_zero()
+    assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+    with pytest.raises(B.AdaptionError):                      # too small a workspace is refused
+        B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st, ws[:need - 256])

@@ -175,29 +175,45 @@ def test_vgg16_full_batch_in_the_benchmark_configuration(n_bits, batch):
     x = wl.vgg16_input(batch, seed=0)
     sub = 2
     rec = orc.run_network(params, x[:sub], None, n_bits)
-    net = LPNetwork(params, batch, (224, 224), 3, n_bits)
     xd = dev(x.reshape(-1, 3))
-    net.set_formats(rec[0]["frac_bits"], [r["frac_bits"] for r in rec[1:] if r["type"] in ("conv", "ip")])
-    net.zero_stats()
-    out, _ = net.forward(xd)
-    torch.cuda.synchronize()
-    got_in = from_qtensor(net.xq)
-    assert np.array_equal(got_in[:sub * 224 * 224].reshape(rec[0]["y"].shape), rec[0]["y"])
-    for L, r in zip(net.layers, rec[1:]):
-        full = from_qtensor(L.y)
-        rows = full.shape[0] // batch * sub
-        assert np.array_equal(full[:rows].reshape(r["y"].shape), r["y"]), L.name
-        assert L.y.padding_is_zero(), L.name
-        if r["type"] in ("conv", "ip"):
-            assert L.w.frac_bits == r["w_frac_bits"], L.name
-            st = B.read_stats(L.stats)
-            assert int(st.status) == 0
-            assert int(st.zeros) == int((full == 0).sum()), L.name
-            qmax, qmin = (1 << (n_bits - 1)) - 1, -(1 << (n_bits - 1))
-            assert int(st.sat_pos) <= int((full == qmax).sum()) and int(st.sat_neg) <= int((full == qmin).sum())
-            if L.relu:
-                assert int(full.min()) >= 0 and int(st.sat_neg) == 0
-        del full
+    counters = {}
+    # first with every layer's output materialised, then as the benchmark runs it: a convolution
+    # whose output only feeds a pooling layer hands over pooled data and keeps no tensor of its own
+    for fuse_pool in (False, True):
+        net = LPNetwork(params, batch, (224, 224), 3, n_bits, fuse_pool=fuse_pool)
+        net.set_formats(rec[0]["frac_bits"], [r["frac_bits"] for r in rec[1:] if r["type"] in ("conv", "ip")])
+        net.zero_stats()
+        out, _ = net.forward(xd)
+        torch.cuda.synchronize()
+        got_in = from_qtensor(net.xq)
+        assert np.array_equal(got_in[:sub * 224 * 224].reshape(rec[0]["y"].shape), rec[0]["y"])
+        n_fused = 0
+        for i, (L, r) in enumerate(zip(net.layers, rec[1:])):
+            if r["type"] in ("conv", "ip"):
+                assert L.w.frac_bits == r["w_frac_bits"], L.name
+                st = B.read_stats(L.stats)
+                assert int(st.status) == 0
+                got = (int(st.zeros), int(st.sat_pos), int(st.sat_neg))
+            if net.fused_pool_after(i):
+                # counters are those of the convolution's own output: equal to the unfused run's
+                assert got == counters[L.name], L.name
+                n_fused += 1
+                continue
+            full = from_qtensor(L.y)
+            rows = full.shape[0] // batch * sub
+            assert np.array_equal(full[:rows].reshape(r["y"].shape), r["y"]), L.name
+            assert L.y.padding_is_zero(), L.name
+            if r["type"] in ("conv", "ip"):
+                counters.setdefault(L.name, got)
+                assert got == counters[L.name], L.name
+                assert got[0] == int((full == 0).sum()), L.name
+                qmax, qmin = (1 << (n_bits - 1)) - 1, -(1 << (n_bits - 1))
+                assert got[1] <= int((full == qmax).sum()) and got[2] <= int((full == qmin).sum())
+                if L.relu:
+                    assert int(full.min()) >= 0 and got[2] == 0
+            del full
+        assert n_fused == (5 if fuse_pool else 0)
+        del net
 
 
 @pytest.mark.parametrize("n_bits,seed", [(4, 0), (8, 1), (12, 2), (16, 3)])
