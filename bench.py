@@ -271,9 +271,10 @@ def run_gpu(args):
             i += 1
         return a
 
-    # kernels of ours per step: range (2) + input LPAct (1) + weight/bias quantize (2 per layer)
-    # + one per layer (+1 finalize where K is split)
-    launches_step = 3 + 2 * n_gemm + len(net.layers) + sum(1 for L in gemm_layers if L.workspace is not None)
+    # kernels of ours per step: range (2) + input LPAct (1) + weight/bias quantization (dense tensors
+    # batched into one launch) + one per layer (+1 finalize where K is split, +1 first-layer packing)
+    launches_step = (3 + net.param_quantize_launches() + len(net.layers) +
+                     sum(1 for L in gemm_layers if L.workspace is not None))
 
     sampler = ClockSampler(local_rank)
     if rank == 0:

@@ -116,6 +116,20 @@ ADAPTION_API int adaption_quantize(const float* d_x, size_t outer, size_t inner,
                       const adaption_qfmt* d_fmt, int32_t rounding, adaption_stats* d_stats,
                       void* stream);
 
+/* Sec. 2.1 (weights and biases are quantized anew in every forward pass): adaption_quantize with
+ * deterministic rounding and no counters for n_items tensors at once.  h_items is a HOST array,
+ * read before the call returns; each item means what the arguments of the same names mean to
+ * adaption_quantize (d_fmt may be NULL).  Dense tensors (inner == q.c_stride, d_x 16-byte aligned)
+ * share one kernel launch per 40 items; the others are quantized by launches of their own.  All
+ * items are validated before anything is launched; the tensors must not overlap. */
+typedef struct adaption_quantize_item {
+  const float* d_x;
+  int64_t outer, inner;
+  adaption_qtensor q;
+  const adaption_qfmt* d_fmt;
+} adaption_quantize_item;
+ADAPTION_API int adaption_quantize_batch(const adaption_quantize_item* h_items, int32_t n_items, void* stream);
+
 /* Sec. 2.4 (rounding_scheme STOCHASTIC).  As adaption_quantize (with the ReLU option of
  * adaption_lp_act), but x * 2^frac_bits = floor + frac is rounded up with probability
  * floor(frac * 2^32) / 2^32 and down otherwise, so that the expectation is the unrounded value and

@@ -33,6 +33,11 @@ class adaption_qtensor(C.Structure):
                 ("fmt", adaption_qfmt), ("c_stride", C.c_int64)]
 
 
+class adaption_quantize_item(C.Structure):
+    _fields_ = [("d_x", C.c_void_p), ("outer", C.c_int64), ("inner", C.c_int64), ("q", adaption_qtensor),
+                ("d_fmt", C.c_void_p)]
+
+
 class adaption_stats(C.Structure):
     _fields_ = [("zeros", C.c_uint64), ("sat_pos", C.c_uint64), ("sat_neg", C.c_uint64),
                 ("max_abs_acc", C.c_int64), ("status", C.c_int32), ("reserved", C.c_int32)]
@@ -52,6 +57,7 @@ EXPORTS = [
     "adaption_quantize_stochastic", "adaption_bit_histogram", "adaption_width_histogram",
     "adaption_choose_frac_bits_from_hist", "adaption_choose_frac_bits_from_widths",
     "adaption_lp_act_stochastic", "adaption_lp_conv_pool_workspace_bytes", "adaption_lp_conv_pool_fwd",
+    "adaption_quantize_batch",
 ]
 HIST_BINS = 17
 
@@ -83,6 +89,7 @@ def load(path: str | None = None):
     lib.adaption_lp_conv_workspace_bytes.restype = SZ
     lib.adaption_lp_conv_fwd.argtypes = [C.POINTER(adaption_conv_shape), adaption_qtensor, adaption_qtensor,
                                          P, I32, I32, I32, I32, adaption_qtensor, P, P, SZ, P]
+    lib.adaption_quantize_batch.argtypes = [C.POINTER(adaption_quantize_item), I32, P]
     lib.adaption_lp_conv_pool_workspace_bytes.argtypes = [C.POINTER(adaption_conv_shape), adaption_qfmt,
                                                           adaption_qfmt, adaption_qfmt, I64, I64, I32]
     lib.adaption_lp_conv_pool_workspace_bytes.restype = SZ
@@ -212,6 +219,20 @@ def adaption_quantize(x: torch.Tensor, outer: int, inner: int, out: QTensor,
                       d_stats: torch.Tensor | None = None):
     _check(load().adaption_quantize(_ptr(x), outer, inner, out.c_struct(), _ptr(d_fmt), rounding,
                                     _ptr(d_stats), _stream()), "adaption_quantize")
+
+
+def quantize_items(entries) -> "C.Array":
+    """Host array of adaption_quantize_item from (x, outer, inner, out, d_fmt or None) tuples."""
+    arr = (adaption_quantize_item * len(entries))()
+    for it, (x, outer, inner, out, d_fmt) in zip(arr, entries):
+        it.d_x, it.outer, it.inner, it.q, it.d_fmt = _ptr(x), outer, inner, out.c_struct(), _ptr(d_fmt)
+    return arr
+
+
+def adaption_quantize_batch(items, n_items: int | None = None):
+    """``items``: a ctypes array from quantize_items() (the tensors it names must stay alive)."""
+    n = len(items) if n_items is None else n_items
+    _check(load().adaption_quantize_batch(items, n, _stream()), "adaption_quantize_batch")
 
 
 def adaption_quantize_stochastic(x: torch.Tensor, outer: int, inner: int, out: QTensor, seed: int,

@@ -13,6 +13,7 @@ int cuda_failure(cudaError_t e, const char* where) {
 
 int quantize_impl(const float*, size_t, size_t, const adaption_qtensor&, const adaption_qfmt*, int32_t,
                   int32_t, adaption_stats*, cudaStream_t);
+int quantize_batch_impl(const adaption_quantize_item*, int32_t, cudaStream_t);
 int requant_impl(const adaption_qtensor&, size_t, size_t, int32_t, const adaption_qtensor&,
                  const adaption_qfmt*, int32_t, adaption_stats*, cudaStream_t);
 int measure_range_impl(const float*, size_t, int32_t, float*, adaption_qfmt*, cudaStream_t);
@@ -189,6 +190,10 @@ int adaption_quantize(const float* d_x, size_t outer, size_t inner, adaption_qte
                       void* stream) {
   return quantize_impl(d_x, outer, inner, out, d_fmt, 0, rounding, d_stats,
                        reinterpret_cast<cudaStream_t>(stream));
+}
+
+int adaption_quantize_batch(const adaption_quantize_item* h_items, int32_t n_items, void* stream) {
+  return quantize_batch_impl(h_items, n_items, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int adaption_quantize_stochastic(const float* d_x, size_t outer, size_t inner, adaption_qtensor out,

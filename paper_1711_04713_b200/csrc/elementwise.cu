@@ -303,6 +303,60 @@ __global__ void __launch_bounds__(256) requant_rows_kernel(const uint32_t* __res
 
 // Dense rows on both sides (pitch == inner extent, no int16 copy): the tensor is one flat array,
 // sixteen elements (one 16-byte vector per plane) per thread and step, no index arithmetic.
+// The kernel has to stay below about ten integer instructions per element to run at memory speed
+// (4 bytes of traffic per element), so bytes are gathered and scattered with byte permutes, the
+// rounding shift is v + h - (v < 0) >> s (equal to the half-away-from-zero form: for v < 0,
+// -((-v + h) >> s) = ceil((v - h) / 2^s) = floor((v + h - 1) / 2^s) with 2 h = 2^s), zeros are counted
+// on the packed output bytes and saturations only where a clamp changed something.
+__device__ __forceinline__ uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
+}
+
+// element b of a word pair: hi * 256 + lo with the sign of the high byte (or of the only byte)
+// replicated upwards (selector nibbles with bit 3 set copy the sign of the byte they name)
+template <bool TWO_PLANES_IN>
+__device__ __forceinline__ int32_t stored_value(uint32_t lw, uint32_t hw, int b) {
+  return TWO_PLANES_IN ? (int32_t)byte_perm(lw, hw, 0xCC40u + 0x1111u * b)
+                       : (int32_t)byte_perm(lw, 0u, 0x8880u + 0x1111u * b);
+}
+
+__device__ __forceinline__ int32_t requant_unclamped(int32_t v, const RequantParams& rq, int32_t half) {
+  if (rq.relu) v = max(v, 0);
+  return rq.shift > 0 ? (v + half + (v >> 31)) >> rq.shift : v * (1 << (-rq.shift));
+}
+
+template <bool TWO_PLANES_IN>
+__device__ __forceinline__ void requant_word(uint32_t lw, uint32_t hw, const RequantParams& rq, int32_t half,
+                                             Counts& c, uint32_t& out_lo, uint32_t& out_hi) {
+  int32_t q[4], clipped = 0;
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    const int32_t r = requant_unclamped(stored_value<TWO_PLANES_IN>(lw, hw, b), rq, half);
+    q[b] = min(max(r, rq.qmin), rq.qmax);
+    clipped |= r ^ q[b];
+  }
+  if (clipped != 0) {             // rare: count exactly
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int32_t r = requant_unclamped(stored_value<TWO_PLANES_IN>(lw, hw, b), rq, half);
+      c.sat_pos += (r > rq.qmax);
+      c.sat_neg += (r < rq.qmin);
+    }
+  }
+  const uint32_t p01 = byte_perm((uint32_t)q[0], (uint32_t)q[1], 0x5410u);   // two int16
+  const uint32_t p23 = byte_perm((uint32_t)q[2], (uint32_t)q[3], 0x5410u);
+  out_lo = byte_perm(p01, p23, 0x6420u);
+  out_hi = byte_perm(p01, p23, 0x7531u);
+  // zero elements: both bytes zero.  A byte of ((x & 0x7f7f7f7f) + 0x7f7f7f7f) | x has its top
+  // bit clear exactly where the byte of x is zero (no carry crosses a byte).
+  const uint32_t x = rq.out_planes == 2 ? (out_lo | out_hi) : out_lo;
+  const uint32_t nz = (((x & 0x7f7f7f7fu) + 0x7f7f7f7fu) | x) & 0x80808080u;
+  c.zeros += 4 - __popc(nz);
+}
+
+template <bool TWO_PLANES_IN>
 __global__ void __launch_bounds__(256) requant_flat_kernel(const uint4* __restrict__ in_hi,
                                                            const uint4* __restrict__ in_lo, size_t n16,
                                                            uint4* __restrict__ out_hi, uint4* __restrict__ out_lo,
@@ -311,31 +365,30 @@ __global__ void __launch_bounds__(256) requant_flat_kernel(const uint4* __restri
                                                            RequantParams rq, adaption_stats* __restrict__ stats) {
   if (d_fmt != nullptr) out_frac_bits = d_fmt->frac_bits;
   rq.shift = in_frac_bits - out_frac_bits;
+  const int32_t half = rq.shift > 0 ? 1 << (rq.shift - 1) : 0;
   Counts c;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += nthreads) {
-    const uint4 lo = __ldcs(in_lo + i);
-    const uint4 hi = in_hi != nullptr ? __ldcs(in_hi + i) : make_uint4(0, 0, 0, 0);
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  auto one = [&](size_t at, const uint4 lo, const uint4 hi) {
     const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
     uint32_t olo[4], ohi[4];
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      uint32_t pl = 0, ph = 0;
-#pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        const int32_t l = (lw[w] >> (8 * b)) & 255;
-        const int32_t v = in_hi != nullptr ? ((int32_t)(int8_t)((hw[w] >> (8 * b)) & 255)) * 256 + l
-                                           : (int32_t)(int8_t)l;
-        const int32_t q = requant_small(v, rq, true, c);
-        pl |= (uint32_t)(q & 255) << (8 * b);
-        ph |= (uint32_t)((q >> 8) & 255) << (8 * b);
-      }
-      olo[w] = pl;
-      ohi[w] = ph;
+    for (int w = 0; w < 4; ++w) requant_word<TWO_PLANES_IN>(lw[w], hw[w], rq, half, c, olo[w], ohi[w]);
+    __stcs(out_lo + at, make_uint4(olo[0], olo[1], olo[2], olo[3]));
+    if (rq.out_planes == 2) __stcs(out_hi + at, make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]));
+  };
+  for (; i + nthreads < n16; i += 2 * nthreads) {      // two vectors per plane in flight
+    const uint4 lo0 = __ldcs(in_lo + i), lo1 = __ldcs(in_lo + i + nthreads);
+    uint4 hi0 = make_uint4(0, 0, 0, 0), hi1 = hi0;
+    if (TWO_PLANES_IN) {
+      hi0 = __ldcs(in_hi + i);
+      hi1 = __ldcs(in_hi + i + nthreads);
     }
-    out_lo[i] = make_uint4(olo[0], olo[1], olo[2], olo[3]);
-    if (rq.out_planes == 2) out_hi[i] = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+    one(i, lo0, hi0);
+    one(i + nthreads, lo1, hi1);
   }
+  for (; i < n16; i += nthreads)
+    one(i, __ldcs(in_lo + i), TWO_PLANES_IN ? __ldcs(in_hi + i) : make_uint4(0, 0, 0, 0));
   if (stats != nullptr) flush_counts_warp(c, stats);
 }
 
@@ -480,6 +533,113 @@ int quantize_impl(const float* d_x, size_t outer, size_t inner, const adaption_q
   return cuda_status(cudaGetLastError());
 }
 
+// ------------------------------------------------------------------------------------------
+// Several dense tensors in one launch (the weights and biases of a whole network, quantized anew
+// in every forward pass): the tensors are cut into chunks of 1024 float4, numbered across the
+// batch; a block walks the chunks with the grid's stride and looks up the tensor a chunk belongs
+// to in the launch parameters (first_chunk is the running sum).  Per element the work is that of
+// quantize_flat_kernel.
+constexpr int kBatchItems = 40;
+constexpr int kBatchChunk4 = 1024;      // float4 per chunk: four per thread of a 256-thread block
+
+struct BatchItem {
+  const float4* x;
+  uint32_t* hi;
+  uint32_t* lo;
+  uint2* q16;
+  const adaption_qfmt* d_fmt;
+  unsigned long long n4;            // float4 in this tensor
+  unsigned long long first_chunk;   // chunks of the tensors before it
+  int32_t frac_bits, qmin, qmax, planes;
+};
+
+struct BatchArgs {
+  BatchItem item[kBatchItems];
+  unsigned long long total_chunks;
+  int32_t n;
+};
+
+__global__ void __launch_bounds__(256) quantize_batch_kernel(const __grid_constant__ BatchArgs a) {
+  Counts unused;
+  int t = 0;                       // chunks come in increasing order: the search only moves forward
+  for (unsigned long long chunk = blockIdx.x; chunk < a.total_chunks; chunk += gridDim.x) {
+    while (t + 1 < a.n && a.item[t + 1].first_chunk <= chunk) ++t;
+    const BatchItem& it = a.item[t];
+    const int32_t f = it.d_fmt != nullptr ? it.d_fmt->frac_bits : it.frac_bits;
+    const float scale = scale_of(f);
+    QuantOut o;
+    o.hi = it.hi; o.lo = it.lo; o.q16 = it.q16; o.planes = it.planes;
+    const unsigned long long base = (chunk - it.first_chunk) * kBatchChunk4 + threadIdx.x;
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const unsigned long long i = base + u * 256;
+      v[u] = i < it.n4 ? __ldcs(it.x + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const unsigned long long i = base + u * 256;
+      if (i < it.n4) {
+        int32_t q[4];
+        quantize_f32x4(v[u], scale, 0, it.qmin, it.qmax, unused, q);
+        store4(o, (size_t)i, q[0], q[1], q[2], q[3]);
+      }
+    }
+  }
+}
+
+int quantize_batch_impl(const adaption_quantize_item* h_items, int32_t n_items, cudaStream_t stream) {
+  if (n_items < 0 || (n_items > 0 && h_items == nullptr)) return ADAPTION_ERR_INVALID_ARG;
+  // validate everything before the first launch
+  for (int32_t k = 0; k < n_items; ++k) {
+    const adaption_quantize_item& h = h_items[k];
+    if (h.outer < 0 || h.inner < 0) return ADAPTION_ERR_INVALID_ARG;
+    int rc = check_qtensor_out(h.q, h.inner);
+    if (rc != ADAPTION_OK) return rc;
+    if (h.outer == 0 || h.inner == 0) continue;
+    if (h.d_x == nullptr) return ADAPTION_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(h.d_x) & 3u) != 0) return ADAPTION_ERR_ALIGNMENT;
+  }
+  BatchArgs args;
+  args.n = 0;
+  args.total_chunks = 0;
+  auto flush = [&]() -> int {
+    if (args.n == 0) return ADAPTION_OK;
+    const int grid = stream_grid((size_t)args.total_chunks, 1, 8);
+    quantize_batch_kernel<<<grid, 256, 0, stream>>>(args);
+    args.n = 0;
+    args.total_chunks = 0;
+    return cuda_status(cudaGetLastError());
+  };
+  for (int32_t k = 0; k < n_items; ++k) {
+    const adaption_quantize_item& h = h_items[k];
+    if (h.outer == 0 || h.inner == 0) continue;
+    const bool dense = h.inner == h.q.c_stride && aligned16(h.d_x);
+    if (!dense) {               // padded rows: the row kernel, on its own
+      int rc = quantize_impl(h.d_x, (size_t)h.outer, (size_t)h.inner, h.q, h.d_fmt, 0,
+                             ADAPTION_ROUND_DETERMINISTIC, nullptr, stream);
+      if (rc != ADAPTION_OK) return rc;
+      continue;
+    }
+    BatchItem& it = args.item[args.n];
+    const QuantOut qo = quant_out_of(h.q);
+    it.x = reinterpret_cast<const float4*>(h.d_x);
+    it.hi = qo.hi; it.lo = qo.lo; it.q16 = qo.q16; it.planes = qo.planes;
+    it.d_fmt = h.d_fmt;
+    it.n4 = (unsigned long long)h.outer * (unsigned long long)h.inner / 4;   // c_stride is a multiple of 16
+    it.first_chunk = args.total_chunks;
+    it.frac_bits = h.q.fmt.frac_bits;
+    it.qmin = -(1 << (h.q.fmt.n_bits - 1));
+    it.qmax = (1 << (h.q.fmt.n_bits - 1)) - 1;
+    args.total_chunks += (it.n4 + kBatchChunk4 - 1) / kBatchChunk4;
+    if (++args.n == kBatchItems) {
+      int rc = flush();
+      if (rc != ADAPTION_OK) return rc;
+    }
+  }
+  return flush();
+}
+
 int requant_impl(const adaption_qtensor& in, size_t outer, size_t inner, int32_t relu,
                  const adaption_qtensor& out, const adaption_qfmt* d_fmt, int32_t rounding,
                  adaption_stats* d_stats, cudaStream_t stream) {
@@ -493,10 +653,16 @@ int requant_impl(const adaption_qtensor& in, size_t outer, size_t inner, int32_t
   RequantParams rq = make_requant(in.fmt.frac_bits, out.fmt, relu);
   if ((int64_t)inner == in.c_stride && in.c_stride == out.c_stride && out.q16 == nullptr) {
     const size_t n16 = outer * inner / 16;
-    requant_flat_kernel<<<stream_grid(n16, 256, 8), 256, 0, stream>>>(
-        in.fmt.n_bits > 8 ? reinterpret_cast<const uint4*>(in.hi) : nullptr,
-        reinterpret_cast<const uint4*>(in.lo), n16, reinterpret_cast<uint4*>(out.hi),
-        reinterpret_cast<uint4*>(out.lo), in.fmt.frac_bits, out.fmt.frac_bits, d_fmt, rq, d_stats);
+    const int grid = stream_grid((n16 + 1) / 2, 256, 8);
+    if (in.fmt.n_bits > 8)
+      requant_flat_kernel<true><<<grid, 256, 0, stream>>>(
+          reinterpret_cast<const uint4*>(in.hi), reinterpret_cast<const uint4*>(in.lo), n16,
+          reinterpret_cast<uint4*>(out.hi), reinterpret_cast<uint4*>(out.lo), in.fmt.frac_bits,
+          out.fmt.frac_bits, d_fmt, rq, d_stats);
+    else
+      requant_flat_kernel<false><<<grid, 256, 0, stream>>>(
+          nullptr, reinterpret_cast<const uint4*>(in.lo), n16, reinterpret_cast<uint4*>(out.hi),
+          reinterpret_cast<uint4*>(out.lo), in.fmt.frac_bits, out.fmt.frac_bits, d_fmt, rq, d_stats);
     return cuda_status(cudaGetLastError());
   }
   const size_t groups = outer * (size_t)(out.c_stride / 4);

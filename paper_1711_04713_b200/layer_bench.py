@@ -3,7 +3,7 @@
     python -m paper_1711_04713_b200.layer_bench conv --N 8 --H 28 --C 512 --K 512 --R 3 --n-bits 16
     python -m paper_1711_04713_b200.layer_bench ip --B 64 --Kin 25088 --O 4096
     python -m paper_1711_04713_b200.layer_bench quantize --numel 268435456
-    python -m paper_1711_04713_b200.layer_bench range|act|pool|hist|squantize ...
+    python -m paper_1711_04713_b200.layer_bench range|act|pool|hist|squantize|params ...
 
 Prints one JSON line with the CUDA-event time per call and the achieved rate (logical TOPS for
 the layers, algorithmic GB/s for the streaming kernels).  Inputs are seeded synthetic tensors
@@ -154,6 +154,20 @@ def bench_stream(a) -> dict:
             "algorithmic_bytes": bytes_}
 
 
+def bench_params(a) -> dict:
+    """All weight and bias tensors of VGG16 (138 M parameters) quantized with fixed formats, as every
+    forward pass does: one adaption_quantize_batch call."""
+    from . import workloads as wl
+    from .network import LPNetwork
+    net = LPNetwork(wl.make_params(wl.vgg16_specs(), seed=a.seed), 1, (224, 224), 3, a.n_bits)
+    net.quantize_params(measure=True)
+    ms = _time(lambda: net.quantize_params(measure=False), a.iters)
+    n = sum(L.w_f32.numel() + L.b_f32.numel() for L in net.layers if L.type in ("conv", "ip"))
+    bytes_ = n * (4 + (2 if a.n_bits > 8 else 1))
+    return {"kind": "params", "numel": n, "n_bits": a.n_bits, "ms": ms, "gbs": bytes_ / (ms / 1e3) / 1e9,
+            "algorithmic_bytes": bytes_, "launches": net.param_quantize_launches()}
+
+
 def bench_peak(a) -> dict:
     """Back-to-back int8 tensor-core instructions on resident operands (the roofline denominator)."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
@@ -182,7 +196,7 @@ def bench_peak(a) -> dict:
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["conv", "ip", "range", "quantize", "act", "requant", "pool", "peak", "hist", "squantize"])
+    ap.add_argument("kind", choices=["conv", "ip", "range", "quantize", "act", "requant", "pool", "peak", "hist", "squantize", "params"])
     ap.add_argument("--N", type=int, default=8)
     ap.add_argument("--H", type=int, default=28)
     ap.add_argument("--C", type=int, default=512)
@@ -210,6 +224,8 @@ def main():
         out = bench_ip(a)
     elif a.kind == "peak":
         out = bench_peak(a)
+    elif a.kind == "params":
+        out = bench_params(a)
     else:
         out = bench_stream(a)
     print(json.dumps(out), flush=True)

@@ -148,6 +148,15 @@ class LPNetwork:
         """Weights and biases -> fixed point (paper Sec. 2.1: quantized in the forward pass).  With
         ``measure`` the decimal point of each layer's weights is taken from max|w| on the device, or,
         with ``threshold`` > 0, from the thresholded allocation of Sec. 2.3."""
+        if not measure:
+            # fixed formats: every weight and bias tensor of the network in one library call
+            entries = []
+            for L in self.layers:
+                if L.type in ("conv", "ip"):
+                    entries.append((L.w_f32, L.w.outer, L.w.inner, L.w, None))
+                    entries.append((L.b_f32, 1, L.K, L.b, None))
+            B.adaption_quantize_batch(B.quantize_items(entries))
+            return
         for L in self.layers:
             if L.type not in ("conv", "ip"):
                 continue
@@ -161,15 +170,24 @@ class LPNetwork:
                 B.adaption_measure_range(L.w_f32, self.n_bits, L.w_max_dev, L.w_fmt_dev)
                 B.adaption_quantize(L.w_f32, L.w.outer, L.w.inner, L.w, L.w_fmt_dev)
                 B.adaption_quantize(L.b_f32, 1, L.K, L.b, L.w_fmt_dev)
-            else:
-                B.adaption_quantize(L.w_f32, L.w.outer, L.w.inner, L.w)
-                B.adaption_quantize(L.b_f32, 1, L.K, L.b)
-        if measure:
-            for L in self.layers:
-                if L.type in ("conv", "ip"):
-                    f = int(L.w_fmt_dev.cpu()[1])
-                    L.w.frac_bits = f
-                    L.b.frac_bits = f
+        for L in self.layers:
+            if L.type in ("conv", "ip"):
+                f = int(L.w_fmt_dev.cpu()[1])
+                L.w.frac_bits = f
+                L.b.frac_bits = f
+
+    def param_quantize_launches(self) -> int:
+        """Kernel launches of one quantize_params(measure=False): dense tensors share one launch per
+        40, a tensor with padded rows takes one of its own."""
+        dense = padded = 0
+        for L in self.layers:
+            if L.type in ("conv", "ip"):
+                for q in (L.w, L.b):
+                    if q.inner == q.c_stride:
+                        dense += 1
+                    else:
+                        padded += 1
+        return (dense + 39) // 40 + padded
 
     # ------------------------------------------------------------------ one layer
     def _workspace(self, L: _Layer, x: B.QTensor) -> torch.Tensor | None:
@@ -303,7 +321,7 @@ class LPNetwork:
         launches += 1
         if requantize_params:
             self.quantize_params(measure=False)
-            launches += 2 * sum(1 for L in self.layers if L.type in ("conv", "ip"))
+            launches += self.param_quantize_launches()
         a = self.xq
         i = 0
         while i < len(self.layers):

@@ -31,6 +31,7 @@ def test_struct_layouts_match_header():
     assert ctypes.sizeof(B.adaption_qtensor) == 40
     assert ctypes.sizeof(B.adaption_stats) == 40
     assert ctypes.sizeof(B.adaption_conv_shape) == 44
+    assert ctypes.sizeof(B.adaption_quantize_item) == 72
 
 
 def test_status_strings(lib):
@@ -71,6 +72,13 @@ def test_host_side_argument_errors_need_no_gpu(lib):
     assert lib.adaption_maxpool2x2(good, 1, 3, 4, 16, good, None) == B.ERR_INVALID_ARG  # odd H
     # zero-sized work is accepted without touching memory
     assert lib.adaption_quantize(None, 0, 16, good, None, 0, None, None) == B.OK
+    items = (B.adaption_quantize_item * 2)()
+    items[0].d_x, items[0].outer, items[0].inner, items[0].q = None, 0, 16, good
+    items[1].d_x, items[1].outer, items[1].inner, items[1].q = fake, 4, 16, bad_fmt
+    assert lib.adaption_quantize_batch(items, 1, None) == B.OK              # only the empty tensor
+    assert lib.adaption_quantize_batch(items, 2, None) == B.ERR_INVALID_ARG  # validated before any launch
+    assert lib.adaption_quantize_batch(None, 1, None) == B.ERR_INVALID_ARG
+    assert lib.adaption_quantize_batch(None, 0, None) == B.OK
 
 
 def test_workspace_queries(lib):

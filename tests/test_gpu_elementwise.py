@@ -157,6 +157,30 @@ def test_lp_act_format_change(n_in, f_in, n_out, f_out, relu):
     assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
 
 
+@pytest.mark.parametrize("n_in,f_in,n_out,f_out,relu", [
+    (16, 15, 16, 0, False), (16, 15, 16, 14, False), (16, 10, 16, 9, True), (16, 10, 8, 3, False),
+    (16, 3, 16, 12, False), (16, 0, 16, 15, True), (16, 8, 5, 2, False), (16, 7, 16, 7, False),
+    (8, 4, 16, 12, True), (8, 7, 8, 0, False), (8, 0, 16, 15, False), (8, 3, 4, 1, True)])
+def test_lp_act_format_change_dense_every_input_value(n_in, f_in, n_out, f_out, relu):
+    """Dense tensors (pitch == extent, planes only) take the flat kernel: every representable
+    input value, in a tensor long enough for the paired and the tail loop, a full-size grid
+    included."""
+    lo, hi = -(1 << (n_in - 1)), 1 << (n_in - 1)
+    vals = np.arange(lo, hi, dtype=np.int64)
+    reps = 65536 // vals.size
+    for rows_mult in (1, 37):
+        q = np.tile(vals, reps * rows_mult + 1)[: (65536 * rows_mult // 48 + 1) * 48]
+        q = q.reshape(-1, 48).astype(np.int16)
+        xin = to_qtensor(q, n_in, f_in, 48)
+        out = B.QTensor.empty(q.shape[0], 48, n_out, f_out, 48)
+        out.lo.fill_(0x77)
+        st = B.new_stats()
+        B.adaption_lp_act(None, xin, q.shape[0], 48, relu, out, None, B.ROUND_DETERMINISTIC, st)
+        want, cnt = orc.requantize(q, f_in, relu, n_out, f_out)
+        assert np.array_equal(from_qtensor(out), want)
+        assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+
+
 @pytest.mark.parametrize("n_bits", [16, 8])
 @pytest.mark.parametrize("shape", [(2, 6, 8, 3), (1, 4, 4, 64), (3, 10, 6, 20), (2, 2, 2, 130)])
 def test_maxpool(n_bits, shape):
@@ -181,3 +205,52 @@ def test_empty_inputs_are_no_ops():
     B.adaption_quantize(torch.empty(0, device="cuda"), 0, 16, out)
     torch.cuda.synchronize()
     assert int(out.lo[0]) == 9
+
+
+def test_quantize_batch_matches_oracle():
+    """Many tensors in one call: mixed sizes (below, at and above a 1024-vector chunk), 16- and 8-bit
+    outputs, with and without the int16 copy, host- and device-side formats, padded rows, an empty
+    tensor, and more dense tensors than one launch carries; every element against the oracle."""
+    rng = np.random.default_rng(77)
+    shapes = [(64, 64), (1, 16), (4096, 16), (4097, 16), (300, 1024), (3, 48), (27, 3), (1, 1000), (0, 16), (1, 64)]
+    shapes += [(rng.integers(1, 40), 16 * int(rng.integers(1, 9))) for _ in range(45)]
+    entries, checks, keep = [], [], []
+    for k, (outer, inner) in enumerate(shapes):
+        outer, inner = int(outer), int(inner)
+        n_bits = 8 if k % 3 == 1 else 16
+        frac_bits = n_bits - 1 - (k % 3)
+        x = (rng.standard_normal((outer, inner)) * 2.0 ** (k % 3) * 0.6).astype(np.float32)
+        if x.size:
+            x.ravel()[0] = np.nan
+            x.ravel()[-1] = np.inf
+        cs = B.pad_to(inner, 16)
+        use_dev_fmt = k % 4 == 2
+        out = B.QTensor.empty(max(outer, 1), inner, n_bits, 0 if use_dev_fmt else frac_bits, cs,
+                              with_q16=(k % 2 == 0))
+        out.lo.fill_(0xAB)
+        if outer == 0:                                     # an empty tensor leaves its output alone
+            entries.append((None, 0, inner, out, None))
+            continue
+        fmt = torch.tensor([n_bits, frac_bits], dtype=torch.int32, device="cuda") if use_dev_fmt else None
+        xd = dev(x)
+        keep.append((xd, fmt))
+        entries.append((xd, outer, inner, out, fmt))
+        checks.append((x, out, n_bits, frac_bits))
+    items = B.quantize_items(entries)
+    B.adaption_quantize_batch(items)
+    torch.cuda.synchronize()
+    for x, out, n_bits, frac_bits in checks:
+        want, _ = orc.quantize(x, n_bits, frac_bits)
+        assert np.array_equal(from_qtensor(out), want), x.shape
+        if out.q16 is not None:
+            assert np.array_equal(q16_of(out), want)
+        assert out.padding_is_zero()
+    B.adaption_quantize_batch(items, 0)                   # nothing to do
+    # one bad item: nothing is launched, the others stay untouched
+    checks[0][1].lo.fill_(0x11)
+    bad = B.QTensor.empty(4, 16, 16, 3, 16)
+    bad.n_bits = 17
+    with pytest.raises(B.AdaptionError):
+        B.adaption_quantize_batch(B.quantize_items(entries[:1] + [(keep[0][0], 4, 16, bad, None)]))
+    torch.cuda.synchronize()
+    assert int(checks[0][1].lo.min()) == 0x11 and int(checks[0][1].lo.max()) == 0x11
