@@ -492,6 +492,8 @@ __device__ __forceinline__ int32_t mad_lo(int32_t a, int32_t b, int32_t c) {
 template <int NACC, bool WIDE>
 __device__ __forceinline__ int32_t shifted32(int32_t x0, int32_t x1, int32_t x2, int2 c, int shift) {
   // name the accumulators by weight: hh (2^16), mid (2^8), ll (1)
+  // a single accumulator (8-bit operands) is the whole sum: one 32-bit add, any shift >= 0
+  if (NACC == 1) return (x0 + mad_lo(c.y, 65536, c.x)) >> shift;
   const int32_t hh = NACC == 3 ? x0 : 0;
   const int32_t mid = NACC == 3 ? x1 : (NACC == 2 ? x0 : 0);
   const int32_t ll = NACC == 3 ? x2 : (NACC == 2 ? x1 : x0);
@@ -709,7 +711,8 @@ __device__ __forceinline__ bool epi_bar_all(int group, int threads, bool pred) {
 // ---------------------------------------------------------------------------------- kernel
 // GROUPED: stages hold several k-blocks and / or the weights are resident in shared memory (short
 // reductions); the plain variant keeps the issue loops free of that bookkeeping.
-// FAST: ReLU layer in requantizing mode whose shift lies in [9, 31], N a multiple of 8, no split-K,
+// FAST: ReLU layer in requantizing mode whose shift lies in [9, 31] ([0, 31] with 8-bit operands
+// on both sides), N a multiple of 8, no split-K,
 // magnitudes within the 32-bit bounds of the fast epilogue: it then contains only that path.
 // 20 warps: one block per SM, 96 registers per thread.
 template <int NAX, int NBW, bool PAIR, bool GROUPED, bool FAST>
@@ -1045,7 +1048,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           long long b = 0;
           if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
           if (FAST) {
-            const long long C = b + (1ll << (p.rq.shift - 1));
+            const long long C = b + (p.rq.shift > 0 ? 1ll << (p.rq.shift - 1) : 0ll);
             reinterpret_cast<int2*>(colconst)[c] = make_int2((int)(C & 0xffff), (int)(C >> 16));
           } else {
             colconst[c] = b;
@@ -1652,17 +1655,22 @@ int launch_tensor(const GemmProblem& g) {
   p.staged = c.staged ? 1 : 0;
   p.stage_off = c.stage_off;
   p.const_off = c.stage_off + c.stage_out_bytes;
-  if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && p.rq.shift >= 9 && p.rq.shift <= 31 &&
-      g.N % 8 == 0 && env_int("ADAPTION_TC_FAST", 1) != 0) {
+  const bool single = c.nacc == 1;
+  if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && p.rq.shift >= (single ? 0 : 9) &&
+      p.rq.shift <= 31 && g.N % 8 == 0 && env_int("ADAPTION_TC_FAST", 1) != 0) {
     // 32-bit bounds of the fast epilogue (see shifted32): with a reduction of kred bytes per plane row
     // |hh| <= kred 2^14, |mid| <= kred 65280, |ll| <= kred 65025, and |C| < 2^(15 + bias_shift) + 2^(shift-1)
     const long long kred = (long long)c.num_kb * c.BK;
-    const long long cmax = (g.bias != nullptr ? (1ll << (15 + g.bias_shift)) : 0ll) + (1ll << (p.rq.shift - 1));
+    const long long cmax = (g.bias != nullptr ? (1ll << (15 + g.bias_shift)) : 0ll) +
+                           (p.rq.shift > 0 ? 1ll << (p.rq.shift - 1) : 0ll);
     const long long hmax = kred * 16384 + (cmax >> 16) + 1;
     const long long tmax = kred * 65280 + ((kred * 65025 + 65535) >> 8) + 1;
     const long long lim = 1ll << 31;
     bool ok32 = kred * 65025 + 65535 < lim && tmax < lim && hmax + (tmax >> 8) + 1 < lim;
-    if (p.rq.shift < 16) ok32 = ok32 && (hmax << (16 - p.rq.shift)) + (tmax >> (p.rq.shift - 8)) + 1 < lim;
+    if (p.rq.shift < 16 && !single)
+      ok32 = ok32 && (hmax << (16 - p.rq.shift)) + (tmax >> (p.rq.shift - 8)) + 1 < lim;
+    // single accumulator: s8 x s8 products only, the constant added in full
+    if (single) ok32 = kred * 16384 + cmax < lim;
     p.fast_relu = ok32 ? 1 : 0;
   }
   p.ws = (long long*)g.workspace; p.ws_ld = g.N;

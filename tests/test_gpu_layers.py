@@ -206,6 +206,23 @@ def test_fast_epilogue_shifts_and_saturation(shift, n_out, cta_mode):
         assert cnt.sat_pos > 0   # the case does exercise saturation
 
 
+@pytest.mark.parametrize("shift", [0, 1, 3, 6, 8, 9, 11, 14])
+@pytest.mark.parametrize("n_out", [8, 5])
+@pytest.mark.parametrize("K,Cin", [(128, 128), (256, 512)])
+def test_single_pass_fast_epilogue_every_shift(shift, n_out, K, Cin, cta_mode):
+    """8-bit operands on both sides give one accumulator: ReLU layers take the 32-bit epilogue at
+    every non-negative shift (128- and 256-column tiles); magnitudes chosen so that outputs span
+    the range and some saturate."""
+    fmts = (shift // 2, shift - shift // 2)
+    f_out = 0
+    bits = 3 if shift <= 3 else (5 if shift <= 8 else 8)
+    cnt = run_conv_case(np.random.default_rng(300 + shift + K), 2, 24, 24, Cin, K, 3, 1, 1, 8, 8, n_out, True,
+                        B.ALGO_TENSOR, f_out=f_out, with_q16=False, mag_bits=(bits, bits), fmts=fmts)
+    assert cnt.zeros > 0
+    if n_out == 5:
+        assert cnt.sat_pos > 0   # the case does exercise saturation
+
+
 def test_epilogue_variants_agree(monkeypatch):
     """Cross-path identity: the generic 64-bit epilogue with direct stores, the staged stores and the
     fast paired path all give the oracle's bits on the same case."""
