@@ -33,8 +33,8 @@ NOMINAL_INT8_OVER_BF16 = 2.0        # nominal dense INT8 : bf16 ratio (4.5 : 2.2
 # DRAM traffic of the layer GEMM per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged
 # over the 16 layer launches of a forward pass of this workload), from the ncu launch list summarised
 # in profiles/bench_vgg16_b64_launch_list.md.  Valid only for the kernel source it was taken on.
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = 159.1e6
-GEMM_TRAFFIC_SOURCE_SHA1 = "8a37371e54e5"
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 159.8e6
+GEMM_TRAFFIC_SOURCE_SHA1 = "c68c4a1720c1"
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_BF16_SUSTAINED = 1400.0
 
@@ -272,9 +272,9 @@ def run_gpu(args):
         return a
 
     # kernels of ours per step: range (2) + input LPAct (1) + weight/bias quantization (dense tensors
-    # batched into one launch) + one per layer (+1 finalize where K is split, +1 first-layer packing)
+    # batched into one launch) + one per layer (+1 finalize where K is split, +2 first-layer tap packing)
     launches_step = (3 + net.param_quantize_launches() + len(net.layers) +
-                     sum(1 for L in gemm_layers if L.workspace is not None))
+                     sum(net.helper_launches(L) for L in gemm_layers))
 
     sampler = ClockSampler(local_rank)
     if rank == 0:

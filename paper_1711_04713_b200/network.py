@@ -176,6 +176,14 @@ class LPNetwork:
                 L.w.frac_bits = f
                 L.b.frac_bits = f
 
+    @staticmethod
+    def helper_launches(L: _Layer) -> int:
+        """Launches beside the layer's own kernel when it runs with a workspace: the tap packing of a
+        first layer with at most 4 channels (activations, weights), else the split-K finalize."""
+        if L.workspace is None:
+            return 0
+        return 2 if L.type == "conv" and L.C <= 4 else 1
+
     def param_quantize_launches(self) -> int:
         """Kernel launches of one quantize_params(measure=False): dense tensors share one launch per
         40, a tensor with padded rows takes one of its own."""
@@ -334,7 +342,7 @@ class LPNetwork:
                 a = self._run_layer(L, a, B.MODE_REQUANT)
             launches += 1
             if L.workspace is not None and L.type != "pool":
-                launches += 1  # split-K finalize or tap packing
+                launches += self.helper_launches(L)
             i += 1
         self.launches_per_forward = launches
         return a, launches
