@@ -42,6 +42,26 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
   return o;
 }
 
+// floor(y) plus one where the draw falls below T = floor(frac(y) 2^32), y = x 2^f, from
+// single-precision and 32-bit integer steps only; every step is exact:
+//   y = x * 2^f never rounds (f >= 0; an overflow gives +-Inf, which the clamp to a little outside
+//   the output range absorbs: beyond it only saturation matters; NaN counts as 0);
+//   a = |y| < 2^16, fa = a - floor(a) is exact (a multiple of ulp(a) below 1, or a itself) and so is
+//   t = fa 2^32 < 2^32;
+//   y >= 0: floor(y) = floor(a), T = floor(t);
+//   y <  0: floor(y) = -floor(a) - [fa > 0], frac = 1 - fa, T = 2^32 - ceil(t) (0 when fa = 0),
+//           which is 0 - ceil(t) in 32-bit arithmetic.
+__device__ __forceinline__ int32_t stochastic_round(float x, float scale, float y_lo, float y_hi, uint32_t draw) {
+  const float y = (x != x) ? 0.0f : fminf(fmaxf(x * scale, y_lo), y_hi);
+  const float a = fabsf(y);
+  const float fl = floorf(a);
+  const float t = (a - fl) * 4294967296.0f;
+  const int32_t ia = __float2int_rz(fl);
+  if (y >= 0.0f) return ia + (draw < __float2uint_rd(t) ? 1 : 0);
+  const uint32_t up = __float2uint_ru(t);
+  return -ia - (up != 0u ? 1 : 0) + (draw < 0u - up ? 1 : 0);
+}
+
 struct Out {
   uint4* hi;      // sixteen bytes per group of sixteen stored channels
   uint4* lo;
@@ -50,9 +70,7 @@ struct Out {
 };
 
 // One thread per group of sixteen stored channels of one row (padding channels receive zeros and
-// are neither drawn for nor counted).  floor(y * 2^32), clamped a little outside the output range
-// (beyond it only saturation matters), is taken with one rounding-down conversion of an exact
-// double product: its high word is floor(y), its low word is T.
+// are neither drawn for nor counted).
 __global__ void __launch_bounds__(256) quantize_stochastic_kernel(const float* __restrict__ x, size_t outer,
                                                                   int64_t inner, int64_t c_stride, Out out,
                                                                   int32_t frac_bits,
@@ -60,8 +78,8 @@ __global__ void __launch_bounds__(256) quantize_stochastic_kernel(const float* _
                                                                   int32_t qmin, int32_t qmax, uint32_t key0,
                                                                   uint32_t key1, adaption_stats* __restrict__ stats) {
   if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
-  const double scale = __longlong_as_double((long long)(1023 + 32 + frac_bits) << 52);   // 2^(frac_bits + 32)
-  const double y_lo = ((double)qmin - 2.0) * 4294967296.0, y_hi = ((double)qmax + 2.0) * 4294967296.0;
+  const float scale = __int_as_float((127 + frac_bits) << 23);   // 2^frac_bits
+  const float y_lo = (float)qmin - 2.0f, y_hi = (float)qmax + 2.0f;
   Counts c;
   const int64_t groups_per_row = c_stride / 16;
   const size_t total = outer * (size_t)groups_per_row;
@@ -91,10 +109,7 @@ __global__ void __launch_bounds__(256) quantize_stochastic_kernel(const float* _
           }
           const uint32_t sel = (uint32_t)(i & 3ull);
           const uint32_t draw = sel == 0 ? rnd.w[0] : (sel == 1 ? rnd.w[1] : (sel == 2 ? rnd.w[2] : rnd.w[3]));
-          const float xv = __ldg(x + i);
-          const double y = (xv != xv) ? 0.0 : fmin(fmax((double)xv * scale, y_lo), y_hi);
-          const long long Y = __double2ll_rd(y);
-          r = (int32_t)(Y >> 32) + (draw < (uint32_t)Y ? 1 : 0);
+          r = stochastic_round(__ldg(x + i), scale, y_lo, y_hi, draw);
           if (relu) r = max(r, 0);
         }
         const int32_t qq = min(max(r, qmin), qmax);
@@ -131,8 +146,8 @@ __global__ void __launch_bounds__(256) quantize_stochastic_flat_kernel(const flo
                                                                        uint32_t key0, uint32_t key1,
                                                                        adaption_stats* __restrict__ stats) {
   if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
-  const double scale = __longlong_as_double((long long)(1023 + 32 + frac_bits) << 52);   // 2^(frac_bits + 32)
-  const double y_lo = ((double)qmin - 2.0) * 4294967296.0, y_hi = ((double)qmax + 2.0) * 4294967296.0;
+  const float scale = __int_as_float((127 + frac_bits) << 23);   // 2^frac_bits
+  const float y_lo = (float)qmin - 2.0f, y_hi = (float)qmax + 2.0f;
   Counts c;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += nthreads) {
@@ -142,9 +157,7 @@ __global__ void __launch_bounds__(256) quantize_stochastic_flat_kernel(const flo
     int32_t q[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const double y = (xs[u] != xs[u]) ? 0.0 : fmin(fmax((double)xs[u] * scale, y_lo), y_hi);
-      const long long Y = __double2ll_rd(y);
-      int32_t r = (int32_t)(Y >> 32) + (rnd.w[u] < (uint32_t)Y ? 1 : 0);
+      int32_t r = stochastic_round(xs[u], scale, y_lo, y_hi, rnd.w[u]);
       if (relu) r = max(r, 0);
       q[u] = min(max(r, qmin), qmax);
       c.sat_pos += (r > qmax);

@@ -76,7 +76,12 @@ def test_width_histogram(n_bits, shape):
 def test_quantize_stochastic_matches_oracle(n_bits, frac_bits, shape, relu):
     rng = np.random.default_rng(n_bits * 100 + frac_bits + shape[0])
     x = (rng.standard_normal(shape) * 2.0 ** (n_bits - 2 - frac_bits)).astype(np.float32)
-    x.flat[:6] = np.array([np.nan, np.inf, -np.inf, 0.0, -0.0, 2.0 ** -frac_bits], dtype=np.float32)
+    g = 2.0 ** -frac_bits                                 # one grid step
+    special = [np.nan, np.inf, -np.inf, 0.0, -0.0, g, -g, 3 * g, -3 * g, g / 2, -g / 2, g * 2.0 ** -20,
+               -g * 2.0 ** -20, g * (1 - 2.0 ** -24), -g * (1 - 2.0 ** -24), g * (1 + 2.0 ** -23),
+               -g * (1 + 2.0 ** -23), 1e-30, -1e-30, 3e38, -3e38, 5.5 * g, -5.5 * g, 2.0 ** (n_bits - 1) * g,
+               -2.0 ** (n_bits - 1) * g - g / 4]
+    x.flat[:len(special)] = np.array(special, dtype=np.float32)
     seed = (0x9E3779B97F4A7C15 * (shape[0] + 1)) & 0xFFFFFFFFFFFFFFFF
     want, (z, sp, sn) = st.quantize_stochastic(x, n_bits, frac_bits, seed, relu)
     out = B.QTensor.empty(shape[0], shape[1], n_bits, frac_bits, None, with_q16=True)

@@ -404,6 +404,9 @@ POOL_CONV = [
     (2, 24, 24, 128, 256, 3, 1, 1, 8, 8, 8, True),        # single pass, 256-column tiles
     (1, 64, 64, 32, 16, 3, 1, 1, 16, 16, 8, True),        # BN = 32 > output pitch 16: direct stores, full temp
     (2, 12, 12, 20, 50, 5, 2, 1, 16, 16, 16, True),       # plain integer kernel (odd pitch), full temp
+    (3, 44, 44, 128, 128, 3, 1, 2, 16, 16, 16, True),     # stride 2: 22 x 22 outputs, M = 1452 (ragged last tile)
+    (1, 36, 20, 256, 128, 3, 1, 1, 16, 16, 12, True),     # H != W, 12-bit outputs, one image
+    (5, 16, 16, 128, 128, 1, 0, 1, 16, 16, 16, True),     # 1x1 filter
 ]
 
 
