@@ -423,31 +423,32 @@ __device__ __forceinline__ void max16(uint4& bh, uint4& bl, const uint4& h, cons
   }
 }
 
+// IDX: 32-bit index arithmetic (three divisions per output vector) whenever the tensors allow it.
+template <typename IDX>
 __global__ void __launch_bounds__(256) maxpool2x2_kernel(const uint4* __restrict__ in_hi,
                                                          const uint4* __restrict__ in_lo,
                                                          uint4* __restrict__ out_hi,
                                                          uint4* __restrict__ out_lo,
                                                          int16_t* __restrict__ out_q16, int N, int H,
-                                                         int W, int kw, int64_t in_vecs, int64_t out_vecs) {
+                                                         int W, int kw, int64_t in_vecs64, int64_t out_vecs64) {
   // in_vecs / out_vecs: 16-byte vectors per pixel (c_stride / 16).  kw = 2: 2x2 windows; kw = 1: the
   // input is already the horizontal maximum of pixel pairs (W columns), only rows are paired.
-  const int OH = H / 2, OW = W / kw;
-  const int64_t vecs = in_vecs < out_vecs ? in_vecs : out_vecs;
-  const size_t total = (size_t)N * OH * OW * (size_t)out_vecs;
-  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  // H is even, so output row r = n * OH + oh (counted over the batch) pairs input rows 2r, 2r + 1.
+  const IDX in_vecs = (IDX)in_vecs64, out_vecs = (IDX)out_vecs64;
+  const IDX OW = (IDX)(W / kw);
+  const IDX vecs = in_vecs < out_vecs ? in_vecs : out_vecs;
+  const IDX total = (IDX)N * (IDX)(H / 2) * OW * out_vecs;
+  const IDX nthreads = (IDX)gridDim.x * (IDX)blockDim.x;
   const bool two = in_hi != nullptr;
-  for (size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += nthreads) {
-    const int64_t v = (int64_t)(t % (size_t)out_vecs);
-    size_t pix = t / (size_t)out_vecs;
-    const int ow = (int)(pix % OW);
-    pix /= OW;
-    const int oh = (int)(pix % OH);
-    const int n = (int)(pix / OH);
+  for (IDX t = (IDX)blockIdx.x * (IDX)blockDim.x + (IDX)threadIdx.x; t < total; t += nthreads) {
+    const IDX q = t / out_vecs;
+    const IDX v = t - q * out_vecs;
+    const IDX r = q / OW;
+    const IDX ow = q - r * OW;
     uint4 bh = make_uint4(0, 0, 0, 0), bl = make_uint4(0, 0, 0, 0);
     if (v < vecs) {
-      const size_t p00 = (((size_t)n * H + 2 * oh) * W + (size_t)kw * ow) * (size_t)in_vecs + (size_t)v;
-      const size_t offs[4] = {p00, p00 + (size_t)W * in_vecs, p00 + (size_t)in_vecs,
-                              p00 + (size_t)W * in_vecs + (size_t)in_vecs};
+      const IDX p00 = ((IDX)2 * r * (IDX)W + (IDX)kw * ow) * in_vecs + v;
+      const IDX offs[4] = {p00, p00 + (IDX)W * in_vecs, p00 + in_vecs, p00 + (IDX)W * in_vecs + in_vecs};
       const int ncand = 2 * kw;          // the two rows first, then (2x2 only) their right neighbours
       uint4 h[4], l[4];
 #pragma unroll
@@ -468,7 +469,7 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const uint4* __restrict
     if (out_q16 != nullptr) {
       const uint32_t* ph = reinterpret_cast<const uint32_t*>(&bh);
       const uint32_t* pl = reinterpret_cast<const uint32_t*>(&bl);
-      int16_t* dst = out_q16 + t * 16;
+      int16_t* dst = out_q16 + (size_t)t * 16;
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
         const int32_t l8 = (pl[e / 4] >> (8 * (e % 4))) & 255;
@@ -706,10 +707,20 @@ int maxpool_impl(const adaption_qtensor& x, int32_t N, int32_t H, int32_t W, int
   if (total == 0) return ADAPTION_OK;
   const bool two = x.fmt.n_bits > 8;
   const int grid = stream_grid(total, 256, 8);
-  maxpool2x2_kernel<<<grid, 256, 0, stream>>>(
-      two ? reinterpret_cast<const uint4*>(x.hi) : nullptr, reinterpret_cast<const uint4*>(x.lo),
-      two ? reinterpret_cast<uint4*>(y.hi) : nullptr, reinterpret_cast<uint4*>(y.lo), y.q16, N, H,
-      half_pooled ? W / 2 : W, half_pooled ? 1 : 2, x.c_stride / 16, y.c_stride / 16);
+  const uint4* xh = two ? reinterpret_cast<const uint4*>(x.hi) : nullptr;
+  const uint4* xl = reinterpret_cast<const uint4*>(x.lo);
+  uint4* yh = two ? reinterpret_cast<uint4*>(y.hi) : nullptr;
+  uint4* yl = reinterpret_cast<uint4*>(y.lo);
+  const int Win = half_pooled ? W / 2 : W, kw = half_pooled ? 1 : 2;
+  const int64_t in_vecs = x.c_stride / 16, out_vecs = y.c_stride / 16;
+  // 32-bit indices while every input vector index and the loop counter plus one grid stride fit
+  const unsigned long long in_total = (unsigned long long)N * H * Win * (unsigned long long)in_vecs;
+  const unsigned long long limit = (1ull << 32) - (unsigned long long)grid * 256ull;
+  if (in_total < limit && (unsigned long long)total < limit)
+    maxpool2x2_kernel<uint32_t><<<grid, 256, 0, stream>>>(xh, xl, yh, yl, y.q16, N, H, Win, kw, in_vecs, out_vecs);
+  else
+    maxpool2x2_kernel<unsigned long long><<<grid, 256, 0, stream>>>(xh, xl, yh, yl, y.q16, N, H, Win, kw, in_vecs,
+                                                                    out_vecs);
   return cuda_status(cudaGetLastError());
 }
 
