@@ -205,8 +205,9 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restr
   const int64_t groups_per_row = c_stride / 16;
   const size_t total = outer * (size_t)groups_per_row;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  const bool small = total <= 0xffffffffull;      // 32-bit division whenever the group index fits
   for (size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += nthreads) {
-    const size_t row = g / groups_per_row;
+    const size_t row = small ? (size_t)((uint32_t)g / (uint32_t)groups_per_row) : g / groups_per_row;
     const int64_t c0 = (int64_t)(g - row * groups_per_row) * 16;
     const float* __restrict__ src = x + row * (size_t)inner + c0;
     const int nreal = (int)min((int64_t)16, max((int64_t)0, inner - c0));

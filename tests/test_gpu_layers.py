@@ -27,7 +27,7 @@ def _pick_f_out(acc, bq, fb, F, relu, n_out):
 
 
 def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, algo, with_bias=True,
-                  extreme=False, f_out=None, with_q16=True, mag_bits=None, fmts=None, cs=None):
+                  extreme=False, f_out=None, with_q16=True, mag_bits=None, fmts=None, cs=None, ws_offset=0):
     """`with_q16=False` leaves out the optional int16 copy of the output, which lets the tensor-core
     kernel stage its byte planes in shared memory and write them with bulk-tensor stores.
     `mag_bits` limits operand magnitudes (small accumulators -> short requantization shifts)."""
@@ -56,7 +56,7 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
     shp = B.conv_shape(N, H, W, Cin, K, R, R, pad, stride)
     bias_dev = dev(bq) if with_bias else None
     need = B.adaption_lp_conv_workspace_bytes(shp, x.fmt(), w.fmt(), cs, algo)
-    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+    ws = torch.empty(max(need, 16) + ws_offset, dtype=torch.uint8, device="cuda")[ws_offset:] if need else None
     st = B.new_stats()
     B.adaption_lp_conv_fwd(shp, x, w, bias_dev, fw, relu, B.MODE_RANGE, algo, None, st, ws)
     s = B.read_stats(st)
@@ -276,6 +276,15 @@ TC_IP = [(8, 800, 500, 16, 16, 16, True), (70, 1000, 260, 16, 16, 16, False), (2
 def test_ip_tensor(case, cta_mode):
     Bsz, K, O, nx, nw, n_out, relu = case
     run_ip_case(np.random.default_rng(sum(case)), Bsz, K, O, nx, nw, n_out, relu, B.ALGO_TENSOR)
+
+
+@pytest.mark.parametrize("case", [FEW_CHANNELS[0], FEW_CHANNELS[3]])
+def test_conv_few_channels_workspace_on_a_16_byte_boundary(case):
+    """A workspace that is only 16-byte aligned (all the interface asks for) serves the packed rows
+    and the bulk-tensor loads that read them."""
+    N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, cs = case
+    run_conv_case(np.random.default_rng(sum(case) + 7), N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu,
+                  B.ALGO_AUTO, with_q16=False, cs=cs, ws_offset=16)
 
 
 WIDE_CONV = [
