@@ -455,3 +455,13 @@ def test_conv_with_fused_pool(case, with_q16):
     assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
     with pytest.raises(B.AdaptionError):                      # too small a workspace is refused
         B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st, ws[:need - 256])
+    # the two phases issued by separate calls give the same tensor and count the outputs once
+    y.lo.fill_(0x3C)
+    st2 = B.new_stats()
+    B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st2, ws, B.PHASE_CONV)
+    B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st2, ws, B.PHASE_POOL)
+    assert np.array_equal(from_qtensor(y).reshape(want.shape), want)
+    assert stats_tuple(st2) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+    for bad_phases in (0, 4):
+        with pytest.raises(B.AdaptionError):
+            B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st2, ws, bad_phases)
