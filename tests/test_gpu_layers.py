@@ -160,6 +160,8 @@ TC_CONV = [
     (2, 24, 24, 128, 128, 3, 1, 1, 8, 16, 12, False),    # 8-bit activations x 16-bit weights
     (2, 24, 24, 128, 128, 3, 1, 1, 12, 12, 12, True),    # 12-bit operands in planes
     (1, 64, 64, 32, 16, 3, 1, 1, 16, 16, 8, True),       # 16-bit in, 8-bit out, BN=32
+    (5, 30, 30, 64, 64, 3, 1, 1, 16, 16, 16, True),      # 64 -> 64 channels: CTA pair on 64-byte k-blocks, M tail
+    (4, 24, 24, 64, 48, 5, 2, 1, 16, 16, 16, False),     # same family without the paired rule (25 taps), signed
 ]
 
 
@@ -416,6 +418,8 @@ POOL_CONV = [
     (3, 44, 44, 128, 128, 3, 1, 2, 16, 16, 16, True),     # stride 2: 22 x 22 outputs, M = 1452 (ragged last tile)
     (1, 36, 20, 256, 128, 3, 1, 1, 16, 16, 12, True),     # H != W, 12-bit outputs, one image
     (5, 16, 16, 128, 128, 1, 0, 1, 16, 16, 16, True),     # 1x1 filter
+    (4, 32, 32, 64, 64, 3, 1, 1, 16, 16, 16, True),       # 64 -> 64 channels: CTA pair, 64-column tiles, two epilogue groups
+    (3, 26, 30, 64, 40, 3, 1, 1, 16, 16, 16, True),       # same with a ragged M tail and 40 channels
 ]
 
 
