@@ -33,8 +33,8 @@ NOMINAL_INT8_OVER_BF16 = 2.0        # nominal dense INT8 : bf16 ratio (4.5 : 2.2
 # DRAM traffic of the layer GEMM per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged
 # over the 16 layer launches of a forward pass of this workload), from the ncu launch list summarised
 # in profiles/bench_vgg16_b64_launch_list.md.  Valid only for the kernel source it was taken on.
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = 159.1e6
-GEMM_TRAFFIC_SOURCE_SHA1 = "449da2a66417"
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 159.9e6
+GEMM_TRAFFIC_SOURCE_SHA1 = "842eb17b4ed0"
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_BF16_SUSTAINED = 1400.0
 

@@ -1323,7 +1323,10 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   // as a pair each CTA stages half of the weight rows and the MMAs find half of their B operand in
   // the peer's shared memory; with one filter row of taps per stage this measured 0.43 ms against
   // 0.53 ms for 64 x 224 x 224 x 64 -> 64 with the weights resident in a single CTA.
-  const bool narrow_pair = pair_ok && g.is_conv && c.BK == 64 && c.BN == 64 && c.num_kb >= 9 && c.num_kb % 3 == 0;
+  // (16-bit operands only: with one int8 product per k-step the single CTA with resident weights
+  // stays ahead, 0.65 ms against 0.79 ms for the same layer at 8 bits and batch 128)
+  const bool narrow_pair = pair_ok && g.is_conv && c.nacc == 3 && c.BK == 64 && c.BN == 64 && c.num_kb >= 9 &&
+                           c.num_kb % 3 == 0;
   if (narrow_pair) c.pair = true;
   if (pair_env == 0) c.pair = false;
   if (pair_env == 1 && c.splits == 1 && (sms % 2) == 0) c.pair = true;
