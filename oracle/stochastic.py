@@ -5,10 +5,12 @@ drawn so that its expectation is the unrounded value.  The paper fixes neither t
 number generator nor how a draw is compared with the fraction, so both are fixed here
 (readings S1-S3) and the CUDA path follows them bit for bit:
 
-S1  The real value y = x * 2^f is split as y = floor(y) + frac, 0 <= frac < 1, exactly (x is
-    fp32, so both parts are exact in fp64).  The result is floor(y) + 1 with probability
-    T / 2^32, T = floor(frac * 2^32), else floor(y); then it is saturated like the deterministic
-    quantizer (NaN -> 0, +-Inf saturate).  A value already on the grid never moves.
+S1  The real value y = x * 2^f is split as y = floor(y) + frac, 0 <= frac < 1, exactly.  The
+    result is floor(y) + 1 with probability T / 2^32, T = floor(frac * 2^32), else floor(y); then
+    it is saturated like the deterministic quantizer (NaN -> 0, +-Inf saturate).  A value already
+    on the grid never moves.  (floor(y) and T are computed from |y|, whose integer and fractional
+    parts are both exact in fp64 because x is fp32; for y < 0 the fraction 1 - frac(|y|) need not
+    be representable, so T is formed in integers: see ``floor_and_threshold``.)
 S2  The draw for element i (index in the logical [outer][inner] order, padding excluded) is the
     32-bit word  R_i = Philox4x32-10(counter = (i >> 2, 0, 0) as (lo32, hi32, 0, 0),
     key = (seed lo32, seed hi32))[i & 3]  and the value moves up iff R_i < T.
@@ -59,6 +61,27 @@ def draws(n: int, seed: int) -> np.ndarray:
     return words[np.arange(n), (i & np.uint64(3)).astype(np.int64)].astype(np.uint64)
 
 
+def floor_and_threshold(y):
+    """Reading S1 for finite fp64 values y that carry at most 24 significant bits (an fp32 value
+    times a power of two): returns (floor(y) as int64, T = floor((y - floor(y)) * 2^32) as uint64),
+    both exact.  With a = |y| = ia + fa (integer and fractional part, both exact in fp64) and
+    U = fa * 2^32 (exact: a power-of-two scaling):
+        y >= 0            : floor = ia,       T = floor(U)
+        y <  0, fa == 0   : floor = -ia,      T = 0
+        y <  0, fa >  0   : floor = -ia - 1,  frac = 1 - fa,  T = floor(2^32 - U) = 2^32 - ceil(U)
+    The last line is taken in integers; 1 - fa itself can need more than 53 bits (fa = 2^-60)."""
+    y = np.asarray(y, dtype=np.float64)
+    a = np.abs(y)
+    ia = np.floor(a)
+    fa = a - ia                                         # exact
+    U = fa * 4294967296.0                               # exact, 0 <= U < 2^32
+    neg = (y < 0) & (fa > 0)
+    lo = np.where(y < 0, -ia, ia).astype(np.int64) - neg.astype(np.int64)
+    T_pos = np.floor(U).astype(np.uint64)
+    T_neg = np.uint64(1 << 32) - np.ceil(U).astype(np.uint64)
+    return lo, np.where(neg, T_neg, T_pos)
+
+
 def quantize_stochastic(x, n_bits: int, frac_bits: int, seed: int, relu: bool = False):
     """Stochastically rounded canonical integers (int16) of a fp32 tensor, with counters
     (zeros, sat_pos, sat_neg) like the deterministic quantizer.  Readings S1-S2."""
@@ -70,11 +93,9 @@ def quantize_stochastic(x, n_bits: int, frac_bits: int, seed: int, relu: bool = 
     y = np.where(nan, 0.0, y)
     # far outside the range the fraction is irrelevant: clamp first so that floor() stays finite
     y = np.clip(y, float(qmin) - 2.0, float(qmax) + 2.0)
-    lo = np.floor(y)
-    frac = y - lo                                       # exact
-    T = np.floor(frac * 4294967296.0).astype(np.uint64)
+    lo, T = floor_and_threshold(y)
     R = draws(flat.size, seed)
-    r = lo.astype(np.int64) + (R < T).astype(np.int64)
+    r = lo + (R < T).astype(np.int64)
     if relu:
         r = np.maximum(r, 0)
     sat_pos = int((r > qmax).sum())
