@@ -196,9 +196,16 @@ void oracle_ip_acc(const int16_t* x, const int16_t* w, int64_t B, int64_t K, int
 }
 
 /* Round v / 2^s to the nearest integer, ties away from zero (s > 0);
- * exact left shift for s <= 0. */
+ * exact left shift for s <= 0.  Where v * 2^-s does not fit 64 bits the result is
+ * INT64_MAX / INT64_MIN: the callers saturate to at most 16 bits right after, so the
+ * stored value and the saturation count are those of the exact product. */
 static int64_t shift_round(int64_t v, int s) {
-  if (s <= 0) return v * ((int64_t)1 << (-s));
+  if (s <= 0) {
+    int64_t lim = INT64_MAX >> (-s);
+    if (v > lim) return INT64_MAX;
+    if (v < -lim) return INT64_MIN;
+    return v * ((int64_t)1 << (-s));
+  }
   int64_t a = v < 0 ? -v : v;
   int64_t r = (a + ((int64_t)1 << (s - 1))) >> s;
   return v < 0 ? -r : r;

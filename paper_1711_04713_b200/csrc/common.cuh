@@ -33,7 +33,13 @@ __device__ __forceinline__ int32_t requant_value(int64_t v, const RequantParams&
     const int64_t half = (int64_t)1 << (rq.shift - 1);
     r = (v + half + (v >> 63)) >> rq.shift;
   } else {
-    r = v * ((int64_t)1 << (-rq.shift));
+    // Exact left shift by at most 15 bits.  Any |v| above 2^16 already lies outside every output
+    // range (at most 16 bits) after the shift, so clipping v there first keeps the stored value and
+    // the saturation decision while the product stays far inside 64 bits (accumulators can reach
+    // 2^61 for the longest reductions).
+    const int64_t lim = (int64_t)1 << 16;
+    const int64_t vc = v > lim ? lim : (v < -lim ? -lim : v);
+    r = vc * ((int64_t)1 << (-rq.shift));
   }
   if (r > (int64_t)rq.qmax) {
     r = rq.qmax;
