@@ -350,6 +350,22 @@ def test_layer_equals_float_layer_then_quantize():
     del yq
 
 
+def test_epilogue_left_shift_of_huge_accumulators():
+    """Requantizing to MORE fractional bits than the accumulator has (an exact left shift) with
+    accumulators as large as the longest admitted reductions produce: v * 2^15 no longer fits 64
+    bits, the result is still the saturated exact product.  Hand-worked: with F = 0 and Q1.15 out,
+    1 -> 32768 saturates to 32767, -1 -> -32768 exactly, anything larger in magnitude saturates."""
+    acc = np.array([[2 ** 50, -(2 ** 50), 2 ** 62, -(2 ** 62), 1, -1, 0]], dtype=np.int64)
+    y, cnt = orc.epilogue(acc, None, 0, 0, False, 16, 15)
+    assert y.tolist() == [[32767, -32768, 32767, -32768, 32767, -32768, 0]]
+    assert (cnt.zeros, cnt.sat_pos, cnt.sat_neg) == (1, 3, 2)
+    y, cnt = orc.epilogue(acc, None, 0, 0, True, 16, 15)
+    assert y.tolist() == [[32767, 0, 32767, 0, 32767, 0, 0]]
+    assert (cnt.zeros, cnt.sat_pos, cnt.sat_neg) == (4, 3, 0)
+    assert orc.shift_round(3, -2) == 12 and orc.shift_round(-3, -2) == -12
+    assert orc.shift_round(2 ** 47, -15) == 2 ** 62 and orc.shift_round(-(2 ** 47), -15) == -(2 ** 62)
+
+
 def test_requantize_format_change():
     q = np.array([5, -5, 6, -6, 3, 4, -4, 32767, -32768, 0], dtype=np.int16)
     y, cnt = orc.requantize(q, 10, False, 16, 9)          # one bit coarser
@@ -403,6 +419,10 @@ def test_bit_allocation_handworked():
     for row in _read_rows("bit_allocation_handworked.txt"):
         if row[0] == "bits":
             assert int(ba.integer_bits_needed(np.array([float(row[1])]))[0]) == int(row[2]), row
+        elif row[0] == "walloc":
+            n, f, thr = int(row[1]), int(row[2]), float(row[3])
+            hist = [int(v) for v in row[4:4 + ba.HIST_BINS]]
+            assert ba.choose_int_bits_from_widths(hist, f, n, thr) == int(row[4 + ba.HIST_BINS]), row
         else:
             n, thr = int(row[1]), float(row[2])
             hist = [int(v) for v in row[3:3 + ba.HIST_BINS]]
@@ -462,7 +482,201 @@ def test_twos_complement_width():
     assert ba.twos_complement_width(q).tolist() == [1, 1, 2, 2, 3, 4, 5, 4, 5, 8, 9, 8, 9, 16, 16]
 
 
+def _fits(q: int, f: int, m: int) -> bool:
+    """Whether the real value q * 2^-f is a code of the format with m integer bits and f fractional
+    bits (plus sign): -2^m <= value <= 2^m - 2^-f.  Exact rationals, from the format's definition."""
+    v = Fraction(q, 1 << f)
+    return -(Fraction(2) ** m) <= v <= Fraction(2) ** m - Fraction(1, 1 << f)
+
+
+def _allocate(lost_with, total: int, n_bits: int, thr: float) -> int:
+    """Sec. 2.3 as stated: start with every non-sign bit in the integer part, take one away while the
+    values that would no longer be representable number at most thr * total."""
+    m = n_bits - 1
+    while m > 0 and lost_with(m - 1) <= thr * total:
+        m -= 1
+    return m
+
+
+def test_width_allocation_against_exact_rational_definition():
+    """choose_int_bits_from_widths on the histogram of a stored tensor == the allocation done value by
+    value with exact rationals on the real values q * 2^-f; a larger threshold never needs more bits;
+    the accepted loss is within the threshold and one bit fewer would exceed it."""
+    from oracle import bit_allocation as ba
+    rng = np.random.default_rng(5)
+    for n, f in [(16, 8), (16, 2), (12, 9), (8, 3), (8, 0), (4, 1)]:
+        qmin, qmax = -(1 << (n - 1)), (1 << (n - 1)) - 1
+        q = np.clip(np.round(rng.standard_normal(700) * 2.0 ** rng.uniform(0, n - 1, 700)), qmin, qmax).astype(np.int64)
+        q[:6] = [qmin, qmax, 0, -1, 1 << f if (1 << f) <= qmax else 1, -(1 << f) if -(1 << f) >= qmin else -1]
+        hist = ba.width_histogram(q)
+        assert int(hist.sum()) == q.size and int(hist[0]) == 0
+        prev = None
+        for thr in (0.0, 0.003, 0.02, 0.1, 0.4, 1.0):
+            want = _allocate(lambda m: sum(1 for v in q.tolist() if not _fits(v, f, m)), q.size, n, thr)
+            got = ba.choose_int_bits_from_widths(hist, f, n, thr)
+            assert got == want, (n, f, thr)
+            lost = sum(1 for v in q.tolist() if not _fits(v, f, got))
+            assert lost <= thr * q.size
+            if got > 0:
+                assert sum(1 for v in q.tolist() if not _fits(v, f, got - 1)) > thr * q.size
+            assert prev is None or got <= prev
+            prev = got
+    # a value that does not fit is exactly one the requantizer to (n, n-1-m) saturates
+    q = rng.integers(-32768, 32768, 3000).astype(np.int16)
+    m = ba.choose_int_bits_from_widths(ba.width_histogram(q), 9, 16, 0.6)
+    f_new = 15 - m
+    assert f_new > 9                                     # bits moved to the fraction: an exact left shift
+    _, cnt = orc.requantize(q, 9, False, 16, f_new)
+    assert cnt.sat_pos + cnt.sat_neg == sum(1 for v in q.tolist() if not _fits(int(v), 9, m))
+
+
+def _restated_threshold_network(layers, x, n, thr):
+    """The thresholded workflow of Sec. 2.1 / 2.3 on a tiny stack, restated from the definitions in
+    exact rational / integer arithmetic with plain loops (nothing of the oracle is called):
+    formats of fp32 tensors from how many values need more integer bits than offered; a layer output
+    first stored with the format its maximum needs, then, if the threshold lets integer bits go,
+    stored again from the exact sums with the finer format."""
+    qmin, qmax = -(1 << (n - 1)), (1 << (n - 1)) - 1
+
+    def rnd(v: Fraction) -> int:                        # nearest integer, ties away from zero
+        a = abs(v)
+        r = int(a + Fraction(1, 2))                     # floor(a + 1/2)
+        return r if v >= 0 else -r
+
+    def fmt_real(vals):                                 # fractional bits for real values
+        vals = [abs(Fraction(float(v))) for v in vals]
+        m = _allocate(lambda mm: sum(1 for v in vals if v >= Fraction(2) ** mm), len(vals), n, thr)
+        return n - 1 - m
+
+    def quant(vals, f):
+        return [min(max(rnd(Fraction(float(v)) * (1 << f)), qmin), qmax) for v in vals]
+
+    out = []
+    fx = fmt_real(x.reshape(-1))
+    a = np.array(quant(x.reshape(-1), fx), dtype=np.int64).reshape(x.shape)
+    out.append((fx, a.copy()))
+    for L in layers:
+        if L["type"] == "pool":
+            N, H, W, C = a.shape
+            p = np.zeros((N, H // 2, W // 2, C), dtype=np.int64)
+            for idx in np.ndindex(*p.shape):
+                nn, i, j, c = idx
+                p[idx] = max(a[nn, 2 * i, 2 * j, c], a[nn, 2 * i + 1, 2 * j, c], a[nn, 2 * i, 2 * j + 1, c],
+                             a[nn, 2 * i + 1, 2 * j + 1, c])
+            a = p
+            out.append((fx, a.copy()))
+            continue
+        fw = fmt_real(L["w"].reshape(-1))
+        w = np.array(quant(L["w"].reshape(-1), fw), dtype=np.int64).reshape(L["w"].shape)
+        b = quant(L["b"], fw)
+        F = fx + fw
+        if L["type"] == "conv":
+            N, H, W, C = a.shape
+            K, R, S, _ = w.shape
+            pad = L["pad"]
+            OH, OW = H + 2 * pad - R + 1, W + 2 * pad - S + 1
+            v = np.zeros((N, OH, OW, K), dtype=object)
+            for nn, i, j, k in np.ndindex(N, OH, OW, K):
+                t = 0
+                for r in range(R):
+                    for s_ in range(S):
+                        ih, iw = i + r - pad, j + s_ - pad
+                        if 0 <= ih < H and 0 <= iw < W:
+                            for c in range(C):
+                                t += int(a[nn, ih, iw, c]) * int(w[k, r, s_, c])
+                v[nn, i, j, k] = t + (b[k] << fx)
+        else:
+            flat = a.reshape(a.shape[0], -1)
+            v = np.zeros((flat.shape[0], w.shape[0]), dtype=object)
+            for i, o in np.ndindex(*v.shape):
+                v[i, o] = sum(int(p) * int(q) for p, q in zip(flat[i], w[o])) + (b[o] << fx)
+        if L["relu"]:
+            for idx in np.ndindex(*v.shape):
+                v[idx] = max(v[idx], 0)
+        vals = [Fraction(int(t), 1 << F) for t in v.reshape(-1)]
+        top = max(abs(t) for t in vals)
+        m0 = 0
+        while m0 < n - 1 and top >= Fraction(2) ** m0:
+            m0 += 1
+        f0 = n - 1 - m0
+        y0 = [min(max(rnd(t * (1 << f0)), qmin), qmax) for t in vals]
+        m = _allocate(lambda mm: sum(1 for q in y0 if not _fits(q, f0, mm)), len(y0), n, thr)
+        f1 = n - 1 - m
+        y = y0 if f1 == f0 else [min(max(rnd(t * (1 << f1)), qmin), qmax) for t in vals]
+        a = np.array(y, dtype=np.int64).reshape(v.shape)
+        fx = f1
+        out.append((fx, a.copy(), fw, w, f0))
+    return out
+
+
+def _check_thresholded_network(n_bits, thr) -> int:
+    """run_network(threshold > 0) on a tiny conv / pool / inner-product stack: every decimal point
+    and every stored integer equals the from-definition restatement above.  Returns how many layer
+    outputs gave integer bits away."""
+    rng = np.random.default_rng(n_bits * 7 + int(thr * 1000))
+    # heavy-tailed values so that a threshold really moves decimal points
+    def heavy(shape, scale):
+        return (rng.standard_normal(shape) * np.exp(rng.uniform(-2.0, 2.0, shape)) * scale).astype(np.float32)
+    layers = [
+        {"type": "conv", "w": heavy((3, 3, 3, 2), 0.4), "b": heavy((3,), 0.05), "pad": 1, "stride": 1, "relu": True},
+        {"type": "pool"},
+        {"type": "ip", "w": heavy((5, 2 * 2 * 3), 0.5), "b": heavy((5,), 0.05), "relu": True},
+        {"type": "ip", "w": heavy((4, 5), 0.8), "b": heavy((4,), 0.05), "relu": False},
+    ]
+    x = heavy((2, 4, 4, 2), 1.5)
+    rec = orc.run_network(layers, x, None, n_bits, threshold=thr)
+    want = _restated_threshold_network(layers, x, n_bits, thr)
+    assert len(rec) == len(want)
+    moved = 0
+    for r, wnt in zip(rec, want):
+        assert r["frac_bits"] == wnt[0], r["type"]
+        assert np.array_equal(r["y"].astype(np.int64), wnt[1]), r["type"]
+        if r["type"] in ("conv", "ip"):
+            assert r["w_frac_bits"] == wnt[2]
+            assert np.array_equal(r["wq"].astype(np.int64), wnt[3])
+            moved += int(wnt[4] != wnt[0])
+    base = orc.run_network(layers, x, None, n_bits)
+    assert all(r["frac_bits"] >= b["frac_bits"] for r, b in zip(rec[:1], base[:1]))
+    return moved
+
+
+def test_thresholded_network_driver_against_restatement():
+    moved = [_check_thresholded_network(n, t) for n, t in [(8, 0.1), (8, 0.02), (16, 0.05), (6, 0.25)]]
+    assert sum(moved) > 0          # not vacuous: somewhere a layer output gives integer bits away
+
+
 # ---------------------------------------------------------------- stochastic rounding (Sec. 2.4)
+def test_stochastic_floor_and_threshold_exact():
+    """floor(y) and T = floor(frac(y) * 2^32) against exact rationals, on the values where a
+    double-precision y - floor(y) is not exact: tiny negative y (frac = 1 - 2^-k), the largest
+    fractions below one, both signs, grid values, and random fp32 values over many binades."""
+    from oracle import stochastic as st
+    f32 = lambda v: float(np.float32(v))
+    ys = [0.0, 1.0, -1.0, 0.5, -0.5, 2.0 ** -60, -(2.0 ** -60), f32(-1e-30), f32(1e-30), -(2.0 ** -33), 2.0 ** -33,
+          -(2.0 ** -32), 2.0 ** -32, -(2.0 ** -31), 1 - 2.0 ** -24, -(1 - 2.0 ** -24), 7 + (1 - 2.0 ** -21),
+          -7 - (1 - 2.0 ** -21), -(2.0 ** -149), 2.0 ** -149, 32766.998046875, -32768.998046875,
+          f32(0.1) * 2.0 ** 15, -f32(0.1) * 2.0 ** 15, 3.0 + 2.0 ** -20, -3.0 - 2.0 ** -20]
+    rng = np.random.default_rng(12)
+    xs = (rng.standard_normal(3000) * np.exp(rng.uniform(-40, 10, 3000))).astype(np.float32)
+    ys += [float(v) * 2.0 ** 9 for v in xs if abs(float(v) * 2.0 ** 9) < 2.0 ** 40]
+    lo, T = st.floor_and_threshold(np.array(ys, dtype=np.float64))
+    for y, l, t in zip(ys, lo.tolist(), T.tolist()):
+        fy = Fraction(y)
+        fl = fy.numerator // fy.denominator            # floor of the exact value
+        frac = fy - fl
+        assert l == fl, y
+        assert t == (frac * (1 << 32)).numerator // (frac * (1 << 32)).denominator, y
+        assert 0 <= t < (1 << 32)
+    # the cases the text names
+    lo, T = st.floor_and_threshold(np.array([-(2.0 ** -60), 1 - 2.0 ** -24, -(1 - 2.0 ** -24), 5.0, -5.0]))
+    assert lo.tolist() == [-1, 0, -1, 5, -5]
+    assert T.tolist() == [(1 << 32) - 1, (1 << 32) - 256, 256, 0, 0]
+    # and through the quantizer: a tiny negative value goes to 0 unless the draw is exactly 2^32 - 1,
+    # a tiny positive one stays 0 (T = 0: no draw is below it)
+    q, _ = st.quantize_stochastic(np.array([-1e-30, 1e-30, -(2.0 ** -140)], dtype=np.float32), 16, 8, seed=5)
+    assert q.tolist() == [0, 0, 0]
+
+
 def test_philox_known_answers():
     from oracle import stochastic as st
     for row in _read_rows("philox4x32_10_kat.txt"):
