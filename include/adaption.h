@@ -53,7 +53,9 @@ enum {
 };
 
 /* rounding_scheme of the paper (Sec. 2, Sec. 2.4).  Deterministic = round to nearest, ties
- * away from zero.  Stochastic rounding is not implemented: ADAPTION_ERR_UNSUPPORTED. */
+ * away from zero.  Stochastic rounding needs a seed and therefore has entry points of its own
+ * (adaption_quantize_stochastic, adaption_lp_act_stochastic); the calls that take a `rounding`
+ * argument but no seed answer ADAPTION_ERR_UNSUPPORTED for ADAPTION_ROUND_STOCHASTIC. */
 enum { ADAPTION_ROUND_DETERMINISTIC = 0, ADAPTION_ROUND_STOCHASTIC = 1 };
 
 /* Bins of the bit-occupancy histograms (Sec. 2.2, 2.3): 0..15 bits, and 16 or more. */
@@ -243,8 +245,13 @@ ADAPTION_API int adaption_lp_ip_fwd(int64_t B, int64_t K, int64_t O, adaption_qt
  *     is split), the call returns ADAPTION_ERR_WORKSPACE and launches nothing; use
  *     adaption_lp_ip_fwd with your own buffer for such shapes.
  *   - The first call on each device looks the array's device address up (one runtime query with
- *     that device current; a failure is reported as ADAPTION_ERR_CUDA).  Make that first call
- *     before any stream capture begins.
+ *     that device current; a failure is reported as ADAPTION_ERR_CUDA).  That query may be the
+ *     moment the CUDA runtime loads the library's device code on that device, array included, so
+ *     "allocates nothing" describes every call after the first.  Make that first call before any
+ *     stream capture begins.  The address is cached per device for the life of the process: do
+ *     not use this entry point on a device after cudaDeviceReset.
+ *   - Shapes that need no workspace (an unsplit reduction, or ADAPTION_ALGO_DIRECT) never touch
+ *     the array.
  *   - All calls on a device share the one array and it keeps the previous call's contents; each
  *     call clears the part it uses before accumulating.  Two calls whose GPU work can overlap
  *     (different streams, or different host threads on the same device) race on it: run them on
@@ -277,6 +284,24 @@ ADAPTION_API int adaption_choose_frac_bits_from_acc(int64_t max_abs_acc, int32_t
  * pipelined mainloop issues them; 0 issues none.  Asynchronous on `stream`. */
 ADAPTION_API int adaption_probe_i8_peak(int32_t bn, int32_t pair, int32_t iters, int32_t commit_every,
                                         uint64_t* d_cycles, int32_t* d_status, void* stream);
+
+/* Test and experiment aid (no counterpart in the paper; not meant for production callers).  Sets one
+ * process-wide override of the tensor-core path's tile heuristics, so that tests can drive the same
+ * layer through its alternative code paths and compare the bits.  h_name is a host string:
+ *   "splits" n     at least n splits of the reduction            (default 0: heuristic)
+ *   "pair" 0|1     forbid / force CTA pairs                       (default -1: heuristic)
+ *   "fast" 0       generic 64-bit epilogue instead of the 32-bit one        (default 1)
+ *   "staged" 0     direct stores instead of shared-memory staging           (default 1)
+ *   "stages" n     cap the depth of the shared-memory ring                  (default 0: none)
+ *   "bk" 32|64, "bn" 32|64, "kps" 1..4, "bres" 0, "wide" 0, "epigroups" 1   narrower tiles etc.
+ *   "timeout_us" t limit of every device-side wait in microseconds (default 0: two seconds)
+ *   "stall_at" i   the copy-issuing warps of every block stop before their i-th stage with nothing
+ *                  in flight for it, so that the waits of the other warps run out: the kernel then
+ *                  sets stats.status = ADAPTION_ERR_TIMEOUT, drains and returns (default -1: never)
+ *   "reset"        every override back to its default (value ignored)
+ * Returns ADAPTION_ERR_INVALID_ARG for an unknown name.  Calls already enqueued are not affected;
+ * do not change overrides while another host thread is inside a layer call. */
+ADAPTION_API int adaption_debug_set(const char* h_name, int32_t value);
 
 ADAPTION_API const char* adaption_status_string(int status);
 

@@ -24,6 +24,7 @@ _SRC = os.path.join(_HERE, "adaption_oracle.c")
 _BUILD = os.path.join(_HERE, "_build")
 _LIB_PATH = os.path.join(_BUILD, "libadaption_oracle.so")
 _lib = None
+BUILD_FLAGS = ["-O2", "-fopenmp", "-std=c11"]
 
 
 def build(force: bool = False) -> str:
@@ -32,7 +33,7 @@ def build(force: bool = False) -> str:
     if force or not os.path.exists(_LIB_PATH) or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC):
         tmp = _LIB_PATH + f".{os.getpid()}.tmp"
         subprocess.check_call(
-            ["gcc", "-O2", "-fopenmp", "-std=c11", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+            ["gcc"] + BUILD_FLAGS + ["-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
         os.replace(tmp, _LIB_PATH)
     return _LIB_PATH
 

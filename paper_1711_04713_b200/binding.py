@@ -57,7 +57,7 @@ EXPORTS = [
     "adaption_quantize_stochastic", "adaption_bit_histogram", "adaption_width_histogram",
     "adaption_choose_frac_bits_from_hist", "adaption_choose_frac_bits_from_widths",
     "adaption_lp_act_stochastic", "adaption_lp_conv_pool_workspace_bytes", "adaption_lp_conv_pool_fwd",
-    "adaption_quantize_batch",
+    "adaption_quantize_batch", "adaption_debug_set",
 ]
 HIST_BINS = 17
 
@@ -113,6 +113,7 @@ def load(path: str | None = None):
                                                         C.POINTER(adaption_qfmt)]
     lib.adaption_choose_frac_bits_from_widths.argtypes = [C.POINTER(C.c_uint64), I32, I32, C.c_double,
                                                           C.POINTER(adaption_qfmt)]
+    lib.adaption_debug_set.argtypes = [C.c_char_p, C.c_int32]
     lib.adaption_status_string.argtypes = [C.c_int]
     lib.adaption_status_string.restype = C.c_char_p
     for name in EXPORTS:
@@ -121,6 +122,11 @@ def load(path: str | None = None):
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
+
+
+def adaption_debug_set(name: str, value: int = 0):
+    """Test / experiment override of the tensor-core path's heuristics (see the header)."""
+    _check(load().adaption_debug_set(name.encode(), int(value)), f"adaption_debug_set({name})")
 
 
 def status_string(status: int) -> str:

@@ -32,6 +32,7 @@ int choose_frac_bits_from_widths(const uint64_t*, int32_t, int32_t, double, adap
 int probe_i8_peak(int bn, int pair, int iters, int commit_every, unsigned long long* d_cycles, int* d_status,
                   cudaStream_t stream);
 int num_sms();
+int debug_set(const char* name, int value);
 
 // Longest reduction the direct kernels and the int64 workspace can take without overflow:
 // |q_x * q_w| <= 2^30, so 2^31 terms still leave a sign bit and headroom for the bias.
@@ -382,6 +383,8 @@ int adaption_probe_i8_peak(int32_t bn, int32_t pair, int32_t iters, int32_t comm
   return probe_i8_peak(bn, pair ? 1 : 0, iters, commit_every, reinterpret_cast<unsigned long long*>(d_cycles), d_status,
                        reinterpret_cast<cudaStream_t>(stream));
 }
+
+int adaption_debug_set(const char* h_name, int32_t value) { return debug_set(h_name, value); }
 
 const char* adaption_status_string(int status) {
   switch (status) {

@@ -1,21 +1,26 @@
 // HBM-bound kernels: dynamic-range measurement, the fp32 -> fixed-point quantizer (LPAct with an
 // fp32 input is the same kernel with the ReLU flag), fixed-point format conversion, 2x2 max-pool.
 // All of them are coalesced streaming kernels sized to a multiple of the SM count.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace adaption {
 
-static int g_num_sms = 0;
-
+// SM count of the current device, cached per device ordinal (each entry is written once with the
+// same value by whichever thread gets there first, so a relaxed atomic is all it needs).
 int num_sms() {
-  if (g_num_sms == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-    g_num_sms = n;
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cache[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  const bool cached = dev >= 0 && dev < kMaxDevices;
+  int n = cached ? cache[dev].load(std::memory_order_relaxed) : 0;
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    if (cached) cache[dev].store(n, std::memory_order_relaxed);
   }
-  return g_num_sms;
+  return n;
 }
 
 static inline int stream_grid(size_t work_items, int threads, int blocks_per_sm) {

@@ -21,8 +21,10 @@
 // caller's stats word, drains what it has in flight, frees its TMEM and returns.
 #include <cuda.h>
 
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -78,6 +80,10 @@ struct TcParams {
   long long ws_ld;
   adaption_stats* stats;
   unsigned long long timeout_ns;
+  // test aid (adaption_debug_set "stall_at"): every producer warp stops, with nothing in flight for
+  // that stage, before its stage number `stall_at` (counted per CTA from 0); -1 = never.  The waits
+  // of the other roles then run out and the kernel reports ADAPTION_ERR_TIMEOUT.
+  int stall_at;
   // epilogue variants chosen on the host
   int fast_relu;              // launch the FAST kernel variant (paired 16-bit epilogue)
   int pool_w;                 // store max(row 2j, row 2j+1) of the tile: half of a 2x2 max-pool (staged only)
@@ -806,7 +812,8 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         __syncwarp();
       }
       const bool in_tile_loop = sub < nsub;
-      for (int t = worker; t < p.total_tiles && ok && in_tile_loop; t += workers) {
+      bool stalled = false;
+      for (int t = worker; t < p.total_tiles && ok && in_tile_loop && !stalled; t += workers) {
         const TileCoord tc = decode_tile(t, p);
         const int m_begin = tc.m0 + (int)rank * kBM;        // first of the 128 rows this CTA stages
         const int n_begin = tc.n0 + (int)rank * b_rows;     // first weight row this CTA stages
@@ -826,6 +833,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           sx = tap - r * p.S;
         }
         for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps, ++it) {
+          if (it == (uint32_t)p.stall_at) { stalled = true; break; }
           const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;      // k-blocks in this stage
           const bool my_turn = (s % nsub) == sub;     // ring slots have fixed owners
           uint32_t full = 0, dst = 0;
@@ -1001,7 +1009,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       }
       if ((!ok || ctrl.abort) && lane == 0) {
         // make sure no MMA still reads shared memory or writes TMEM when the CTAs tear down
-        tc_commit<false>(smem_u32(&ctrl.drain));
+        tc_commit<PAIR>(smem_u32(&ctrl.drain));
         const unsigned long long t0 = global_ns();
         while (!mbar_try_wait(smem_u32(&ctrl.drain), 0) && global_ns() - t0 < 50000000ull) {
         }
@@ -1179,21 +1187,25 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 
 EncodeTiledFn g_encode_tiled = nullptr;
 EncodeIm2colFn g_encode_im2col = nullptr;
+std::once_flag g_encode_once;
 
+// The two tensor-map encoders of the driver, looked up once per process (they are the same for
+// every device).
 bool load_driver_entry_points() {
-  if (g_encode_tiled != nullptr && g_encode_im2col != nullptr) return true;
-  void* f1 = nullptr;
-  void* f2 = nullptr;
-  cudaDriverEntryPointQueryResult q1, q2;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f1, cudaEnableDefault, &q1) != cudaSuccess ||
-      q1 != cudaDriverEntryPointSuccess || f1 == nullptr)
-    return false;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f2, cudaEnableDefault, &q2) != cudaSuccess ||
-      q2 != cudaDriverEntryPointSuccess || f2 == nullptr)
-    return false;
-  g_encode_tiled = reinterpret_cast<EncodeTiledFn>(f1);
-  g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(f2);
-  return true;
+  std::call_once(g_encode_once, [] {
+    void* f1 = nullptr;
+    void* f2 = nullptr;
+    cudaDriverEntryPointQueryResult q1, q2;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f1, cudaEnableDefault, &q1) != cudaSuccess ||
+        q1 != cudaDriverEntryPointSuccess || f1 == nullptr)
+      return;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f2, cudaEnableDefault, &q2) != cudaSuccess ||
+        q2 != cudaDriverEntryPointSuccess || f2 == nullptr)
+      return;
+    g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(f2);
+    g_encode_tiled = reinterpret_cast<EncodeTiledFn>(f1);
+  });
+  return g_encode_tiled != nullptr && g_encode_im2col != nullptr;
 }
 
 struct TcConfig {
@@ -1222,11 +1234,16 @@ struct TcConfig {
   size_t workspace_bytes = 0;
 };
 
-int env_int(const char* name, int dflt) {
-  const char* v = std::getenv(name);
-  if (v == nullptr || *v == 0) return dflt;
-  return std::atoi(v);
-}
+// Test and experiment overrides of the tile heuristics, set through adaption_debug_set (never read
+// from the environment, so the layer calls themselves do no string work).  Each holds its
+// default until set; the setter is the only writer.
+enum Knob { kSplits, kPair, kFast, kStaged, kStages, kBK, kBN, kKps, kBres, kWide, kEpiGroups, kTimeoutUs, kStallAt,
+            kNumKnobs };
+const char* const kKnobNames[kNumKnobs] = {"splits", "pair", "fast", "staged", "stages", "bk", "bn", "kps", "bres",
+                                           "wide", "epigroups", "timeout_us", "stall_at"};
+const int kKnobDefaults[kNumKnobs] = {0, -1, 1, 1, 0, 0, 0, 0, 1, 1, 2, 0, -1};
+std::atomic<int> g_knobs[kNumKnobs] = {{0}, {-1}, {1}, {1}, {0}, {0}, {0}, {0}, {1}, {1}, {2}, {0}, {-1}};
+inline int knob(Knob k) { return g_knobs[k].load(std::memory_order_relaxed); }
 
 TcConfig make_config_impl(const GemmProblem& g, bool allow_wide);
 
@@ -1263,7 +1280,7 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   } else {
     if (g.K < 32) return c;
     c.BK = g.K >= 128 ? 128 : (g.K >= 64 ? 64 : 32);
-    const int forced_bk = env_int("ADAPTION_TC_BK", 0);   // experiment knob: narrower K-blocks
+    const int forced_bk = knob(kBK);   // experiment knob: narrower K-blocks
     if ((forced_bk == 32 || forced_bk == 64) && forced_bk < c.BK) c.BK = forced_bk;
     c.num_kb = (int)((g.K + c.BK - 1) / c.BK);
     k_padded = g.K;
@@ -1273,14 +1290,14 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
                           : (c.BK == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
   c.layout_type = c.BK == 128 ? 2u : (c.BK == 64 ? 4u : 6u);
   c.BN = g.N <= 32 ? 32 : (g.N <= 64 ? 64 : 128);
-  const int forced_bn = env_int("ADAPTION_TC_BN", 0);    // experiment knob: narrower tiles
+  const int forced_bn = knob(kBN);    // experiment knob: narrower tiles
   if ((forced_bn == 32 || forced_bn == 64) && forced_bn < c.BN) c.BN = forced_bn;
   // Single-pass (8-bit) layers with many output channels take 256-column pair tiles: one int32
   // accumulator per tile leaves room for two sets of 256 columns, and a 256 x 256 tile halves the
   // operand bytes per MMA cycle, which is what limits the int8 rate (see make_config's pair notes).
   const bool wide = allow_wide && c.nacc == 1 && c.BK == 128 && g.N >= 256 && c.num_kb >= 9 && g.M >= 1024 &&
-                    (num_sms() % 2) == 0 && forced_bn == 0 && env_int("ADAPTION_TC_PAIR", -1) != 0 &&
-                    env_int("ADAPTION_TC_WIDE", 1) != 0;
+                    (num_sms() % 2) == 0 && forced_bn == 0 && knob(kPair) != 0 &&
+                    knob(kWide) != 0;
   if (wide) c.BN = 256;
   c.tiles_m = (int)((g.M + kBM - 1) / kBM);
   c.tiles_n = (int)((g.N + c.BN - 1) / c.BN);
@@ -1302,7 +1319,7 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
     if (want > cap) want = cap;
     if (want > splits) splits = want;
   }
-  const int forced = env_int("ADAPTION_TC_SPLITS", 0);
+  const int forced = knob(kSplits);
   if (forced > 0) splits = forced > splits ? forced : splits;
   if (splits > c.num_kb) splits = c.num_kb;
   if (splits < 1) splits = 1;
@@ -1313,7 +1330,7 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   c.workspace_bytes = c.splits > 1 ? (size_t)g.M * (size_t)g.N * sizeof(long long) : 0;
   // Large unsplit problems run as CTA pairs: 256-row tiles, each CTA stages its own 128 rows of A
   // and only half of the weight rows, which cuts the bytes (and TMA rows) per MAC by a quarter.
-  const int pair_env = env_int("ADAPTION_TC_PAIR", -1);
+  const int pair_env = knob(kPair);
   // (measured: pairs win from K = 1152 bytes per plane row on; 256 x 64 pair tiles with two
   // accumulator sets were tried for medium reductions and lost to these once the epilogue hands the
   // accumulators back early)
@@ -1340,11 +1357,11 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   // the output planes (pitch a multiple of 16 bytes and at least one tile wide) and no int16 copy.
   const int out_planes = g.y.fmt.n_bits > 8 ? 2 : 1;
   c.staged = g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.y.q16 == nullptr && g.y.lo != nullptr &&
-             g.y.c_stride >= c.BN && g.y.c_stride % 16 == 0 && env_int("ADAPTION_TC_STAGED", 1) != 0;
+             g.y.c_stride >= c.BN && g.y.c_stride % 16 == 0 && knob(kStaged) != 0;
   // two epilogue groups when two tiles can be in flight in TMEM and their constants fit the halves
   // of the per-column array
   c.epi_groups = (c.acc_bufs >= 2 && c.acc_bufs % 2 == 0 && c.BN <= 64 &&
-                  env_int("ADAPTION_TC_EPIGROUPS", 2) == 2) ? 2 : 1;
+                  knob(kEpiGroups) == 2) ? 2 : 1;
   c.stage_out_bytes = c.staged ? (uint32_t)(kBM * c.BN * out_planes * c.epi_groups) : 0u;
   // dynamic shared memory: everything up to the per-block limit except the control block
   c.const_bytes = (uint32_t)(c.BN * c.epi_groups * sizeof(long long));
@@ -1355,7 +1372,7 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
     const int cyc_per_kb = (c.BK / 32) * products * (c.BN >= 128 ? c.BN / 2 : 48);
     int kps = (768 + cyc_per_kb - 1) / cyc_per_kb;
     if (kps > 4) kps = 4;
-    const int kps_env = env_int("ADAPTION_TC_KPS", 0);
+    const int kps_env = knob(kKps);
     if (narrow_pair && c.pair) kps = 3;
     if (kps_env >= 1 && kps_env <= 4) kps = kps_env;
     if (kps > c.kb_per_split) kps = c.kb_per_split;
@@ -1368,7 +1385,7 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   // 3-channel layers).  Only if at least three activation stages still fit.
   const size_t res_bytes = (size_t)c.num_kb * c.nbw * c.b_bytes;
   if (!c.pair && c.tiles_n == 1 && c.splits == 1 && c.tiles_m >= 4 * sms &&
-      res_bytes + 3 * (size_t)c.kps * c.nax * c.a_bytes + 1024 <= budget && env_int("ADAPTION_TC_BRES", 1) != 0) {
+      res_bytes + 3 * (size_t)c.kps * c.nax * c.a_bytes + 1024 <= budget && knob(kBres) != 0) {
     c.b_resident = true;
     c.b_res_bytes = (uint32_t)res_bytes;
     c.kb_bytes = c.nax * c.a_bytes;
@@ -1382,7 +1399,7 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
     c.stage_out_bytes = 0;
   }
   if (c.stages > kMaxStages) c.stages = kMaxStages;
-  const int stage_cap = env_int("ADAPTION_TC_STAGES", 0);   // experiment knob: shallower ring
+  const int stage_cap = knob(kStages);   // experiment knob: shallower ring
   if (stage_cap >= 2 && stage_cap < c.stages) c.stages = stage_cap;
   if (c.stages < 2) return c;
   c.stage_off = (uint32_t)(((size_t)c.stages * c.stage_bytes + c.b_res_bytes + 1023) & ~(size_t)1023);
@@ -1418,12 +1435,22 @@ bool encode_im2col_nhwc(CUtensorMap* map, const void* base, const adaption_conv_
 
 template <int NAX, int NBW, bool PAIR, bool GROUPED, bool FAST>
 int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem, cudaStream_t stream) {
-  static size_t attr_size = 0;
-  if (smem > attr_size) {
+  // The dynamic shared-memory limit is a per-device attribute of the kernel: remember, per device
+  // ordinal, the largest size it has been raised to (a racing thread at worst sets it once more).
+  constexpr int kMaxDevices = 64;
+  static std::atomic<size_t> attr_size[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ADAPTION_ERR_CUDA;
+  const bool cached = dev >= 0 && dev < kMaxDevices;
+  if (!cached || smem > attr_size[dev].load(std::memory_order_acquire)) {
     const cudaError_t ae = cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, FAST>,
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (ae != cudaSuccess) return cuda_failure(ae, "lp_gemm_kernel shared-memory attribute");
-    attr_size = smem;
+    if (cached) {
+      size_t seen = attr_size[dev].load(std::memory_order_relaxed);
+      while (seen < smem && !attr_size[dev].compare_exchange_weak(seen, smem, std::memory_order_release)) {
+      }
+    }
   }
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
@@ -1585,6 +1612,20 @@ extern "C" __attribute__((visibility("default"))) int adaption_debug_timeline(lo
 }
 #endif
 
+int debug_set(const char* name, int value) {
+  if (name == nullptr) return ADAPTION_ERR_INVALID_ARG;
+  if (std::strcmp(name, "reset") == 0) {
+    for (int k = 0; k < kNumKnobs; ++k) g_knobs[k].store(kKnobDefaults[k], std::memory_order_relaxed);
+    return ADAPTION_OK;
+  }
+  for (int k = 0; k < kNumKnobs; ++k)
+    if (std::strcmp(name, kKnobNames[k]) == 0) {
+      g_knobs[k].store(value, std::memory_order_relaxed);
+      return ADAPTION_OK;
+    }
+  return ADAPTION_ERR_INVALID_ARG;
+}
+
 bool tensor_path_supported(const GemmProblem& g) { return make_config(g).ok; }
 
 // The horizontal half of a 2x2 max-pool can ride on the staged stores of a requantizing layer.
@@ -1667,7 +1708,7 @@ int launch_tensor(const GemmProblem& g) {
   p.const_off = c.stage_off + c.stage_out_bytes;
   const bool single = c.nacc == 1;
   if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && p.rq.shift >= (single ? 0 : 9) &&
-      p.rq.shift <= 31 && g.N % 8 == 0 && env_int("ADAPTION_TC_FAST", 1) != 0) {
+      p.rq.shift <= 31 && g.N % 8 == 0 && knob(kFast) != 0) {
     // 32-bit bounds of the fast epilogue (see shifted32): with a reduction of kred bytes per plane row
     // |hh| <= kred 2^14, |mid| <= kred 65280, |ll| <= kred 65025, and |C| < 2^(15 + bias_shift) + 2^(shift-1)
     const long long kred = (long long)c.num_kb * c.BK;
@@ -1685,7 +1726,8 @@ int launch_tensor(const GemmProblem& g) {
   }
   p.ws = (long long*)g.workspace; p.ws_ld = g.N;
   p.stats = g.stats;
-  p.timeout_ns = 2000000000ull;
+  p.timeout_ns = knob(kTimeoutUs) > 0 ? 1000ull * (unsigned long long)knob(kTimeoutUs) : 2000000000ull;
+  p.stall_at = knob(kStallAt);
 
   if (c.splits > 1) {
     const cudaError_t me = cudaMemsetAsync(g.workspace, 0, c.workspace_bytes, g.stream);

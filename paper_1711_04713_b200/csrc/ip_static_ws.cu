@@ -16,7 +16,9 @@ constexpr int kMaxDevices = 64;
 void* g_ws_addr[kMaxDevices] = {};
 std::mutex g_ws_mutex;
 
-// Device address of the scratch array on the current device, looked up once per device.
+// Device address of the scratch array on the current device, looked up once per device.  (The
+// cached address belongs to the device's current primary context: after a cudaDeviceReset the
+// process must not call this entry point on that device again.)
 int scratch_address(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ADAPTION_ERR_CUDA;
@@ -34,15 +36,6 @@ int scratch_address(void** out) {
 }
 
 }  // namespace
-
-namespace adaption {
-// Device code may name the array directly.  This reader (external linkage, so it is always kept)
-// holds a device-side reference to the array and lets a debugger compare the address the runtime
-// reports with the one kernels see.
-__global__ void static_ws_address_kernel(unsigned long long* out) {
-  *out = (unsigned long long)(uintptr_t)g_ip_static_ws;
-}
-}  // namespace adaption
 
 extern "C" int adaption_lp_ip_fwd_static_ws(int64_t B, int64_t K, int64_t O, adaption_qtensor x,
                                             adaption_qtensor w, const int16_t* d_bias_q,

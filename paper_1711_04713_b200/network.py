@@ -16,6 +16,40 @@ import numpy as np
 import torch
 
 from . import binding as B
+from . import replicas
+
+
+def calibration_loop(be, kinds: list[str], threshold: float = 0.0, group=None, device="cpu"):
+    """The calibration workflow of paper Sec. 2.1 / 2.3 as host logic over a backend `be` that runs the
+    layers (the CUDA library for LPNetwork; anything with the same methods in tests): measure the
+    input's range, quantize it, then per layer a RANGE pass, the decimal point from the measured
+    range, a REQUANT pass (and, with `threshold` > 0, the width histogram of that output and a second
+    REQUANT pass if integer bits can go).  With a process group every range, histogram and counter
+    is reduced over the replicas, so that all of them fix the same decimal points (each replica holds
+    its own shard of the batch, the weights are replicated).  Returns the per-layer records."""
+    rec = []
+    fx = be.input_frac_bits(threshold, group)
+    rec.append({"type": "input", "frac_bits": fx, "stats": be.quantize_input(fx)})
+    for i, kind in enumerate(kinds):
+        if kind == "pool":
+            rec.append({"type": "pool", "frac_bits": be.pool(i)})
+            continue
+        local = int(be.range_pass(i))
+        A = replicas.agree_on_range(local, device, group)
+        F = be.acc_frac_bits(i)
+        f = be.choose_from_acc(A, F)
+        st = be.requant_pass(i, f)
+        if threshold > 0:
+            hist = replicas.sum_histogram(be.width_histogram(i), device, group)
+            f2 = be.choose_from_widths(hist, f, threshold)
+            if f2 != f:
+                f = f2
+                st = be.requant_pass(i, f)
+        totals = replicas.sum_counters(int(st.zeros), int(st.sat_pos), int(st.sat_neg), device, group)
+        rec.append({"type": kind, "name": be.layer_name(i), "frac_bits": f, "w_frac_bits": be.w_frac_bits(i),
+                    "max_abs_acc": A, "local_max_abs_acc": local, "acc_frac_bits": F, "stats": st,
+                    "counters_all_replicas": totals})
+    return rec
 
 
 def act_c_stride(c: int) -> int:
@@ -247,60 +281,96 @@ class LPNetwork:
         return L.y
 
     # ------------------------------------------------------------------ calibration
-    def calibrate(self, x_f32: torch.Tensor, x_fmt: tuple[int, int] | None = None, threshold: float = 0.0):
+    def calibrate(self, x_f32: torch.Tensor, x_fmt: tuple[int, int] | None = None, threshold: float = 0.0,
+                  group=None):
         """Run one batch layer by layer, measuring each layer's range on it and fixing its decimal
         point (paper Sec. 2.1, 2.3).  Returns the per-layer records (formats, counters, ranges).
         ``threshold`` > 0: thresholded allocation of the integer bits instead of the maximum (fp32
         tensors from their bit-occupancy histogram; a layer output is first stored with the
-        max-based format, the widths of those integers decide, then the layer is run again)."""
+        max-based format, the widths of those integers decide, then the layer is run again).
+        ``group`` (or an initialised default process group): data-parallel replicas, each calibrating
+        on its own shard of the batch, agree on every decimal point (see ``calibration_loop``)."""
         self.quantize_params(measure=True, threshold=threshold)
-        rec = []
-        self.x_stats.zero_()
-        if x_fmt is None and threshold > 0:
-            self.xq.frac_bits = self._fp32_fmt_by_threshold(x_f32, threshold)
-        elif x_fmt is None:
-            self.x_max_dev.zero_()
-            B.adaption_measure_range(x_f32, self.n_bits, self.x_max_dev, self.x_fmt_dev)
-            self.xq.frac_bits = int(self.x_fmt_dev.cpu()[1])
-        else:
-            assert x_fmt[0] == self.n_bits
-            self.xq.frac_bits = x_fmt[1]
-        B.adaption_quantize(x_f32, self.xq.outer, self.xq.inner, self.xq, None, B.ROUND_DETERMINISTIC,
-                            self.x_stats)
-        rec.append({"type": "input", "frac_bits": self.xq.frac_bits, "stats": B.read_stats(self.x_stats)})
-        a = self.xq
-        for L in self.layers:
-            if L.type == "pool":
-                a = self._run_layer(L, a, B.MODE_REQUANT)
-                rec.append({"type": "pool", "frac_bits": a.frac_bits})
-                continue
-            L.stats.zero_()
-            self._run_layer(L, a, B.MODE_RANGE)
-            st = B.read_stats(L.stats)
-            if st.status != 0:
-                raise B.AdaptionError(st.status, f"layer {L.name} (range)")
-            F = a.frac_bits + L.w.frac_bits
-            L.y.frac_bits = B.adaption_choose_frac_bits_from_acc(int(st.max_abs_acc), F, self.n_bits)
-            L.stats.zero_()
-            a_in = a
-            a = self._run_layer(L, a_in, B.MODE_REQUANT)
-            if threshold > 0:
-                hist = B.new_hist(self.device)
-                B.adaption_width_histogram(L.y, hist)
-                f = B.adaption_choose_frac_bits_from_widths(hist.cpu().tolist(), L.y.frac_bits, self.n_bits,
-                                                            threshold)
-                if f != L.y.frac_bits:
-                    L.y.frac_bits = f
-                    L.stats.zero_()
-                    a = self._run_layer(L, a_in, B.MODE_REQUANT)
-            st2 = B.read_stats(L.stats)
-            if st2.status != 0:
-                raise B.AdaptionError(st2.status, f"layer {L.name}")
-            rec.append({"type": L.type, "name": L.name, "frac_bits": L.y.frac_bits,
-                        "w_frac_bits": L.w.frac_bits, "max_abs_acc": int(st.max_abs_acc),
-                        "acc_frac_bits": F, "stats": st2})
+        self._cal_x, self._cal_x_fmt, self._cal_in = x_f32, x_fmt, {}
+        try:
+            rec = calibration_loop(self, [L.type for L in self.layers], threshold, group, self.device)
+        finally:
+            self._cal_x, self._cal_in = None, {}
         self.calibrated = True
         return rec
+
+    # ---- backend of calibration_loop: every method is one or two library calls
+    def input_frac_bits(self, threshold: float, group) -> int:
+        x = self._cal_x
+        if self._cal_x_fmt is not None:
+            assert self._cal_x_fmt[0] == self.n_bits
+            return self._cal_x_fmt[1]
+        if threshold > 0:
+            hist = B.new_hist(self.device)
+            B.adaption_bit_histogram(x, hist)
+            total = replicas.sum_histogram(hist.cpu().tolist(), self.device, group)
+            return B.adaption_choose_frac_bits_from_hist(total, self.n_bits, threshold)
+        self.x_max_dev.zero_()
+        B.adaption_measure_range(x, self.n_bits, self.x_max_dev, self.x_fmt_dev)
+        local = float(self.x_max_dev.cpu()[0])
+        agreed = replicas.largest_float(local, self.device, group)
+        if agreed != local:
+            # fold the replicas' maximum in and let the library derive the format from it
+            self.x_max_dev.fill_(agreed)
+            B.adaption_measure_range(x[:0], self.n_bits, self.x_max_dev, self.x_fmt_dev)
+        return int(self.x_fmt_dev.cpu()[1])
+
+    def quantize_input(self, frac_bits: int):
+        self.x_stats.zero_()
+        self.xq.frac_bits = frac_bits
+        B.adaption_quantize(self._cal_x, self.xq.outer, self.xq.inner, self.xq, None, B.ROUND_DETERMINISTIC,
+                            self.x_stats)
+        self._cal_act = self.xq
+        return B.read_stats(self.x_stats)
+
+    def pool(self, i: int) -> int:
+        self._cal_act = self._run_layer(self.layers[i], self._cal_act, B.MODE_REQUANT)
+        return self._cal_act.frac_bits
+
+    def range_pass(self, i: int) -> int:
+        L = self.layers[i]
+        L.stats.zero_()
+        self._cal_in[i] = self._cal_act
+        self._run_layer(L, self._cal_act, B.MODE_RANGE)
+        st = B.read_stats(L.stats)
+        if st.status != 0:
+            raise B.AdaptionError(st.status, f"layer {L.name} (range)")
+        return int(st.max_abs_acc)
+
+    def acc_frac_bits(self, i: int) -> int:
+        return self._cal_in[i].frac_bits + self.layers[i].w.frac_bits
+
+    def choose_from_acc(self, max_abs_acc: int, acc_frac_bits: int) -> int:
+        return B.adaption_choose_frac_bits_from_acc(max_abs_acc, acc_frac_bits, self.n_bits)
+
+    def requant_pass(self, i: int, frac_bits: int):
+        L = self.layers[i]
+        L.y.frac_bits = frac_bits
+        L.stats.zero_()
+        self._cal_act = self._run_layer(L, self._cal_in[i], B.MODE_REQUANT)
+        st = B.read_stats(L.stats)
+        if st.status != 0:
+            raise B.AdaptionError(st.status, f"layer {L.name}")
+        return st
+
+    def width_histogram(self, i: int) -> list[int]:
+        hist = B.new_hist(self.device)
+        B.adaption_width_histogram(self.layers[i].y, hist)
+        return hist.cpu().tolist()
+
+    def choose_from_widths(self, hist: list[int], frac_bits: int, threshold: float) -> int:
+        return B.adaption_choose_frac_bits_from_widths(hist, frac_bits, self.n_bits, threshold)
+
+    def layer_name(self, i: int) -> str:
+        return self.layers[i].name
+
+    def w_frac_bits(self, i: int) -> int:
+        return self.layers[i].w.frac_bits
 
     def set_formats(self, x_frac_bits: int, layer_frac_bits: list[int]):
         """Fix the decimal points without a calibration run (formats chosen elsewhere, e.g. on another

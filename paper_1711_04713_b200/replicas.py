@@ -31,6 +31,25 @@ def sum_counters(zeros: int, sat_pos: int, sat_neg: int, device="cpu", group=Non
     return int(t[0]), int(t[1]), int(t[2])
 
 
+def largest_float(value: float, device="cpu", group=None) -> float:
+    """Largest value over all replicas (the input's max |x| during calibration)."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float32, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
+    return float(t[0])
+
+
+def sum_histogram(hist, device="cpu", group=None) -> list[int]:
+    """Bin-wise sum of a bit-occupancy histogram over all replicas (thresholded allocation)."""
+    hist = [int(v) for v in hist]
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return hist
+    t = torch.tensor(hist, dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+    return [int(v) for v in t.tolist()]
+
+
 def slowest_rank_ms(elapsed_ms: float, device="cpu", group=None) -> float:
     """A multi-GPU step takes as long as its slowest replica."""
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:

@@ -10,6 +10,8 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
+    config.addinivalue_line("markers", "slow: full-size workload (the oracle takes seconds to minutes); "
+                                       "part of -m gpu, deselect with -m 'gpu and not slow'")
 
 
 def _have_gpu() -> bool:

@@ -9,9 +9,17 @@ import torch
 
 from oracle import reference as orc
 from paper_1711_04713_b200 import binding as B
-from tests.util import dev, from_qtensor, q16_of, stats_tuple, to_qtensor
+from tests.util import Guards, dev, from_qtensor, q16_of, stats_tuple, to_qtensor
 
 pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _default_overrides():
+    """Every test starts from and leaves behind the library's default heuristics."""
+    B.adaption_debug_set("reset")
+    yield
+    B.adaption_debug_set("reset")
 
 
 def _rand_q(rng, shape, n_bits, zero_frac=0.0):
@@ -49,14 +57,12 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
     x = to_qtensor(xq.reshape(-1, Cin), nx, fx, cs)
     w = to_qtensor(wq.reshape(-1, Cin), nw, fw, cs)
     ycs = B.pad_to(K, 32)
-    y = B.QTensor.empty(N * OH * OW, K, n_out, f_out, ycs, with_q16=with_q16)
-    y.lo.fill_(0x3C)
-    if y.hi is not None:
-        y.hi.fill_(0x3C)
+    guards = Guards()         # canaries around the output planes and the workspace
+    y = guards.qtensor(N * OH * OW, K, n_out, f_out, ycs, with_q16=with_q16)
     shp = B.conv_shape(N, H, W, Cin, K, R, R, pad, stride)
     bias_dev = dev(bq) if with_bias else None
     need = B.adaption_lp_conv_workspace_bytes(shp, x.fmt(), w.fmt(), cs, algo)
-    ws = torch.empty(max(need, 16) + ws_offset, dtype=torch.uint8, device="cuda")[ws_offset:] if need else None
+    ws = guards.alloc(max(need, 16) + ws_offset)[ws_offset:] if need else None
     st = B.new_stats()
     B.adaption_lp_conv_fwd(shp, x, w, bias_dev, fw, relu, B.MODE_RANGE, algo, None, st, ws)
     s = B.read_stats(st)
@@ -74,6 +80,7 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
         assert np.array_equal(q16_of(y).reshape(want.shape), want)
     assert y.padding_is_zero()
     assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+    guards.check()
     return cnt
 
 
@@ -89,13 +96,11 @@ def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out
     want, cnt = orc.epilogue(acc, bq, fw, F, relu, n_out, f_out)
     x = to_qtensor(xq, nx, fx)
     w = to_qtensor(wq, nw, fw)
-    y = B.QTensor.empty(Bsz, O, n_out, f_out, None, with_q16=with_q16)
-    y.lo.fill_(0x3C)
-    if y.hi is not None:
-        y.hi.fill_(0x3C)
+    guards = Guards()
+    y = guards.qtensor(Bsz, O, n_out, f_out, None, with_q16=with_q16)
     bias_dev = dev(bq) if with_bias else None
     need = B.adaption_lp_ip_workspace_bytes(Bsz, K, O, x.fmt(), w.fmt(), algo)
-    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+    ws = guards.alloc(max(need, 16)) if need else None
     st = B.new_stats()
     B.adaption_lp_ip_fwd(Bsz, K, O, x, w, bias_dev, fw, relu, B.MODE_RANGE, algo, None, st, ws)
     s = B.read_stats(st)
@@ -111,6 +116,7 @@ def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out
         assert np.array_equal(q16_of(y), want)
     assert y.padding_is_zero()
     assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+    guards.check()
     return need
 
 
@@ -166,10 +172,10 @@ TC_CONV = [
 
 
 @pytest.fixture(params=["single", "pair"])
-def cta_mode(request, monkeypatch):
+def cta_mode(request, _default_overrides):
     """Run a tensor-core case with one CTA per 128-row tile and with CTA pairs on 256-row tiles
     (cross-path identity: both must give the oracle's bits)."""
-    monkeypatch.setenv("ADAPTION_TC_PAIR", "1" if request.param == "pair" else "0")
+    B.adaption_debug_set("pair", 1 if request.param == "pair" else 0)
     return request.param
 
 
@@ -225,13 +231,13 @@ def test_single_pass_fast_epilogue_every_shift(shift, n_out, K, Cin, cta_mode):
         assert cnt.sat_pos > 0   # the case does exercise saturation
 
 
-def test_epilogue_variants_agree(monkeypatch):
+def test_epilogue_variants_agree():
     """Cross-path identity: the generic 64-bit epilogue with direct stores, the staged stores and the
     fast paired path all give the oracle's bits on the same case."""
     case = (2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True)
-    for fast, staged in (("0", "0"), ("0", "1"), ("1", "0"), ("1", "1")):
-        monkeypatch.setenv("ADAPTION_TC_FAST", fast)
-        monkeypatch.setenv("ADAPTION_TC_STAGED", staged)
+    for fast, staged in ((0, 0), (0, 1), (1, 0), (1, 1)):
+        B.adaption_debug_set("fast", fast)
+        B.adaption_debug_set("staged", staged)
         run_conv_case(np.random.default_rng(5), *case, B.ALGO_TENSOR, with_q16=False, mag_bits=(10, 10))
 
 
@@ -301,9 +307,9 @@ WIDE_CONV = [
 
 @pytest.mark.parametrize("case", WIDE_CONV)
 @pytest.mark.parametrize("with_q16", [False, True])
-@pytest.mark.parametrize("wide", ["1", "0"])
-def test_conv_single_pass_wide_tiles(case, with_q16, wide, monkeypatch):
-    monkeypatch.setenv("ADAPTION_TC_WIDE", wide)
+@pytest.mark.parametrize("wide", [1, 0])
+def test_conv_single_pass_wide_tiles(case, with_q16, wide):
+    B.adaption_debug_set("wide", wide)
     run_conv_case(np.random.default_rng(sum(case)), *case, B.ALGO_TENSOR, with_q16=with_q16)
 
 
@@ -312,12 +318,12 @@ def test_ip_single_pass_wide_tiles():
     run_ip_case(np.random.default_rng(78), 2048, 2304, 256, 8, 8, 8, False, B.ALGO_TENSOR, with_q16=True)
 
 
-@pytest.mark.parametrize("groups", ["1", "2"])
+@pytest.mark.parametrize("groups", [1, 2])
 @pytest.mark.parametrize("with_q16", [False, True])
-def test_epilogue_groups_agree(groups, with_q16, monkeypatch):
+def test_epilogue_groups_agree(groups, with_q16):
     """Narrow tiles (two accumulator sets in TMEM): one group of epilogue warps, or two groups taking
     alternate tiles, give the same bits; odd and even tile counts per CTA, ReLU and signed outputs."""
-    monkeypatch.setenv("ADAPTION_TC_EPIGROUPS", groups)
+    B.adaption_debug_set("epigroups", groups)
     for case in [(5, 40, 40, 64, 64, 3, 1, 1, 16, 16, 16, True),       # 63 tiles of 128 x 64
                  (2, 30, 30, 256, 48, 3, 1, 1, 16, 16, 16, False),     # signed outputs, ragged N
                  (37, 64, 64, 32, 32, 3, 1, 1, 16, 16, 8, True),       # BN = 32, more tiles than CTAs
@@ -336,15 +342,12 @@ def test_ip_tensor_split_k_paths():
     need = run_ip_case(np.random.default_rng(11), 64, 25088, 256, 16, 16, 16, True, B.ALGO_TENSOR)
     assert need == 64 * 256 * 8
     # forcing other split factors gives the same bits
-    for splits in ("3", "7"):
-        os.environ["ADAPTION_TC_SPLITS"] = splits
-        try:
-            need = run_ip_case(np.random.default_rng(12), 40, 2048, 200, 16, 16, 16, False, B.ALGO_TENSOR)
-            assert need == 40 * 200 * 8
-            run_conv_case(np.random.default_rng(13), 2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True,
-                          B.ALGO_TENSOR)
-        finally:
-            del os.environ["ADAPTION_TC_SPLITS"]
+    for splits in (3, 7):
+        B.adaption_debug_set("splits", splits)
+        need = run_ip_case(np.random.default_rng(12), 40, 2048, 200, 16, 16, 16, False, B.ALGO_TENSOR)
+        assert need == 40 * 200 * 8
+        run_conv_case(np.random.default_rng(13), 2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True,
+                      B.ALGO_TENSOR)
 
 
 def test_workspace_too_small_is_rejected():
@@ -443,12 +446,12 @@ def test_conv_with_fused_pool(case, with_q16):
     OH, OW = acc.shape[1], acc.shape[2]
     x = to_qtensor(xq.reshape(-1, Cin), nx, fx, cs)
     w = to_qtensor(wq.reshape(-1, Cin), nw, fw, cs)
-    y = B.QTensor.empty(N * (OH // 2) * (OW // 2), K, n_out, f_out, B.pad_to(K, 16), with_q16=with_q16)
-    y.lo.fill_(0x3C)
+    guards = Guards()
+    y = guards.qtensor(N * (OH // 2) * (OW // 2), K, n_out, f_out, B.pad_to(K, 16), with_q16=with_q16)
     shp = B.conv_shape(N, H, W, Cin, K, R, R, pad, stride)
     need = B.adaption_lp_conv_pool_workspace_bytes(shp, x.fmt(), w.fmt(), y.fmt(), cs, y.c_stride, B.ALGO_AUTO)
     assert need > 0
-    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    ws = guards.alloc(need)
     st = B.new_stats()
     B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st, ws)
     assert B.read_stats(st).status == 0
@@ -469,3 +472,77 @@ def test_conv_with_fused_pool(case, with_q16):
     for bad_phases in (0, 4):
         with pytest.raises(B.AdaptionError):
             B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st2, ws, bad_phases)
+    guards.check()
+
+
+# ------------------------------------------------------------------ robustness of the boundary
+@pytest.mark.parametrize("mode", ["single", "pair"])
+@pytest.mark.parametrize("stall_at", [0, 5])
+def test_device_side_wait_runs_out_and_the_next_call_is_exact(mode, stall_at):
+    """Failure detection without a fault: the copy-issuing warps are told to stop before one of their
+    stages (nothing is in flight for it), the waits of the other warps run out after a few
+    milliseconds, the kernel flags ADAPTION_ERR_TIMEOUT in the caller's stats word, drains, frees its
+    tensor memory and returns.  The context stays usable: the same call without the stall gives the
+    oracle's bits."""
+    case = (4, 16, 16, 128, 128, 3, 1, 1, 16, 16, 16, True)       # four tiles of 256 rows / eight of 128
+    N, H, W, Cin, K = case[:5]
+    rng = np.random.default_rng(21)
+    xq, wq = _rand_q(rng, (N, H, W, Cin), 16, 0.4), _rand_q(rng, (K, 3, 3, Cin), 16)
+    x, w = to_qtensor(xq.reshape(-1, Cin), 16, 13, Cin), to_qtensor(wq.reshape(-1, Cin), 16, 15, Cin)
+    shp = B.conv_shape(N, H, W, Cin, K, 3, 3, 1, 1)
+    y = B.QTensor.empty(N * H * W, K, 16, 5, K)
+    B.adaption_debug_set("pair", 1 if mode == "pair" else 0)
+    B.adaption_debug_set("timeout_us", 3000)
+    B.adaption_debug_set("stall_at", stall_at)
+    st = B.new_stats()
+    B.adaption_lp_conv_fwd(shp, x, w, None, 0, True, B.MODE_REQUANT, B.ALGO_TENSOR, y, st, None)
+    torch.cuda.synchronize()                                   # the kernel returned by itself
+    assert B.read_stats(st).status == B.ERR_TIMEOUT
+    assert B.status_string(B.read_stats(st).status) == "device-side wait timed out"
+    B.adaption_debug_set("stall_at", -1)
+    B.adaption_debug_set("timeout_us", 0)
+    run_conv_case(np.random.default_rng(22), *case, B.ALGO_TENSOR, with_q16=False)
+
+
+def test_left_shift_of_accumulators_beyond_2_to_the_48():
+    """An inner product long enough for |acc| = 2^48 (262144 products of -32768 * -32768) requantized
+    to MORE fractional bits than the accumulator has: the exact product acc * 2^15 does not fit 64 bits
+    and must still saturate (both kernels)."""
+    Bsz, K, O = 2, 1 << 18, 3
+    xq = np.full((Bsz, K), -32768, dtype=np.int16)
+    xq[1, :] = 32767
+    wq = np.full((O, K), -32768, dtype=np.int16)
+    wq[2, :] = 0
+    wq[2, 0] = 1
+    want, cnt = orc.epilogue(orc.ip_acc(xq, wq), None, 0, 0, False, 16, 15)
+    assert want.tolist() == [[32767, 32767, -32768], [-32768, -32768, 32767]]
+    x, w = to_qtensor(xq, 16, 0), to_qtensor(wq, 16, 0)
+    for algo in (B.ALGO_DIRECT, B.ALGO_TENSOR):
+        need = B.adaption_lp_ip_workspace_bytes(Bsz, K, O, x.fmt(), w.fmt(), algo)
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda") if need else None
+        y = B.QTensor.empty(Bsz, O, 16, 15)
+        st = B.new_stats()
+        B.adaption_lp_ip_fwd(Bsz, K, O, x, w, None, 0, False, B.MODE_REQUANT, algo, y, st, ws)
+        assert np.array_equal(from_qtensor(y), want)
+        assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
+
+
+def test_layer_calls_from_two_host_threads():
+    """The library keeps no per-call state: two host threads, each with its own stream and buffers,
+    run different layers at the same time and both get the oracle's bits."""
+    import threading
+    errors = []
+
+    def work(seed, case):
+        try:
+            torch.cuda.set_device(0)
+            with torch.cuda.stream(torch.cuda.Stream()):
+                for rep in range(3):
+                    run_conv_case(np.random.default_rng(seed + rep), *case, B.ALGO_TENSOR, with_q16=False)
+        except Exception as exc:                              # noqa: BLE001 - reported to the main thread
+            errors.append(exc)
+
+    t1 = threading.Thread(target=work, args=(31, (2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True)))
+    t2 = threading.Thread(target=work, args=(41, (5, 30, 30, 64, 64, 3, 1, 1, 16, 16, 16, True)))
+    t1.start(); t2.start(); t1.join(); t2.join()
+    assert not errors, errors

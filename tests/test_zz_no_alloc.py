@@ -15,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import reference as orc
 from paper_1711_04713_b200 import binding as B
 from tests.util import dev, from_qtensor, stats_tuple, to_qtensor
 
@@ -27,17 +28,21 @@ def _case(seed, Bsz, K, O, relu):
     xq[rng.random(xq.shape) < 0.4] = 0
     wq = rng.integers(-32768, 32768, (O, K)).astype(np.int16)
     bq = rng.integers(-32768, 32768, (O,)).astype(np.int16)
-    return to_qtensor(xq, 16, 12), to_qtensor(wq, 16, 15), dev(bq)
+    return to_qtensor(xq, 16, 12), to_qtensor(wq, 16, 15), dev(bq), (xq, wq, bq)
 
 
-def _run_both(seed, Bsz, K, O, relu, f_out):
-    x, w, bias = _case(seed, Bsz, K, O, relu)
+def _run_both(seed, Bsz, K, O, relu, f_out, uses_scratch=True):
+    x, w, bias, host = _case(seed, Bsz, K, O, relu)
     need = B.adaption_lp_ip_workspace_bytes(Bsz, K, O, x.fmt(), w.fmt(), B.ALGO_TENSOR)
-    assert 0 < need <= B.STATIC_WORKSPACE_BYTES          # the split-K (scratch-using) path is exercised
+    if uses_scratch:
+        assert 0 < need <= B.STATIC_WORKSPACE_BYTES      # the split-K (scratch-using) path is exercised
+    else:
+        assert need == 0                                 # an unsplit reduction: the array is not touched
+    ws_bytes = max(need, 16)
     # regular entry point, caller-owned workspace
     y_ref = B.QTensor.empty(Bsz, O, 16, f_out, None, with_q16=True)
     st_ref = B.new_stats()
-    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     B.adaption_lp_ip_fwd(Bsz, K, O, x, w, bias, 15, relu, B.MODE_REQUANT, B.ALGO_TENSOR, y_ref, st_ref, ws)
     rg_ref = B.new_stats()
     B.adaption_lp_ip_fwd(Bsz, K, O, x, w, bias, 15, relu, B.MODE_RANGE, B.ALGO_TENSOR, None, rg_ref, ws)
@@ -54,6 +59,11 @@ def _run_both(seed, Bsz, K, O, relu, f_out):
     assert torch.equal(y.q16, y_ref.q16)
     assert stats_tuple(st) == stats_tuple(st_ref)
     assert int(B.read_stats(rg).max_abs_acc) == int(B.read_stats(rg_ref).max_abs_acc) > 0
+    # and against the CPU oracle directly, not only through the regular entry point
+    xq, wq, bq = host
+    want, cnt = orc.epilogue(orc.ip_acc(xq, wq), bq, 15, 27, relu, 16, f_out)
+    assert np.array_equal(from_qtensor(y), want)
+    assert stats_tuple(st) == (cnt.zeros, cnt.sat_pos, cnt.sat_neg)
     return from_qtensor(y)
 
 
@@ -62,6 +72,19 @@ def test_static_workspace_matches_regular_entry_point_twice_in_a_row():
     second = _run_both(2, 48, 8192, 200, False, 3)       # other shape and data on the same scratch
     assert first.shape == (64, 256) and second.shape == (48, 200)
     assert first.any() and second.any()
+
+
+def test_shapes_without_scratch_and_calls_on_another_stream():
+    """A reduction short enough to stay unsplit needs no scratch (the entry point then passes none on);
+    and the entry point honours the caller's stream like every other call."""
+    _run_both(3, 256, 512, 384, True, 4, uses_scratch=False)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        out = _run_both(4, 64, 25088, 256, True, 2)
+    side.synchronize()
+    torch.cuda.current_stream().wait_stream(side)
+    assert out.any()
 
 
 def test_shape_beyond_the_built_in_scratch_is_refused():
