@@ -128,3 +128,43 @@ def requantize_stochastic(xq, in_frac_bits: int, relu: bool, out_n_bits: int, ou
     sat_neg = int((r < qmin).sum())
     y = np.clip(r, qmin, qmax)
     return y.astype(np.int16).reshape(q.shape), (int((y == 0).sum()), sat_pos, sat_neg)
+
+
+def epilogue_stochastic(acc, bias_q, bias_frac_bits: int, acc_frac_bits: int, relu: bool, out_n_bits: int,
+                        out_frac_bits: int, seed: int):
+    """Epilogue of an LP layer whose rounding_scheme is STOCHASTIC (paper Sec. 2: a per-layer
+    parameter; Sec. 2.4): bias, ReLU, then the pre-activation value v (an integer in units of
+    2^-acc_frac_bits) is brought to the output format by one of its two neighbouring codes.
+    Readings (the paper gives no formula), in line with S1-S2 above:
+    E1  s = acc_frac_bits - out_frac_bits.  For s > 0, v / 2^s = q + rem / 2^s with q = floor(v / 2^s)
+        and 0 <= rem < 2^s, all integers; the result is q + 1 with probability T / 2^32,
+        T = rem * 2^(32 - s) (exact: s <= 30 because both operand formats have at most 15
+        fractional bits), else q.  rem = 0 never moves.  For s <= 0 the left shift is exact.
+    E2  The draw of the output with row-major index i over acc's [outer][channels] elements is the
+        word R_i of reading S2 (same generator, same key = seed); the value moves up iff R_i < T.
+    E3  Saturation and the three counters as in the deterministic epilogue, after the rounding.
+    acc: int64 array [..., channels]; returns (int16 array, (zeros, sat_pos, sat_neg))."""
+    acc = np.ascontiguousarray(acc, dtype=np.int64)
+    ch = acc.shape[-1]
+    v = acc.reshape(-1, ch).copy()
+    if bias_q is not None:
+        b = np.asarray(bias_q, dtype=np.int64).reshape(1, ch)
+        v = v + b * np.int64(1 << (acc_frac_bits - bias_frac_bits))
+    if relu:
+        v = np.maximum(v, 0)
+    v = v.reshape(-1)
+    s = acc_frac_bits - out_frac_bits
+    qmin, qmax = -(1 << (out_n_bits - 1)), (1 << (out_n_bits - 1)) - 1
+    if s > 0:
+        assert s <= 32
+        q = v >> s                                    # floor (arithmetic shift)
+        rem = v - (q << s)                            # 0 <= rem < 2^s
+        T = rem.astype(np.uint64) << np.uint64(32 - s)
+        r = q + (draws(v.size, seed) < T).astype(np.int64)
+    else:
+        lim = np.int64(1) << np.int64(40)             # beyond any output range after the shift
+        r = np.clip(v, -lim, lim) << np.int64(-s)
+    sat_pos = int((r > qmax).sum())
+    sat_neg = int((r < qmin).sum())
+    y = np.clip(r, qmin, qmax)
+    return y.astype(np.int16).reshape(acc.shape), (int((y == 0).sum()), sat_pos, sat_neg)

@@ -747,3 +747,56 @@ def test_stochastic_requantization_support_expectation_and_exact_cases():
         assert np.all(np.abs(ys.astype(np.int64) - yd.astype(np.int64)) <= 1)
         assert z == int((ys == 0).sum()) and sn == (0 if relu else sn)
         assert abs(sp - cd.sat_pos) <= int((np.abs(q.astype(np.int64) - 127 * 512) < 512).sum()) + 1
+
+
+def test_stochastic_epilogue_handworked_support_expectation_and_exact_cases():
+    """The fused layer epilogue with stochastic rounding (Sec. 2 rounding_scheme, Sec. 2.4):
+    hand-worked outcomes from the generator's own draws, support on the two neighbours, unbiased
+    mean, values on the grid never move, exact left shifts, bias / ReLU / saturation / counters as
+    in the deterministic epilogue, and agreement with the (separately pinned) format change of a
+    stored tensor where the two coincide."""
+    from oracle import stochastic as st
+    # hand-worked: four outputs in one row, s = 3, bias 1 * 2^2 added to every accumulator
+    seed = 2024
+    R = [int(v) for v in st.draws(4, seed)]                   # pinned by the known-answer vectors
+    acc = np.array([[5, -5, 16, 1]], dtype=np.int64)          # + 4 -> 9, -1, 20, 5
+    y, cnt = st.epilogue_stochastic(acc, np.array([1, 1, 1, 1], dtype=np.int16), 1, 3, False, 16, 0, seed)
+    want = []
+    for v, r in zip([9, -1, 20, 5], R):
+        fl = Fraction(v, 8).numerator // Fraction(v, 8).denominator
+        frac = Fraction(v, 8) - fl
+        want.append(fl + (1 if r < int(frac * (1 << 32)) else 0))
+    assert y.tolist() == [want]
+    assert all(t in pair for t, pair in zip(want, [(1, 2), (-1, 0), (2, 3), (0, 1)]))
+    assert cnt[0] == sum(1 for t in want if t == 0)
+    # support and expectation over many draws, positive and negative values, with ReLU and without
+    vals = np.array([5, -5, 1, -1, 1023, -1023, 123457, -123457, 7, 64], dtype=np.int64)
+    reps = 20000
+    y, _ = st.epilogue_stochastic(np.tile(vals, (reps, 1)), None, 0, 20, False, 16, 14, seed=11)   # s = 6
+    y = y.astype(np.float64)
+    exact = vals.astype(np.float64) / 64.0
+    assert np.all((y == np.floor(exact)) | (y == np.floor(exact) + 1))
+    assert np.all(np.abs(y.mean(axis=0) - exact) < 5 * np.sqrt(0.25 / reps))
+    assert np.all(y[:, 9] == 1.0)                             # 64 / 64: on the grid
+    yr, _ = st.epilogue_stochastic(np.tile(vals, (200, 1)), None, 0, 20, True, 16, 14, seed=12)
+    assert np.all(yr[:, [1, 3, 5, 7]] == 0)                   # ReLU before rounding: negatives are exactly 0
+    # grid values never move; left shifts are exact; huge accumulators saturate
+    grid = (np.arange(-300, 300, dtype=np.int64) * 32).reshape(1, -1)
+    yg, _ = st.epilogue_stochastic(grid, None, 0, 5, False, 16, 0, seed=3)
+    assert np.array_equal(yg.reshape(-1), np.arange(-300, 300))
+    up, c = st.epilogue_stochastic(np.array([[3, -3, 2 ** 50, -(2 ** 50), 0]], dtype=np.int64), None, 0, 2, False,
+                                   16, 4, seed=4)
+    assert up.tolist() == [[12, -12, 32767, -32768, 0]] and c == (1, 1, 1)
+    # same rule as the stored-tensor format change where both apply (16-bit values, no bias)
+    rng = np.random.default_rng(6)
+    q = rng.integers(-32768, 32768, (37, 24)).astype(np.int16)
+    for relu in (False, True):
+        a, ca = st.epilogue_stochastic(q.astype(np.int64), None, 0, 12, relu, 8, 3, seed=77)
+        b, cb = st.requantize_stochastic(q, 12, relu, 8, 3, seed=77)
+        assert np.array_equal(a, b) and ca == cb
+    # never further than one step from the deterministic epilogue, equal where rem = 0
+    accr = rng.integers(-(2 ** 34), 2 ** 34, (50, 16)).astype(np.int64)
+    bq = rng.integers(-32768, 32768, 16).astype(np.int16)
+    ys, _ = st.epilogue_stochastic(accr, bq, 15, 28, True, 16, 9, seed=8)
+    yd, _ = orc.epilogue(accr, bq, 15, 28, True, 16, 9)
+    assert np.all(np.abs(ys.astype(np.int64) - yd.astype(np.int64)) <= 1)
