@@ -202,6 +202,28 @@ ADAPTION_API int adaption_lp_conv_fwd(const adaption_conv_shape* h_shape, adapti
                          adaption_stats* d_stats, void* d_workspace, size_t workspace_bytes,
                          void* stream);
 
+/* Sec. 2 (rounding_scheme is a parameter of every LP layer) + Sec. 2.4: the layer calls with
+ * stochastic rounding in the fused requantization.  As adaption_lp_conv_fwd / adaption_lp_ip_fwd in
+ * ADAPTION_MODE_REQUANT (same workspace queries), except for the rounding of the pre-activation value
+ * v (accumulator + bias, after ReLU), an integer in units of 2^-F with F = x.fmt.frac_bits +
+ * w.fmt.frac_bits: with s = F - y.fmt.frac_bits > 0, v / 2^s = q + rem / 2^s (q = floor, 0 <= rem <
+ * 2^s) becomes q + 1 with probability rem / 2^s and q otherwise, so that the expectation is the
+ * unrounded value and a value on the output grid never moves; for s <= 0 the shift is exact.  The
+ * draw of output element i (row-major index over the real [M][K] outputs, M = N*OH*OW pixels or B
+ * rows) is word i & 3 of Philox4x32-10 with counter (i >> 2, 0, 0) and key `seed`, and the value
+ * moves up iff draw < rem * 2^(32 - s): a pure function of (operands, formats, seed), whatever
+ * kernel or tile shape runs the layer.  Saturation and counters as in the deterministic calls. */
+ADAPTION_API int adaption_lp_conv_fwd_stochastic(const adaption_conv_shape* h_shape, adaption_qtensor x,
+                                    adaption_qtensor w, const int16_t* d_bias_q, int32_t bias_frac_bits,
+                                    int32_t relu, int32_t algo, adaption_qtensor y, uint64_t seed,
+                                    adaption_stats* d_stats, void* d_workspace, size_t workspace_bytes,
+                                    void* stream);
+ADAPTION_API int adaption_lp_ip_fwd_stochastic(int64_t B, int64_t K, int64_t O, adaption_qtensor x,
+                                  adaption_qtensor w, const int16_t* d_bias_q, int32_t bias_frac_bits,
+                                  int32_t relu, int32_t algo, adaption_qtensor y, uint64_t seed,
+                                  adaption_stats* d_stats, void* d_workspace, size_t workspace_bytes,
+                                  void* stream);
+
 /* Sec. 2 + Table 1 "Pooling" (LPConvolution followed by the 2x2 / stride-2 max-pool of its output,
  * as in VGG16 and Giga1Net).  y is the pooled tensor [N, OH/2, OW/2, K] in the layer's output format;
  * OH and OW must be even.  The result equals adaption_lp_conv_fwd followed by adaption_maxpool2x2

@@ -276,8 +276,25 @@ def _thresholded_fmt(t, n_bits: int, threshold: float) -> int:
     return ba.choose_frac_bits(ba.bit_histogram(t), n_bits, threshold)
 
 
-def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None, threshold: float = 0.0):
+def rounding_seeds(rounding_seed: int, layer_index: int | None):
+    """Seeds of the stochastic-rounding draws of one network pass (Sec. 2.4): every tensor that is
+    rounded gets its own stream.  Input: base; layer li (counting conv / inner-product layers from 0):
+    weights base + 16 li + 1, biases base + 16 li + 2, output base + 16 li + 3, with
+    base = rounding_seed * 1000003, all modulo 2^64."""
+    base = (int(rounding_seed) * 1000003) & 0xFFFFFFFFFFFFFFFF
+    if layer_index is None:
+        return base
+    return tuple((base + 16 * layer_index + k) & 0xFFFFFFFFFFFFFFFF for k in (1, 2, 3))
+
+
+def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None, threshold: float = 0.0,
+                rounding_seed: int | None = None):
     """Forward pass of a stack of LP layers on a batch.
+
+    ``rounding_seed`` not None: every LP layer's rounding_scheme is STOCHASTIC (Sec. 2, Sec. 2.4):
+    the input, the weights, the biases and every layer output are rounded stochastically with the
+    seeds of ``rounding_seeds``; decimal points still come from the measured ranges (of the unrounded
+    values), and pooling is unaffected.
 
     ``threshold`` > 0 (only without ``fixed_formats``): decimal points by the thresholded allocation
     of Sec. 2.3 instead of the maximum: fp32 tensors (input, weights) from their bit-occupancy
@@ -299,7 +316,12 @@ def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None, threshold: fl
         nx = n_bits
     else:
         nx, fx = x_fmt
-    a, cnt = quantize(x, nx, fx)
+    if rounding_seed is not None:
+        from . import stochastic as st
+        a, c3 = st.quantize_stochastic(x, nx, fx, rounding_seeds(rounding_seed, None))
+        cnt = Counters(*c3)
+    else:
+        a, cnt = quantize(x, nx, fx)
     records.append({"type": "input", "y": a, "n_bits": nx, "frac_bits": fx, "counters": cnt})
     li = 0
     for L in layers:
@@ -313,18 +335,32 @@ def run_network(layers, x, x_fmt, n_bits: int, fixed_formats=None, threshold: fl
         else:
             wq, fw = quantize_param(L["w"], n_bits)
         bq, _ = quantize(L["b"], n_bits, fw)
+        if rounding_seed is not None:
+            sw, sb, sy = rounding_seeds(rounding_seed, li)
+            wq, _ = st.quantize_stochastic(L["w"], n_bits, fw, sw)
+            bq, _ = st.quantize_stochastic(L["b"], n_bits, fw, sb)
         if L["type"] == "conv":
             p, s = L["pad"], L["stride"]
             acc = conv_acc(a, wq, (p, p), (s, s))
         else:
             acc = ip_acc(a.reshape(a.shape[0], -1), wq)
         f_out = None if fixed_formats is None else fixed_formats[li]
-        res = lp_layer(acc, fx, fw, bq, fw, L["relu"], n_bits, f_out)
+
+        def layer_with(f):
+            """Epilogue with the given output decimal point (None: chosen from the measured range),
+            rounding as the network's rounding_scheme says."""
+            r = lp_layer(acc, fx, fw, bq, fw, L["relu"], n_bits, f)
+            if rounding_seed is None:
+                return r
+            y, c3 = st.epilogue_stochastic(acc, bq, fw, fx + fw, L["relu"], n_bits, r.frac_bits, sy)
+            return LayerResult(y, n_bits, r.frac_bits, Counters(*c3), r.max_abs_acc, r.acc_frac_bits)
+
+        res = layer_with(f_out)
         if threshold > 0 and fixed_formats is None:
             from . import bit_allocation as ba
             m = ba.choose_int_bits_from_widths(ba.width_histogram(res.y), res.frac_bits, n_bits, threshold)
             if n_bits - 1 - m != res.frac_bits:
-                res = lp_layer(acc, fx, fw, bq, fw, L["relu"], n_bits, n_bits - 1 - m)
+                res = layer_with(n_bits - 1 - m)
         records.append({"type": L["type"], "y": res.y, "n_bits": n_bits, "frac_bits": res.frac_bits,
                         "w_frac_bits": fw, "wq": wq, "bq": bq, "counters": res.counters,
                         "max_abs_acc": res.max_abs_acc, "acc_frac_bits": res.acc_frac_bits})

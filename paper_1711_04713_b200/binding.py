@@ -57,7 +57,8 @@ EXPORTS = [
     "adaption_quantize_stochastic", "adaption_bit_histogram", "adaption_width_histogram",
     "adaption_choose_frac_bits_from_hist", "adaption_choose_frac_bits_from_widths",
     "adaption_lp_act_stochastic", "adaption_lp_conv_pool_workspace_bytes", "adaption_lp_conv_pool_fwd",
-    "adaption_quantize_batch", "adaption_debug_set",
+    "adaption_quantize_batch", "adaption_debug_set", "adaption_lp_conv_fwd_stochastic",
+    "adaption_lp_ip_fwd_stochastic",
 ]
 HIST_BINS = 17
 
@@ -90,6 +91,11 @@ def load(path: str | None = None):
     lib.adaption_lp_conv_fwd.argtypes = [C.POINTER(adaption_conv_shape), adaption_qtensor, adaption_qtensor,
                                          P, I32, I32, I32, I32, adaption_qtensor, P, P, SZ, P]
     lib.adaption_quantize_batch.argtypes = [C.POINTER(adaption_quantize_item), I32, P]
+    lib.adaption_lp_conv_fwd_stochastic.argtypes = [C.POINTER(adaption_conv_shape), adaption_qtensor,
+                                                    adaption_qtensor, P, I32, I32, I32, adaption_qtensor,
+                                                    C.c_uint64, P, P, SZ, P]
+    lib.adaption_lp_ip_fwd_stochastic.argtypes = [I64, I64, I64, adaption_qtensor, adaption_qtensor, P, I32, I32,
+                                                  I32, adaption_qtensor, C.c_uint64, P, P, SZ, P]
     lib.adaption_lp_conv_pool_workspace_bytes.argtypes = [C.POINTER(adaption_conv_shape), adaption_qfmt,
                                                           adaption_qfmt, adaption_qfmt, I64, I64, I32]
     lib.adaption_lp_conv_pool_workspace_bytes.restype = SZ
@@ -315,6 +321,26 @@ def adaption_lp_conv_fwd(shape: adaption_conv_shape, x: QTensor, w: QTensor, bia
     _check(load().adaption_lp_conv_fwd(C.byref(shape), x.c_struct(), w.c_struct(), _ptr(bias_q),
                                        bias_frac_bits, int(relu), mode, algo, ys, _ptr(d_stats),
                                        _ptr(workspace), wsb, _stream()), "adaption_lp_conv_fwd")
+
+
+def adaption_lp_conv_fwd_stochastic(shape: adaption_conv_shape, x: QTensor, w: QTensor, bias_q: torch.Tensor | None,
+                                    bias_frac_bits: int, relu: bool, algo: int, y: QTensor, seed: int,
+                                    d_stats: torch.Tensor, workspace: torch.Tensor | None = None):
+    wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().adaption_lp_conv_fwd_stochastic(C.byref(shape), x.c_struct(), w.c_struct(), _ptr(bias_q),
+                                                  bias_frac_bits, int(relu), algo, y.c_struct(),
+                                                  seed & 0xFFFFFFFFFFFFFFFF, _ptr(d_stats), _ptr(workspace), wsb,
+                                                  _stream()), "adaption_lp_conv_fwd_stochastic")
+
+
+def adaption_lp_ip_fwd_stochastic(B: int, K: int, O: int, x: QTensor, w: QTensor, bias_q: torch.Tensor | None,
+                                  bias_frac_bits: int, relu: bool, algo: int, y: QTensor, seed: int,
+                                  d_stats: torch.Tensor, workspace: torch.Tensor | None = None):
+    wsb = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().adaption_lp_ip_fwd_stochastic(B, K, O, x.c_struct(), w.c_struct(), _ptr(bias_q), bias_frac_bits,
+                                                int(relu), algo, y.c_struct(), seed & 0xFFFFFFFFFFFFFFFF,
+                                                _ptr(d_stats), _ptr(workspace), wsb, _stream()),
+           "adaption_lp_ip_fwd_stochastic")
 
 
 def adaption_lp_conv_pool_workspace_bytes(shape: adaption_conv_shape, fx: adaption_qfmt, fw: adaption_qfmt,

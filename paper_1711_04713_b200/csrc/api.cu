@@ -277,6 +277,18 @@ int adaption_lp_conv_fwd(const adaption_conv_shape* h_shape, adaption_qtensor x,
   return dispatch(g, algo);
 }
 
+int adaption_lp_conv_fwd_stochastic(const adaption_conv_shape* h_shape, adaption_qtensor x, adaption_qtensor w,
+                                    const int16_t* d_bias_q, int32_t bias_frac_bits, int32_t relu, int32_t algo,
+                                    adaption_qtensor y, uint64_t seed, adaption_stats* d_stats, void* d_workspace,
+                                    size_t workspace_bytes, void* stream) {
+  GemmProblem g;
+  int rc = build_conv_problem(h_shape, x, w, d_bias_q, bias_frac_bits, relu, ADAPTION_MODE_REQUANT, y, d_stats,
+                              d_workspace, workspace_bytes, stream, g);
+  if (rc != ADAPTION_OK) return rc;
+  g.stochastic = StochasticParams{1, (uint32_t)seed, (uint32_t)(seed >> 32)};
+  return dispatch(g, algo);
+}
+
 size_t adaption_lp_conv_pool_workspace_bytes(const adaption_conv_shape* h_shape, adaption_qfmt fx, adaption_qfmt fw,
                                              adaption_qfmt fy, int64_t c_stride, int64_t y_c_stride, int32_t algo) {
   if (h_shape == nullptr) return 0;
@@ -351,6 +363,18 @@ int adaption_lp_ip_fwd(int64_t B, int64_t K, int64_t O, adaption_qtensor x, adap
   int rc = build_ip_problem(B, K, O, x, w, d_bias_q, bias_frac_bits, relu, mode, y, d_stats, d_workspace,
                             workspace_bytes, stream, g);
   if (rc != ADAPTION_OK) return rc;
+  return dispatch(g, algo);
+}
+
+int adaption_lp_ip_fwd_stochastic(int64_t B, int64_t K, int64_t O, adaption_qtensor x, adaption_qtensor w,
+                                  const int16_t* d_bias_q, int32_t bias_frac_bits, int32_t relu, int32_t algo,
+                                  adaption_qtensor y, uint64_t seed, adaption_stats* d_stats, void* d_workspace,
+                                  size_t workspace_bytes, void* stream) {
+  GemmProblem g;
+  int rc = build_ip_problem(B, K, O, x, w, d_bias_q, bias_frac_bits, relu, ADAPTION_MODE_REQUANT, y, d_stats,
+                            d_workspace, workspace_bytes, stream, g);
+  if (rc != ADAPTION_OK) return rc;
+  g.stochastic = StochasticParams{1, (uint32_t)seed, (uint32_t)(seed >> 32)};
   return dispatch(g, algo);
 }
 

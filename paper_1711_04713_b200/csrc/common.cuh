@@ -23,6 +23,46 @@ struct Counts {
   uint32_t zeros = 0, sat_pos = 0, sat_neg = 0;
 };
 
+// Seed of a layer whose rounding_scheme is stochastic (paper Sec. 2, Sec. 2.4); enabled = 0 means
+// deterministic rounding.
+struct StochasticParams {
+  int32_t enabled;
+  uint32_t key0, key1;
+};
+
+struct Philox4 {
+  uint32_t w[4];
+};
+
+// Philox4x32 with ten rounds, from its published definition: per round two 32x32 -> 64-bit
+// products with fixed multipliers, the high halves mixed with the other counter words and the
+// key, the key bumped by the Weyl constants between rounds.
+__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    if (r > 0) {
+      k0 += 0x9E3779B9u;
+      k1 += 0xBB67AE85u;
+    }
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+  }
+  Philox4 o;
+  o.w[0] = c0; o.w[1] = c1; o.w[2] = c2; o.w[3] = c3;
+  return o;
+}
+
+// The 32-bit draw of element `i` (row-major index over the real elements of a tensor): word i & 3 of
+// Philox4x32-10 with counter (i >> 2 as two 32-bit words, 0, 0) and the caller's seed as key.
+__device__ __forceinline__ uint32_t philox_draw(uint64_t i, uint32_t k0, uint32_t k1) {
+  const Philox4 b = philox4x32_10((uint32_t)(i >> 2), (uint32_t)(i >> 34), 0u, 0u, k0, k1);
+  const uint32_t w = (uint32_t)i & 3u;
+  return w == 0 ? b.w[0] : (w == 1 ? b.w[1] : (w == 2 ? b.w[2] : b.w[3]));
+}
+
 // v / 2^shift rounded half away from zero, saturated.  For shift > 0 and negative v the
 // identity -((-v + h) >> s) == (v + h - 1) >> s (h = 2^(s-1), arithmetic shift) is used.
 __device__ __forceinline__ int32_t requant_value(int64_t v, const RequantParams& rq, bool counted,
@@ -41,6 +81,28 @@ __device__ __forceinline__ int32_t requant_value(int64_t v, const RequantParams&
     const int64_t vc = v > lim ? lim : (v < -lim ? -lim : v);
     r = vc * ((int64_t)1 << (-rq.shift));
   }
+  if (r > (int64_t)rq.qmax) {
+    r = rq.qmax;
+    c.sat_pos += counted;
+  } else if (r < (int64_t)rq.qmin) {
+    r = rq.qmin;
+    c.sat_neg += counted;
+  }
+  c.zeros += (counted && r == 0);
+  return (int32_t)r;
+}
+
+// The same with stochastic rounding (Sec. 2.4) for shift > 0: v / 2^shift = q + rem / 2^shift with
+// q = floor(v / 2^shift); the result is q + 1 iff draw < T, T = rem * 2^(32 - shift), so that the
+// expectation is the unrounded value and rem = 0 never moves.  shift <= 32 (the formats allow at most 30).
+__device__ __forceinline__ int32_t requant_value_stochastic(int64_t v, const RequantParams& rq, uint32_t draw,
+                                                            bool counted, Counts& c) {
+  if (rq.shift <= 0) return requant_value(v, rq, counted, c);
+  if (rq.relu && v < 0) v = 0;
+  const int64_t q = v >> rq.shift;
+  const uint64_t rem = (uint64_t)(v - (q << rq.shift));
+  const uint32_t T = (uint32_t)(rem << (32 - rq.shift));
+  int64_t r = q + (draw < T ? 1 : 0);
   if (r > (int64_t)rq.qmax) {
     r = rq.qmax;
     c.sat_pos += counted;
@@ -145,6 +207,8 @@ struct GemmProblem {
   // Tensor-core path only: y receives max(row 2j, row 2j+1) of the layer's output as its row j (the
   // horizontal half of a 2x2 max-pool; y then has M / 2 rows).  Counters still refer to all M rows.
   bool pool_w = false;
+  // rounding_scheme STOCHASTIC for the requantization of this layer (REQUANT mode only)
+  StochasticParams stochastic{0, 0u, 0u};
 };
 
 int launch_direct(const GemmProblem& p);

@@ -18,6 +18,7 @@ struct DirectParams {
   const int16_t* bias; int32_t bias_shift;
   int8_t* y_hi; uint8_t* y_lo; int16_t* y_q16; int64_t y_stride;
   RequantParams rq;
+  StochasticParams st;
   int mode;
   adaption_stats* stats;
 };
@@ -73,7 +74,10 @@ __global__ void __launch_bounds__(256) direct_kernel(DirectParams p) {
       const int64_t a = acc < 0 ? -acc : acc;
       vmax = a > vmax ? a : vmax;
     } else {
-      const int32_t q = requant_value(acc, p.rq, real, c);
+      const int32_t q = (p.st.enabled && real)
+                            ? requant_value_stochastic(acc, p.rq, philox_draw((uint64_t)m * (uint64_t)p.N + (uint64_t)n,
+                                                                              p.st.key0, p.st.key1), real, c)
+                            : requant_value(acc, p.rq, real, c);
       store_q(p.rq.out_planes == 2 ? p.y_hi : nullptr, p.y_lo, p.y_q16,
               (size_t)m * (size_t)p.y_stride + (size_t)n, q);
     }
@@ -90,6 +94,7 @@ struct FinalizeParams {
   const int16_t* bias; int32_t bias_shift;
   uint32_t* y_hi; uint32_t* y_lo; uint2* y_q16; int64_t y_stride;
   RequantParams rq;
+  StochasticParams st;
   int mode;
   adaption_stats* stats;
 };
@@ -120,7 +125,10 @@ __global__ void __launch_bounds__(256) finalize_kernel(FinalizeParams p) {
         vmax = a > vmax ? a : vmax;
         q[u] = 0;
       } else {
-        q[u] = requant_value(v, p.rq, real, c);
+        q[u] = (p.st.enabled && real)
+                   ? requant_value_stochastic(v, p.rq, philox_draw((uint64_t)m * (uint64_t)p.N + (uint64_t)n,
+                                                                   p.st.key0, p.st.key1), real, c)
+                   : requant_value(v, p.rq, real, c);
       }
     }
     if (p.mode != ADAPTION_MODE_RANGE) {
@@ -166,6 +174,7 @@ int launch_direct(const GemmProblem& g) {
   p.w_lo = (const uint8_t*)g.w.lo; p.w_stride = g.w.c_stride;
   p.bias = g.bias; p.bias_shift = g.bias_shift;
   p.mode = g.mode; p.stats = g.stats;
+  p.st = g.stochastic;
   if (g.mode == ADAPTION_MODE_REQUANT) {
     p.rq = make_requant(g.acc_frac_bits, g.y.fmt, g.relu);
     p.y_hi = (int8_t*)g.y.hi; p.y_lo = (uint8_t*)g.y.lo; p.y_q16 = g.y.q16; p.y_stride = g.y.c_stride;
@@ -183,6 +192,7 @@ int launch_finalize(const int64_t* acc, int64_t ld, const GemmProblem& g) {
   p.acc = acc; p.ld = ld; p.M = g.M; p.N = g.N;
   p.bias = g.bias; p.bias_shift = g.bias_shift;
   p.mode = g.mode; p.stats = g.stats;
+  p.st = g.stochastic;
   if (g.mode == ADAPTION_MODE_REQUANT) {
     p.rq = make_requant(g.acc_frac_bits, g.y.fmt, g.relu);
     p.y_hi = (uint32_t*)g.y.hi; p.y_lo = (uint32_t*)g.y.lo; p.y_q16 = (uint2*)g.y.q16;

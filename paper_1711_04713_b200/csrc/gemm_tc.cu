@@ -47,6 +47,9 @@ constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
 // int32 accumulators: the shared middle accumulator takes two products of magnitude
 // <= 128*255 per k, so a reduction of up to 32768 stays below 2^31.
 constexpr int64_t kMaxKPerAccumulation = 32768;
+// epilogue variants (a template parameter of the kernel): generic 64-bit, the 32-bit fast path of
+// ReLU layers, generic with stochastic rounding
+constexpr int kEpiGeneric = 0, kEpiFast = 1, kEpiStochastic = 2;
 
 struct TcParams {
   int M, N;
@@ -71,6 +74,7 @@ struct TcParams {
   const int16_t* bias;
   int bias_shift;
   RequantParams rq;
+  StochasticParams st;         // stochastic rounding in the requantization (generic epilogue only)
   int mode;
   int8_t* y_hi;
   uint8_t* y_lo;
@@ -318,6 +322,30 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&lo)[8], int3
       : "r"(taddr)
       : "memory");
 }
+// thirty-two consecutive columns in one instruction (a TMEM load costs about the same latency
+// whatever its width, so the widest form that the register budget allows drains fastest)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void pin_after_wait32(int32_t (&r)[32]) {
+  asm volatile(""
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                 "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
+                 "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
+                 "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
 // Placed after tcgen05.wait::ld: ties the loaded registers to that point so that no use of them can
 // be scheduled before the wait (the load fills them asynchronously).
 __device__ __forceinline__ void pin_after_wait(int32_t (&r)[8]) {
@@ -495,20 +523,6 @@ __device__ __forceinline__ int32_t mad_lo(int32_t a, int32_t b, int32_t c) {
   asm("mad.lo.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
-template <int NACC, bool WIDE>
-__device__ __forceinline__ int32_t shifted32(int32_t x0, int32_t x1, int32_t x2, int2 c, int shift) {
-  // name the accumulators by weight: hh (2^16), mid (2^8), ll (1)
-  // a single accumulator (8-bit operands) is the whole sum: one 32-bit add, any shift >= 0
-  if (NACC == 1) return (x0 + mad_lo(c.y, 65536, c.x)) >> shift;
-  const int32_t hh = NACC == 3 ? x0 : 0;
-  const int32_t mid = NACC == 3 ? x1 : (NACC == 2 ? x0 : 0);
-  const int32_t ll = NACC == 3 ? x2 : (NACC == 2 ? x1 : x0);
-  const int32_t T = mid + ((ll + c.x) >> 8);
-  const int32_t H = hh + c.y;
-  if (WIDE) return (H + (T >> 8)) >> (shift - 16);
-  return mad_lo(H, 1 << (16 - shift), T >> (shift - 8));
-}
-
 // two 32-bit values -> two 16-bit values saturated to [-32768, 32767]; `lo` lands in the low half
 __device__ __forceinline__ uint32_t pack_sat_s16x2(int32_t hi, int32_t lo) {
   uint32_t d;
@@ -524,6 +538,51 @@ __device__ __forceinline__ uint32_t min_s16x2(uint32_t a, uint32_t b) {
   uint32_t d;
   asm("min.s16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
   return d;
+}
+
+// Fast path, accumulator by accumulator over thirty-two columns of one row.  With T and H as derived
+// above, `t` holds T (with a mixed 16 x 8-bit layer hh is absent and H = Ch) or, with 8-bit
+// operands on both sides, the single accumulator (the whole sum: one 32-bit add, any shift >= 0);
+// `h` holds hh.  Outputs are handled as pairs of 16-bit lanes (saturating pack, ReLU, upper bound,
+// zero count).  Saturation is only detected here (some lane reached the bound); the exact count of
+// that group of eight is then redone from the 32-bit results, which is rare.  Every group of eight
+// columns is either entirely real or entirely padding (N is a multiple of 8).
+template <int NACC, bool WIDE>
+__device__ __forceinline__ int32_t fast_result(int32_t t, int32_t h, int shift) {
+  if (NACC == 1) return t >> shift;
+  if (WIDE) return (h + (t >> 8)) >> (shift - 16);
+  return mad_lo(h, 1 << (16 - shift), t >> (shift - 8));
+}
+// sixteen of the thirty-two columns (`half` = 0 or 1) -> eight packed words; `t` and `h` hold T and H
+// (or, with a single accumulator, t holds the sum plus its constant)
+template <int NACC, bool WIDE>
+__device__ __forceinline__ void fast_outputs16(const int32_t (&t)[32], const int32_t (&h)[32], int half, int shift,
+                                               int32_t qmax, bool row_ok, int col, int N, Counts& cnt,
+                                               uint32_t (&w)[8]) {
+  const uint32_t qmax2 = (uint32_t)qmax * 0x00010001u;
+  const int32_t bound = qmax == 32767 ? 32767 : qmax + 1;      // a lane that reached this may have been clipped
+#pragma unroll
+  for (int g = 0; g < 2; ++g) {
+    const int base = 16 * half + 8 * g;
+    const bool counted = row_ok && col + base < N;
+    uint32_t top = 0, nonzero = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int k = base + 2 * j;
+      const int32_t r0 = fast_result<NACC, WIDE>(t[k], h[k], shift);
+      const int32_t r1 = fast_result<NACC, WIDE>(t[k + 1], h[k + 1], shift);
+      uint32_t v = max_s16x2(pack_sat_s16x2(r1, r0), 0u);
+      top = max_s16x2(top, v);
+      if (qmax != 32767) v = min_s16x2(v, qmax2);
+      nonzero += min_s16x2(v, 0x00010001u);
+      w[4 * g + j] = v;
+    }
+    if (counted) cnt.zeros += 8u - (nonzero & 0xffffu) - (nonzero >> 16);
+    if (counted && ((int32_t)(top & 0xffffu) >= bound || (int32_t)(top >> 16) >= bound)) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) cnt.sat_pos += (fast_result<NACC, WIDE>(t[base + j], h[base + j], shift) > qmax);
+    }
+  }
 }
 
 // One group of accumulators for eight consecutive columns of one row.
@@ -549,59 +608,37 @@ __device__ __forceinline__ long long acc_value(const Acc8<NACC>& x, int j) {
   return combine<NACC>(x.a[0][j], NACC >= 2 ? x.a[1][j] : 0, NACC == 3 ? x.a[2][j] : 0);
 }
 
-// Eight columns of one row on the fast path: outputs are handled as pairs of 16-bit lanes
-// (saturating pack, ReLU, upper bound, zero count).  Saturation is only detected here (some lane
-// reached the bound); the exact count is then redone from the accumulators, which is rare.
-// Returns the packed outputs w[j] = q[2j] | q[2j+1] << 16.  `counted`: real columns of a real row
-// (the others are padding and only stored).
-template <int NACC, bool WIDE>
-__device__ __forceinline__ void requant_relu_pairs_x8(const Acc8<NACC>& x, const int2* c2, int shift, int32_t qmax,
-                                                      bool counted, Counts& cnt, uint32_t* w) {
-  const uint32_t qmax2 = (uint32_t)qmax * 0x00010001u;
-  uint32_t top = 0, nonzero = 0;
+// Draws of the eight consecutive elements i0 .. i0 + 7 (two or three generator blocks).
+__device__ __forceinline__ void philox_draws8(uint64_t i0, uint32_t k0, uint32_t k1, uint32_t (&R)[8]) {
+  const uint64_t b0 = i0 >> 2;
+  const uint32_t off = (uint32_t)i0 & 3u;
+  const Philox4 a = philox4x32_10((uint32_t)b0, (uint32_t)(b0 >> 32), 0u, 0u, k0, k1);
+  const Philox4 b = philox4x32_10((uint32_t)(b0 + 1), (uint32_t)((b0 + 1) >> 32), 0u, 0u, k0, k1);
+  if (off == 0) {
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int32_t r0 = shifted32<NACC, WIDE>(x.a[0][2 * j], NACC >= 2 ? x.a[1][2 * j] : 0,
-                                             NACC == 3 ? x.a[2][2 * j] : 0, c2[2 * j], shift);
-    const int32_t r1 = shifted32<NACC, WIDE>(x.a[0][2 * j + 1], NACC >= 2 ? x.a[1][2 * j + 1] : 0,
-                                             NACC == 3 ? x.a[2][2 * j + 1] : 0, c2[2 * j + 1], shift);
-    uint32_t v = max_s16x2(pack_sat_s16x2(r1, r0), 0u);
-    top = max_s16x2(top, v);
-    if (qmax != 32767) v = min_s16x2(v, qmax2);
-    nonzero += min_s16x2(v, 0x00010001u);
-    w[j] = v;
+    for (int j = 0; j < 4; ++j) { R[j] = a.w[j]; R[4 + j] = b.w[j]; }
+    return;
   }
-  if (counted) cnt.zeros += 8u - (nonzero & 0xffffu) - (nonzero >> 16);
-  const int32_t bound = qmax == 32767 ? 32767 : qmax + 1;      // a lane that reached this may have been clipped
-  if (counted && ((int32_t)(top & 0xffffu) >= bound || (int32_t)(top >> 16) >= bound)) {
+  const Philox4 c = philox4x32_10((uint32_t)(b0 + 2), (uint32_t)((b0 + 2) >> 32), 0u, 0u, k0, k1);
+  const uint32_t w[12] = {a.w[0], a.w[1], a.w[2], a.w[3], b.w[0], b.w[1], b.w[2], b.w[3], c.w[0], c.w[1], c.w[2], c.w[3]};
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const long long c = (long long)c2[j].y * 65536ll + (long long)c2[j].x;
-      cnt.sat_pos += (((acc_value<NACC>(x, j) + c) >> shift) > (long long)qmax);
-    }
-  }
+  for (int j = 0; j < 8; ++j) R[j] = off == 1 ? w[j + 1] : (off == 2 ? w[j + 2] : w[j + 3]);
 }
 
-// Eight consecutive output columns of one row: recombine, add bias, requantize.  Returns the
-// outputs packed in pairs, w[j] = (q[2j] & 0xffff) | q[2j+1] << 16.
-// Fast path (kernels built with FAST): every group of eight columns is either entirely real or
-// entirely padding (N is a multiple of 8), `counted` says which.
-template <int NACC>
-__device__ __forceinline__ void requant8_fast(const Acc8<NACC>& x, const long long* c64, const TcParams& p,
-                                              bool counted, Counts& cnt, uint32_t* w) {
-  // per-column constants were staged as (C mod 2^16, C div 2^16) with the rounding half in C
-  const int2* c2 = reinterpret_cast<const int2*>(c64);
-  if (p.rq.shift >= 16)
-    requant_relu_pairs_x8<NACC, true>(x, c2, p.rq.shift, p.rq.qmax, counted, cnt, w);
-  else
-    requant_relu_pairs_x8<NACC, false>(x, c2, p.rq.shift, p.rq.qmax, counted, cnt, w);
-}
-template <int NACC, bool RELU>
+template <int NACC, bool RELU, bool STOCH>
 __device__ __forceinline__ void requant8(const Acc8<NACC>& x, const long long* c64, const TcParams& p, bool row_ok,
-                                         int col, Counts& cnt, uint32_t* w) {
+                                         int m, int col, Counts& cnt, uint32_t* w) {
   const int nvalid = row_ok ? min(max(p.N - col, 0), 8) : 0;
   int32_t q[8];
-  if (p.rq.shift > 0) {
+  if (STOCH && p.rq.shift > 0) {
+    // stochastic rounding: element index = row-major index over the real M x N outputs
+    uint32_t R[8];
+    if (nvalid > 0) philox_draws8((uint64_t)m * (uint64_t)p.N + (uint64_t)col, p.st.key0, p.st.key1, R);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      q[j] = j < nvalid ? requant_value_stochastic(acc_value<NACC>(x, j) + c64[j], p.rq, R[j], true, cnt)
+                        : requant_value(0, p.rq, false, cnt);
+  } else if (p.rq.shift > 0) {
     const long long half = 1ll << (p.rq.shift - 1);
 #pragma unroll
     for (int j = 0; j < 8; ++j)
@@ -639,17 +676,17 @@ __device__ __forceinline__ void partial_or_range8(const Acc8<NACC>& x, const lon
 }
 
 // byte planes of sixteen packed outputs: four low bytes / four high bytes per word
-__device__ __forceinline__ uint4 plane_lo(const uint32_t (&w)[8]) {
+__device__ __forceinline__ uint4 plane_lo(const uint32_t* w) {
   return make_uint4(__byte_perm(w[0], w[1], 0x6420), __byte_perm(w[2], w[3], 0x6420),
                     __byte_perm(w[4], w[5], 0x6420), __byte_perm(w[6], w[7], 0x6420));
 }
-__device__ __forceinline__ uint4 plane_hi(const uint32_t (&w)[8]) {
+__device__ __forceinline__ uint4 plane_hi(const uint32_t* w) {
   return make_uint4(__byte_perm(w[0], w[1], 0x7531), __byte_perm(w[2], w[3], 0x7531),
                     __byte_perm(w[4], w[5], 0x7531), __byte_perm(w[6], w[7], 0x7531));
 }
 
 // Direct stores of sixteen outputs of one row (16 bytes per plane; optional int16 copy).
-__device__ __forceinline__ void store16_global(const uint32_t (&w)[8], const TcParams& p, bool row_ok, int m,
+__device__ __forceinline__ void store16_global(const uint32_t* w, const TcParams& p, bool row_ok, int m,
                                                int col) {
   if (row_ok && col < p.y_stride) {
     const size_t off = (size_t)m * (size_t)p.y_stride + (size_t)col;
@@ -721,13 +758,15 @@ __device__ __forceinline__ bool epi_bar_all(int group, int threads, bool pred) {
 // on both sides), N a multiple of 8, no split-K,
 // magnitudes within the 32-bit bounds of the fast epilogue: it then contains only that path.
 // 20 warps: one block per SM, 96 registers per thread.
-template <int NAX, int NBW, bool PAIR, bool GROUPED, bool FAST>
+template <int NAX, int NBW, bool PAIR, bool GROUPED, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ CUtensorMap map_y_hi, const __grid_constant__ CUtensorMap map_y_lo,
                const TcParams p) {
   constexpr int NACC = NAX + NBW - 1;
+  constexpr bool FAST = EPI == kEpiFast;
+  constexpr bool STOCH = EPI == kEpiStochastic;
   extern __shared__ uint8_t smem_raw[];
   __shared__ Ctrl ctrl;
 
@@ -1056,8 +1095,12 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           long long b = 0;
           if (p.bias != nullptr && n < p.N && p.splits == 1) b = (long long)p.bias[n] * (1ll << p.bias_shift);
           if (FAST) {
+            // two arrays of BN 32-bit words: C mod 2^16 and C div 2^16 (a single accumulator takes all
+            // of C from the first), read four columns per load
             const long long C = b + (p.rq.shift > 0 ? 1ll << (p.rq.shift - 1) : 0ll);
-            reinterpret_cast<int2*>(colconst)[c] = make_int2((int)(C & 0xffff), (int)(C >> 16));
+            int* cw = reinterpret_cast<int*>(colconst);
+            cw[c] = NACC == 1 ? (int)C : (int)(C & 0xffff);
+            cw[p.BN + c] = (int)(C >> 16);
           } else {
             colconst[c] = b;
           }
@@ -1081,7 +1124,108 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       // the last step's values are in registers, before the arithmetic on them.
       const bool storing = FAST || (p.splits == 1 && p.mode == ADAPTION_MODE_REQUANT);
       bool released = false;
-      for (int c0 = col_begin; c0 < col_end || !released; c0 += 16) {
+      // Fast path with thirty-two columns per warp step: one TMEM load per accumulator, the low and
+      // middle accumulators first (they fold into T), the high one last; the accumulators go back
+      // to the issuing warp as soon as the last load has landed.
+      // (the host launches the FAST kernels only where every warp owns a multiple of 32 columns)
+      if (FAST) {
+        if (col_begin >= col_end) {          // a warp without columns only hands the accumulators back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
+            if (PAIR)
+              mbar_arrive_cluster(mapa_rank(bar, 0));
+            else
+              mbar_arrive(bar);
+          }
+          released = true;
+        }
+        for (int c0 = col_begin; c0 < col_end; c0 += 32) {
+          int32_t t[32], h[32];
+          const int4* cl4 = reinterpret_cast<const int4*>(reinterpret_cast<const int*>(colconst) + c0);
+          const int4* ch4 = reinterpret_cast<const int4*>(reinterpret_cast<const int*>(colconst) + p.BN + c0);
+          if (NACC == 3) {
+            tmem_ld32(taddr + (uint32_t)(c0 + 2 * p.BN), t);       // ll
+            tmem_ld32(taddr + (uint32_t)(c0 + p.BN), h);           // mid
+          } else if (NACC == 2) {
+            tmem_ld32(taddr + (uint32_t)(c0 + p.BN), t);           // weight 1
+            tmem_ld32(taddr + (uint32_t)c0, h);                    // weight 2^8
+          } else {
+            tmem_ld32(taddr + (uint32_t)c0, t);
+          }
+          tmem_ld_wait();
+          pin_after_wait32(t);
+          if (NACC >= 2) pin_after_wait32(h);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int4 c = cl4[j];
+            if (NACC >= 2) {                                       // T = mid + floor((ll + Cl) / 2^8)
+              t[4 * j + 0] = h[4 * j + 0] + ((t[4 * j + 0] + c.x) >> 8);
+              t[4 * j + 1] = h[4 * j + 1] + ((t[4 * j + 1] + c.y) >> 8);
+              t[4 * j + 2] = h[4 * j + 2] + ((t[4 * j + 2] + c.z) >> 8);
+              t[4 * j + 3] = h[4 * j + 3] + ((t[4 * j + 3] + c.w) >> 8);
+            } else {
+              t[4 * j + 0] += c.x; t[4 * j + 1] += c.y; t[4 * j + 2] += c.z; t[4 * j + 3] += c.w;
+            }
+          }
+          if (NACC == 3) {
+            tmem_ld32(taddr + (uint32_t)c0, h);                    // hh
+            tmem_ld_wait();
+            pin_after_wait32(h);
+          }
+          if (c0 + 32 >= col_end) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+              const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
+              if (PAIR)
+                mbar_arrive_cluster(mapa_rank(bar, 0));
+              else
+                mbar_arrive(bar);
+            }
+            released = true;
+          }
+          if (NACC >= 2) {                                         // H = hh + Ch
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int4 c = ch4[j];
+              if (NACC == 3) {
+                h[4 * j + 0] += c.x; h[4 * j + 1] += c.y; h[4 * j + 2] += c.z; h[4 * j + 3] += c.w;
+              } else {
+                h[4 * j + 0] = c.x; h[4 * j + 1] = c.y; h[4 * j + 2] = c.z; h[4 * j + 3] = c.w;
+              }
+            }
+          }
+          const int col = tc.n0 + c0;
+          const bool wide = NACC == 1 || p.rq.shift >= 16;
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t wq[8];
+            if (wide)
+              fast_outputs16<NACC, true>(t, h, half, p.rq.shift, p.rq.qmax, row_ok, col, p.N, cnt, wq);
+            else
+              fast_outputs16<NACC, false>(t, h, half, p.rq.shift, p.rq.qmax, row_ok, col, p.N, cnt, wq);
+            const int chunk = (c0 >> 4) + half;
+            if (p.staged && p.pool_w) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) wq[j] = max_s16x2(wq[j], __shfl_xor_sync(0xffffffffu, wq[j], 1));
+              if ((lane & 1) == 0) {
+                const uint32_t off = staged_offset(row >> 1, chunk, p.BN);
+                st_shared_v4(stage_lo + off, plane_lo(wq));
+                if (p.rq.out_planes == 2) st_shared_v4(stage_hi + off, plane_hi(wq));
+              }
+            } else if (p.staged) {
+              const uint32_t off = staged_offset(row, chunk, p.BN);
+              st_shared_v4(stage_lo + off, plane_lo(wq));
+              if (p.rq.out_planes == 2) st_shared_v4(stage_hi + off, plane_hi(wq));
+            } else {
+              store16_global(wq, p, row_ok, m, col + 16 * half);
+            }
+          }
+        }
+      }
+      for (int c0 = col_begin; !FAST && (c0 < col_end || !released); c0 += 16) {
         const bool have = c0 < col_end;
         Acc8<NACC> xa, xb;
         if (have) {
@@ -1105,20 +1249,17 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         if (!have) break;
         const int col = tc.n0 + c0;
         const long long* bcol = colconst + c0;
-        if (!FAST && !storing) {
+        if (!storing) {
           partial_or_range8<NACC>(xa, bcol, p, row_ok, m, col, vmax);
           partial_or_range8<NACC>(xb, bcol + 8, p, row_ok, m, col + 8, vmax);
         } else {
           uint32_t wq[8];
-          if (FAST) {
-            requant8_fast<NACC>(xa, bcol, p, row_ok && col < p.N, cnt, wq);
-            requant8_fast<NACC>(xb, bcol + 8, p, row_ok && col + 8 < p.N, cnt, wq + 4);
-          } else if (p.rq.relu) {
-            requant8<NACC, true>(xa, bcol, p, row_ok, col, cnt, wq);
-            requant8<NACC, true>(xb, bcol + 8, p, row_ok, col + 8, cnt, wq + 4);
+          if (p.rq.relu) {
+            requant8<NACC, true, STOCH>(xa, bcol, p, row_ok, m, col, cnt, wq);
+            requant8<NACC, true, STOCH>(xb, bcol + 8, p, row_ok, m, col + 8, cnt, wq + 4);
           } else {
-            requant8<NACC, false>(xa, bcol, p, row_ok, col, cnt, wq);
-            requant8<NACC, false>(xb, bcol + 8, p, row_ok, col + 8, cnt, wq + 4);
+            requant8<NACC, false, STOCH>(xa, bcol, p, row_ok, m, col, cnt, wq);
+            requant8<NACC, false, STOCH>(xb, bcol + 8, p, row_ok, m, col + 8, cnt, wq + 4);
           }
           if (p.staged && p.pool_w) {
             // Horizontal half of a 2x2 max-pool: rows 2j and 2j+1 of the tile are neighbouring
@@ -1433,7 +1574,7 @@ bool encode_im2col_nhwc(CUtensorMap* map, const void* base, const adaption_conv_
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NAX, int NBW, bool PAIR, bool GROUPED, bool FAST>
+template <int NAX, int NBW, bool PAIR, bool GROUPED, int EPI>
 int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem, cudaStream_t stream) {
   // The dynamic shared-memory limit is a per-device attribute of the kernel: remember, per device
   // ordinal, the largest size it has been raised to (a racing thread at worst sets it once more).
@@ -1443,7 +1584,7 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
   if (cudaGetDevice(&dev) != cudaSuccess) return ADAPTION_ERR_CUDA;
   const bool cached = dev >= 0 && dev < kMaxDevices;
   if (!cached || smem > attr_size[dev].load(std::memory_order_acquire)) {
-    const cudaError_t ae = cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, FAST>,
+    const cudaError_t ae = cudaFuncSetAttribute(lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, EPI>,
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (ae != cudaSuccess) return cuda_failure(ae, "lp_gemm_kernel shared-memory attribute");
     if (cached) {
@@ -1468,7 +1609,7 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
     cfg.numAttrs = 1;
   }
   const cudaError_t le =
-      cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, FAST>, maps[0], maps[1], maps[2], maps[3], maps[4],
+      cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, EPI>, maps[0], maps[1], maps[2], maps[3], maps[4],
                          maps[5], p);
   if (le != cudaSuccess) {
     (void)cudaGetLastError();
@@ -1477,23 +1618,22 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
   return cuda_status(cudaGetLastError(), "after lp_gemm_kernel launch");
 }
 
+template <int NAX, int NBW, bool PAIR, bool GROUPED>
+int launch_epi(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem, cudaStream_t stream) {
+  if (p.fast_relu != 0) return launch_kernel<NAX, NBW, PAIR, GROUPED, kEpiFast>(maps, p, grid, smem, stream);
+  if (p.st.enabled != 0) return launch_kernel<NAX, NBW, PAIR, GROUPED, kEpiStochastic>(maps, p, grid, smem, stream);
+  return launch_kernel<NAX, NBW, PAIR, GROUPED, kEpiGeneric>(maps, p, grid, smem, stream);
+}
+
 template <int NAX, int NBW>
 int launch_either(bool pair, const CUtensorMap* maps, const TcParams& p, int grid, size_t smem,
                   cudaStream_t stream) {
   const bool grouped = p.kps > 1 || p.b_resident != 0;
-  const bool fast = p.fast_relu != 0;
-  if (pair) {
-    if (grouped)
-      return fast ? launch_kernel<NAX, NBW, true, true, true>(maps, p, grid, smem, stream)
-                  : launch_kernel<NAX, NBW, true, true, false>(maps, p, grid, smem, stream);
-    return fast ? launch_kernel<NAX, NBW, true, false, true>(maps, p, grid, smem, stream)
-                : launch_kernel<NAX, NBW, true, false, false>(maps, p, grid, smem, stream);
-  }
-  if (grouped)
-    return fast ? launch_kernel<NAX, NBW, false, true, true>(maps, p, grid, smem, stream)
-                : launch_kernel<NAX, NBW, false, true, false>(maps, p, grid, smem, stream);
-  return fast ? launch_kernel<NAX, NBW, false, false, true>(maps, p, grid, smem, stream)
-              : launch_kernel<NAX, NBW, false, false, false>(maps, p, grid, smem, stream);
+  if (pair)
+    return grouped ? launch_epi<NAX, NBW, true, true>(maps, p, grid, smem, stream)
+                   : launch_epi<NAX, NBW, true, false>(maps, p, grid, smem, stream);
+  return grouped ? launch_epi<NAX, NBW, false, true>(maps, p, grid, smem, stream)
+                 : launch_epi<NAX, NBW, false, false>(maps, p, grid, smem, stream);
 }
 
 
@@ -1707,9 +1847,18 @@ int launch_tensor(const GemmProblem& g) {
   p.stage_off = c.stage_off;
   p.const_off = c.stage_off + c.stage_out_bytes;
   const bool single = c.nacc == 1;
-  if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && p.rq.shift >= (single ? 0 : 9) &&
-      p.rq.shift <= 31 && g.N % 8 == 0 && knob(kFast) != 0) {
-    // 32-bit bounds of the fast epilogue (see shifted32): with a reduction of kred bytes per plane row
+  // (its epilogue takes 32 columns per warp step: tiles of 64 columns need the two warp groups,
+  // tiles of 32 columns take the generic epilogue)
+  const int cols_per_epi_warp = c.BN / (kEpiWarps / c.epi_groups / 4);
+  // stochastic rounding happens where the value is requantized: in this kernel's epilogue, or in the
+  // finalize kernel when the reduction is split
+  p.st = g.stochastic;
+  if (g.mode != ADAPTION_MODE_REQUANT || c.splits > 1) p.st.enabled = 0;
+  if (g.mode == ADAPTION_MODE_REQUANT && c.splits == 1 && g.relu && !g.stochastic.enabled &&
+      p.rq.shift >= (single ? 0 : 9) &&
+      p.rq.shift <= 31 && g.N % 8 == 0 && cols_per_epi_warp >= 32 && cols_per_epi_warp % 32 == 0 &&
+      knob(kFast) != 0) {
+    // 32-bit bounds of the fast epilogue (see fast_result): with a reduction of kred bytes per plane row
     // |hh| <= kred 2^14, |mid| <= kred 65280, |ll| <= kred 65025, and |C| < 2^(15 + bias_shift) + 2^(shift-1)
     const long long kred = (long long)c.num_kb * c.BK;
     const long long cmax = (g.bias != nullptr ? (1ll << (15 + g.bias_shift)) : 0ll) +

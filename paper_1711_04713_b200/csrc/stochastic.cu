@@ -17,31 +17,6 @@ int num_sms();
 
 namespace {
 
-struct Philox4 {
-  uint32_t w[4];
-};
-
-// Philox4x32 with ten rounds, from its published definition: per round two 32x32 -> 64-bit
-// products with fixed multipliers, the high halves mixed with the other counter words and the
-// key, the key bumped by the Weyl constants between rounds.
-__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                                 uint32_t k0, uint32_t k1) {
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    if (r > 0) {
-      k0 += 0x9E3779B9u;
-      k1 += 0xBB67AE85u;
-    }
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
-    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-  }
-  Philox4 o;
-  o.w[0] = c0; o.w[1] = c1; o.w[2] = c2; o.w[3] = c3;
-  return o;
-}
-
 // floor(y) plus one where the draw falls below T = floor(frac(y) 2^32), y = x 2^f, from
 // single-precision and 32-bit integer steps only; every step is exact:
 //   y = x * 2^f never rounds (f >= 0; an overflow gives +-Inf, which the clamp to a little outside

@@ -52,6 +52,16 @@ def calibration_loop(be, kinds: list[str], threshold: float = 0.0, group=None, d
     return rec
 
 
+def rounding_seeds(rounding_seed: int, layer_index: int | None):
+    """Seeds of the stochastic-rounding draws of one pass: input = base; layer li (conv / inner-product
+    layers counted from 0): weights base + 16 li + 1, biases + 2, output + 3; base = rounding_seed *
+    1000003; all modulo 2^64."""
+    base = (int(rounding_seed) * 1000003) & 0xFFFFFFFFFFFFFFFF
+    if layer_index is None:
+        return base
+    return tuple((base + 16 * layer_index + k) & 0xFFFFFFFFFFFFFFFF for k in (1, 2, 3))
+
+
 def act_c_stride(c: int) -> int:
     """Channel pitch of activation / weight planes: a multiple of 32 so that every layer can take
     the tensor-core path."""
@@ -92,7 +102,12 @@ class _Layer:
 
 class LPNetwork:
     def __init__(self, params: list[dict], batch: int, in_hw: tuple[int, int], in_c: int, n_bits: int,
-                 algo: int = B.ALGO_AUTO, keep_q16: bool = False, device="cuda", fuse_pool: bool = True):
+                 algo: int = B.ALGO_AUTO, keep_q16: bool = False, device="cuda", fuse_pool: bool = True,
+                 rounding_seed: int | None = None):
+        """``rounding_seed`` not None: rounding_scheme STOCHASTIC for every layer (paper Sec. 2, 2.4): the
+        input, weights, biases and layer outputs are rounded stochastically, each tensor with its own
+        seed (see ``rounding_seeds``); decimal points still come from the measured ranges."""
+        self.rounding_seed = rounding_seed
         self.n_bits = n_bits
         self.fuse_pool = fuse_pool
         self.algo = algo
@@ -182,6 +197,8 @@ class LPNetwork:
         """Weights and biases -> fixed point (paper Sec. 2.1: quantized in the forward pass).  With
         ``measure`` the decimal point of each layer's weights is taken from max|w| on the device, or,
         with ``threshold`` > 0, from the thresholded allocation of Sec. 2.3."""
+        if self.rounding_seed is not None:
+            return self._quantize_params_stochastic(measure, threshold)
         if not measure:
             # fixed formats: every weight and bias tensor of the network in one library call
             entries = []
@@ -209,6 +226,25 @@ class LPNetwork:
                 f = int(L.w_fmt_dev.cpu()[1])
                 L.w.frac_bits = f
                 L.b.frac_bits = f
+
+    def _quantize_params_stochastic(self, measure: bool, threshold: float):
+        """Weights and biases with rounding_scheme STOCHASTIC: formats as in the deterministic case
+        (from max|w| or the thresholded allocation), values by the stochastic quantizer."""
+        li = 0
+        for L in self.layers:
+            if L.type not in ("conv", "ip"):
+                continue
+            if measure and threshold > 0:
+                L.w.frac_bits = L.b.frac_bits = self._fp32_fmt_by_threshold(L.w_f32, threshold)
+            elif measure:
+                L.w_max_dev.zero_()
+                B.adaption_measure_range(L.w_f32, self.n_bits, L.w_max_dev, L.w_fmt_dev)
+                L.w.frac_bits = L.b.frac_bits = int(L.w_fmt_dev.cpu()[1])
+            sw, sb, _ = rounding_seeds(self.rounding_seed, li)
+            B.adaption_quantize_stochastic(L.w_f32, L.w.outer, L.w.inner, L.w, sw)
+            B.adaption_quantize_stochastic(L.b_f32, 1, L.K, L.b, sb)
+            L.extra["li"] = li
+            li += 1
 
     @staticmethod
     def helper_launches(L: _Layer) -> int:
@@ -247,7 +283,7 @@ class LPNetwork:
         """True where layer i is a convolution whose output only feeds the 2x2 max-pool after it, so
         that inference may run the pair as one library call (the convolution's own output is then not
         materialised in ``layers[i].y``)."""
-        if not self.fuse_pool or self.keep_q16 or i + 1 >= len(self.layers):
+        if not self.fuse_pool or self.keep_q16 or i + 1 >= len(self.layers) or self.rounding_seed is not None:
             return False
         L, P = self.layers[i], self.layers[i + 1]
         return L.type == "conv" and P.type == "pool" and L.OH % 2 == 0 and L.OW % 2 == 0
@@ -269,15 +305,25 @@ class LPNetwork:
             return L.y
         ws = self._workspace(L, x)
         y = L.y if mode == B.MODE_REQUANT else None
+        stochastic = self.rounding_seed is not None and mode == B.MODE_REQUANT
+        seed_y = rounding_seeds(self.rounding_seed, L.extra["li"])[2] if stochastic else 0
         if L.type == "conv":
-            B.adaption_lp_conv_fwd(L.shape, x, L.w, L.b.q16, L.b.frac_bits, L.relu, mode, self.algo, y,
-                                   L.stats, ws)
+            if stochastic:
+                B.adaption_lp_conv_fwd_stochastic(L.shape, x, L.w, L.b.q16, L.b.frac_bits, L.relu, self.algo, y,
+                                                  seed_y, L.stats, ws)
+            else:
+                B.adaption_lp_conv_fwd(L.shape, x, L.w, L.b.q16, L.b.frac_bits, L.relu, mode, self.algo, y,
+                                       L.stats, ws)
         else:
             xin = x.reshaped(L.N, L.ip_k, L.ip_k)
             O, kp = L.extra["w_view"]
             win = L.w.reshaped(O, kp, kp)
-            B.adaption_lp_ip_fwd(L.N, L.ip_k, L.K, xin, win, L.b.q16, L.b.frac_bits, L.relu, mode,
-                                 self.algo, y, L.stats, ws)
+            if stochastic:
+                B.adaption_lp_ip_fwd_stochastic(L.N, L.ip_k, L.K, xin, win, L.b.q16, L.b.frac_bits, L.relu,
+                                                self.algo, y, seed_y, L.stats, ws)
+            else:
+                B.adaption_lp_ip_fwd(L.N, L.ip_k, L.K, xin, win, L.b.q16, L.b.frac_bits, L.relu, mode,
+                                     self.algo, y, L.stats, ws)
         return L.y
 
     # ------------------------------------------------------------------ calibration
@@ -323,8 +369,7 @@ class LPNetwork:
     def quantize_input(self, frac_bits: int):
         self.x_stats.zero_()
         self.xq.frac_bits = frac_bits
-        B.adaption_quantize(self._cal_x, self.xq.outer, self.xq.inner, self.xq, None, B.ROUND_DETERMINISTIC,
-                            self.x_stats)
+        self._quantize_input(self._cal_x)
         self._cal_act = self.xq
         return B.read_stats(self.x_stats)
 
@@ -384,6 +429,14 @@ class LPNetwork:
                 L.y.frac_bits = int(next(it))
         self.calibrated = True
 
+    def _quantize_input(self, x_f32: torch.Tensor):
+        if self.rounding_seed is not None:
+            B.adaption_quantize_stochastic(x_f32, self.xq.outer, self.xq.inner, self.xq,
+                                           rounding_seeds(self.rounding_seed, None), False, None, self.x_stats)
+        else:
+            B.adaption_quantize(x_f32, self.xq.outer, self.xq.inner, self.xq, None, B.ROUND_DETERMINISTIC,
+                                self.x_stats)
+
     # ------------------------------------------------------------------ inference
     def forward(self, x_f32: torch.Tensor, requantize_params: bool = True, measure_input: bool = True):
         """One forward pass with the calibrated formats; enqueues work only (no host sync).
@@ -394,8 +447,7 @@ class LPNetwork:
             # range of the incoming batch (monitoring; the calibrated input format stays in force)
             B.adaption_measure_range(x_f32, self.n_bits, self.x_max_dev, self.x_fmt_dev)
             launches += 2
-        B.adaption_quantize(x_f32, self.xq.outer, self.xq.inner, self.xq, None, B.ROUND_DETERMINISTIC,
-                            self.x_stats)
+        self._quantize_input(x_f32)
         launches += 1
         if requantize_params:
             self.quantize_params(measure=False)

@@ -8,6 +8,7 @@ import pytest
 import torch
 
 from oracle import reference as orc
+from oracle import stochastic as orc_st
 from paper_1711_04713_b200 import binding as B
 from tests.util import Guards, dev, from_qtensor, q16_of, stats_tuple, to_qtensor
 
@@ -35,7 +36,8 @@ def _pick_f_out(acc, bq, fb, F, relu, n_out):
 
 
 def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, algo, with_bias=True,
-                  extreme=False, f_out=None, with_q16=True, mag_bits=None, fmts=None, cs=None, ws_offset=0):
+                  extreme=False, f_out=None, with_q16=True, mag_bits=None, fmts=None, cs=None, ws_offset=0,
+                  stochastic_seed=None):
     """`with_q16=False` leaves out the optional int16 copy of the output, which lets the tensor-core
     kernel stage its byte planes in shared memory and write them with bulk-tensor stores.
     `mag_bits` limits operand magnitudes (small accumulators -> short requantization shifts)."""
@@ -52,6 +54,9 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
     A, f_auto = _pick_f_out(acc, bq, fw, F, relu, n_out)
     f_out = f_auto if f_out is None else f_out
     want, cnt = orc.epilogue(acc, bq, fw, F, relu, n_out, f_out)
+    if stochastic_seed is not None:
+        want, c3 = orc_st.epilogue_stochastic(acc, bq, fw, F, relu, n_out, f_out, stochastic_seed)
+        cnt = orc.Counters(*c3)
     OH, OW = acc.shape[1], acc.shape[2]
 
     x = to_qtensor(xq.reshape(-1, Cin), nx, fx, cs)
@@ -70,7 +75,10 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
     assert int(s.max_abs_acc) == A
     assert B.adaption_choose_frac_bits_from_acc(A, F, n_out) == f_auto
     st = B.new_stats()
-    B.adaption_lp_conv_fwd(shp, x, w, bias_dev, fw, relu, B.MODE_REQUANT, algo, y, st, ws)
+    if stochastic_seed is not None:
+        B.adaption_lp_conv_fwd_stochastic(shp, x, w, bias_dev, fw, relu, algo, y, stochastic_seed, st, ws)
+    else:
+        B.adaption_lp_conv_fwd(shp, x, w, bias_dev, fw, relu, B.MODE_REQUANT, algo, y, st, ws)
     s = B.read_stats(st)
     assert s.status == 0
     got = from_qtensor(y).reshape(want.shape)
@@ -84,7 +92,8 @@ def run_conv_case(rng, N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu, alg
     return cnt
 
 
-def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out=None, with_q16=True):
+def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out=None, with_q16=True,
+                stochastic_seed=None):
     xq = _rand_q(rng, (Bsz, K), nx, 0.4)
     wq = _rand_q(rng, (O, K), nw)
     fx, fw = nx - 2, nw - 1
@@ -94,6 +103,9 @@ def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out
     A, f_auto = _pick_f_out(acc, bq, fw, F, relu, n_out)
     f_out = f_auto if f_out is None else f_out
     want, cnt = orc.epilogue(acc, bq, fw, F, relu, n_out, f_out)
+    if stochastic_seed is not None:
+        want, c3 = orc_st.epilogue_stochastic(acc, bq, fw, F, relu, n_out, f_out, stochastic_seed)
+        cnt = orc.Counters(*c3)
     x = to_qtensor(xq, nx, fx)
     w = to_qtensor(wq, nw, fw)
     guards = Guards()
@@ -106,7 +118,10 @@ def run_ip_case(rng, Bsz, K, O, nx, nw, n_out, relu, algo, with_bias=True, f_out
     s = B.read_stats(st)
     assert s.status == 0 and int(s.max_abs_acc) == A
     st = B.new_stats()
-    B.adaption_lp_ip_fwd(Bsz, K, O, x, w, bias_dev, fw, relu, B.MODE_REQUANT, algo, y, st, ws)
+    if stochastic_seed is not None:
+        B.adaption_lp_ip_fwd_stochastic(Bsz, K, O, x, w, bias_dev, fw, relu, algo, y, stochastic_seed, st, ws)
+    else:
+        B.adaption_lp_ip_fwd(Bsz, K, O, x, w, bias_dev, fw, relu, B.MODE_REQUANT, algo, y, st, ws)
     s = B.read_stats(st)
     assert s.status == 0
     got = from_qtensor(y)
@@ -473,6 +488,71 @@ def test_conv_with_fused_pool(case, with_q16):
         with pytest.raises(B.AdaptionError):
             B.adaption_lp_conv_pool_fwd(shp, x, w, dev(bq), fw, relu, B.ALGO_AUTO, y, st2, ws, bad_phases)
     guards.check()
+
+
+# ------------------------------------------------------------------ stochastic rounding in the layer epilogue
+STOCHASTIC_CONV = [
+    # N, H, W, Cin, K, R, pad, stride, nx, nw, n_out, relu
+    (2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True),     # 128-column tiles (pair or single)
+    (6, 20, 20, 64, 96, 3, 1, 1, 16, 16, 16, False),      # signed outputs, ragged N tile, M tail
+    (4, 33, 31, 64, 130, 3, 1, 2, 16, 16, 12, True),      # N = 130: element indices misaligned to the generator's blocks
+    (2, 30, 30, 256, 61, 3, 1, 1, 16, 16, 16, True),      # odd N: every row starts at another word of a block
+    (2, 24, 24, 128, 128, 3, 1, 1, 8, 8, 8, True),        # single int8 pass
+    (2, 24, 24, 128, 256, 3, 1, 1, 8, 8, 8, True),        # 256-column tiles
+    (8, 32, 32, 3, 64, 3, 1, 1, 16, 16, 16, True),        # packed first-layer taps
+    (2, 12, 12, 20, 50, 5, 2, 1, 16, 16, 16, True),       # plain integer kernel (odd pitch)
+]
+
+
+@pytest.mark.parametrize("case", STOCHASTIC_CONV)
+@pytest.mark.parametrize("with_q16", [False, True])
+def test_conv_stochastic_rounding(case, with_q16, cta_mode):
+    """rounding_scheme STOCHASTIC in the fused requantization: every kernel and tile shape gives the
+    oracle's bits for the same seed (the draw depends on the output's index only)."""
+    seed = 0xC0FFEE123456789 + sum(case)
+    cs = 48 if case[3] == 20 else None
+    cnt = run_conv_case(np.random.default_rng(sum(case) + 3), *case, B.ALGO_AUTO, with_q16=with_q16, cs=cs,
+                        stochastic_seed=seed)
+    assert cnt.zeros > 0
+
+
+@pytest.mark.parametrize("shift_case", [(13, 15, 12), (4, 8, 12), (2, 3, 9), (0, 0, 0)])
+def test_conv_stochastic_rounding_across_shifts(shift_case):
+    """Long and short right shifts, an exact left shift (more fractional bits out than in) and shift 0."""
+    fx, fw, f_out = shift_case
+    run_conv_case(np.random.default_rng(sum(shift_case)), 2, 24, 24, 128, 128, 3, 1, 1, 16, 16, 16, True,
+                  B.ALGO_TENSOR, f_out=f_out, with_q16=False, mag_bits=(6, 6), fmts=(fx, fw), stochastic_seed=99)
+
+
+@pytest.mark.parametrize("case", [(70, 1000, 260, 16, 16, 16, False), (64, 25088, 250, 16, 16, 16, True),
+                                  (130, 256, 128, 8, 8, 8, True), (5, 64, 33, 16, 8, 16, False)])
+@pytest.mark.parametrize("algo", [B.ALGO_AUTO, B.ALGO_DIRECT])
+def test_ip_stochastic_rounding(case, algo):
+    """Inner products, including a split reduction (the finalize kernel rounds) and the plain kernel."""
+    if algo == B.ALGO_DIRECT and case[1] > 2000:
+        pytest.skip("the plain kernel takes too long on the long reduction")
+    run_ip_case(np.random.default_rng(sum(case) + 9), *case, algo, stochastic_seed=0xFEEDFACE + case[0])
+
+
+def test_stochastic_layer_statistics():
+    """Sec. 2.4 at the level of a layer: another seed gives other bits, the same seed the same; every
+    output is one of the two neighbours of the unrounded value; the mean error over a large layer
+    vanishes where the deterministic tie rule does not matter."""
+    rng = np.random.default_rng(4)
+    N, H, W, Cin, K = 2, 24, 24, 128, 128
+    xq, wq = _rand_q(rng, (N, H, W, Cin), 12, 0.4), _rand_q(rng, (K, 3, 3, Cin), 12)
+    x, w = to_qtensor(xq.reshape(-1, Cin), 16, 9, Cin), to_qtensor(wq.reshape(-1, Cin), 16, 11, Cin)
+    shp = B.conv_shape(N, H, W, Cin, K, 3, 3, 1, 1)
+    acc = orc.conv_acc(xq, wq, (1, 1))
+    outs = []
+    for seed in (1, 1, 2):
+        y = B.QTensor.empty(N * H * W, K, 16, 2, K)
+        B.adaption_lp_conv_fwd_stochastic(shp, x, w, None, 0, False, B.ALGO_TENSOR, y, seed, B.new_stats(), None)
+        outs.append(from_qtensor(y).reshape(acc.shape).astype(np.float64))
+    assert np.array_equal(outs[0], outs[1]) and not np.array_equal(outs[0], outs[2])
+    exact = acc.astype(np.float64) / 2.0 ** 18
+    assert np.all((outs[0] == np.floor(exact)) | (outs[0] == np.floor(exact) + 1))
+    assert abs(float((outs[0] - exact).mean())) < 5 * 0.5 / np.sqrt(exact.size)
 
 
 # ------------------------------------------------------------------ robustness of the boundary

@@ -15,9 +15,9 @@ from tests.util import dev, from_qtensor
 pytestmark = pytest.mark.gpu
 
 
-def _compare_stack(params, x, x_fmt, n_bits, in_hw, in_c, algo, threshold=0.0):
-    rec = orc.run_network(params, x, x_fmt, n_bits, threshold=threshold)
-    net = LPNetwork(params, x.shape[0], in_hw, in_c, n_bits, algo=algo)
+def _compare_stack(params, x, x_fmt, n_bits, in_hw, in_c, algo, threshold=0.0, rounding_seed=None):
+    rec = orc.run_network(params, x, x_fmt, n_bits, threshold=threshold, rounding_seed=rounding_seed)
+    net = LPNetwork(params, x.shape[0], in_hw, in_c, n_bits, algo=algo, rounding_seed=rounding_seed)
     xd = dev(x.reshape(-1, in_c))
     grec = net.calibrate(xd, x_fmt, threshold=threshold)
     assert len(grec) == len(rec)
@@ -53,6 +53,8 @@ def _compare_stack(params, x, x_fmt, n_bits, in_hw, in_c, algo, threshold=0.0):
            (last["wq"].astype(np.float64) * 2.0 ** -last["w_frac_bits"]).T + \
            last["bq"].astype(np.float64) * 2.0 ** -last["w_frac_bits"]
     deq = from_qtensor(out).astype(np.float64) * 2.0 ** -last["frac_bits"]
+    # (stochastic rounding may land on either neighbour: up to one LSB; deterministic: half an LSB plus
+    # the one-LSB saturation edge)
     assert np.all(np.abs(deq - real) <= 2.0 ** -last["frac_bits"])
     return rec
 
@@ -97,6 +99,26 @@ def test_stacks_with_thresholded_bit_allocation(threshold):
              wl.LayerSpec("ip", "f2", 256, 10, relu=False)]
     _compare_stack(wl.make_params(specs, seed=4), wl.vgg16_input(8, seed=4, hw=32), None, 8, (32, 32), 3,
                    B.ALGO_AUTO, threshold=threshold)
+
+
+@pytest.mark.parametrize("algo", [B.ALGO_AUTO, B.ALGO_DIRECT])
+def test_stacks_with_stochastic_rounding(algo):
+    """rounding_scheme STOCHASTIC for every layer (paper Sec. 2, 2.4): input, weights, biases and layer
+    outputs rounded stochastically with per-tensor seeds; every tensor, decimal point and counter equals
+    the oracle's, in calibration and in inference, on the tensor-core path and on the plain kernels;
+    also together with the thresholded allocation."""
+    params = wl.make_params(wl.lenet_specs(), seed=0)
+    x = wl.lenet_input(8, seed=0)
+    rec = _compare_stack(params, x, None, 16, (28, 28), 1, algo, rounding_seed=11)
+    base = orc.run_network(params, x, None, 16)
+    assert any(not np.array_equal(r["y"], b["y"]) for r, b in zip(rec, base))      # it is another rounding
+    specs = [wl.LayerSpec("conv", "c1", 3, 64, 3, 1, 1, True), wl.LayerSpec("conv", "c2", 64, 64, 3, 1, 1, True),
+             wl.LayerSpec("pool", "p1"), wl.LayerSpec("conv", "c3", 64, 128, 3, 1, 1, True),
+             wl.LayerSpec("pool", "p2"), wl.LayerSpec("ip", "f1", 8 * 8 * 128, 256, relu=True),
+             wl.LayerSpec("ip", "f2", 256, 10, relu=False)]
+    for n_bits, thr in ((16, 0.0), (8, 0.0), (16, 0.01)):
+        _compare_stack(wl.make_params(specs, seed=6), wl.vgg16_input(8, seed=6, hw=32), None, n_bits, (32, 32), 3,
+                       algo, threshold=thr, rounding_seed=12)
 
 
 def test_giga1net_stack():
