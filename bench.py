@@ -353,6 +353,7 @@ def run_gpu(args):
     if dist is not None:
         dist.barrier()
     B.load()
+    apply_overrides(B, args)
     peaks = read_peaks()
 
     # ---- workload: each rank owns its own batch of images (weak scaling, no data-path collective)
@@ -672,6 +673,7 @@ def run_kernel(args):
         raise RuntimeError("bench.py --kernel needs a CUDA device")
     bld.build_library()
     B.load()
+    apply_overrides(B, args)
     a = args
     peaks = read_peaks()
     g = torch.Generator(device="cuda").manual_seed(a.seed)
@@ -801,6 +803,12 @@ def run_kernel(args):
     print(json.dumps(out), flush=True)
 
 
+def apply_overrides(B, args):
+    for kv in args.set:
+        name, _, value = kv.partition("=")
+        B.adaption_debug_set(name, int(value))
+
+
 def respawn_ranks(args) -> int:
     """`python bench.py --gpus N` without a launcher: start N ranks of this script, one per GPU."""
     import socket
@@ -845,6 +853,8 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--algo", type=int, default=0)
+    ap.add_argument("--set", action="append", default=[], metavar="NAME=VALUE",
+                    help="experiment override of a tile heuristic (adaption_debug_set), e.g. --set pdl=0")
     args = ap.parse_args()
     if args.kernel is not None:
         run_kernel(args)

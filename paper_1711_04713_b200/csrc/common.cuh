@@ -188,6 +188,44 @@ inline int cuda_status(cudaError_t e, const char* where = "") {
   return e == cudaSuccess ? ADAPTION_OK : cuda_failure(e, where);
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------
+// A kernel launched with the stream-serialization attribute may start while its predecessor in the
+// stream is still running (its blocks take the SMs the predecessor's blocks leave), which hides the
+// launch latency between the many short kernels of a forward pass.  Such a kernel must not touch
+// global memory before pdl_wait(), which returns once the predecessor has completed and its writes
+// are visible; pdl_launch_dependents() lets the scheduler launch the successor as soon as resources
+// free up.  Both are no-ops in kernels launched the ordinary way.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// first statement of every kernel launched through launch_after_predecessor
+__device__ __forceinline__ void pdl_prologue() {
+  pdl_launch_dependents();
+  pdl_wait();
+}
+
+bool pdl_enabled();      // process-wide switch (adaption_debug_set "pdl")
+
+// Launch of a kernel whose first statement is pdl_prologue().
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after_predecessor(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream,
+                                            Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  if (pdl_enabled()) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- launches implemented in the other translation units ---------------------------------
 struct GemmProblem {
   // logical GEMM: rows M (pixels or batch), columns N (output channels), reduction over K

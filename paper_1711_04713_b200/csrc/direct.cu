@@ -35,6 +35,7 @@ __device__ __forceinline__ int64_t dot_row(const int8_t* __restrict__ ah, const 
 }
 
 __global__ void __launch_bounds__(256) direct_kernel(DirectParams p) {
+  pdl_prologue();
   const int64_t cols = p.mode == ADAPTION_MODE_RANGE ? p.N : p.y_stride;
   const size_t total = (size_t)p.M * (size_t)cols;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
@@ -101,6 +102,7 @@ struct FinalizeParams {
 
 // one thread per four consecutive output columns
 __global__ void __launch_bounds__(256) finalize_kernel(FinalizeParams p) {
+  pdl_prologue();
   const int64_t groups_per_row = (p.mode == ADAPTION_MODE_RANGE ? (p.N + 3) / 4 : p.y_stride / 4);
   const size_t total = (size_t)p.M * (size_t)groups_per_row;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
@@ -183,7 +185,7 @@ int launch_direct(const GemmProblem& g) {
   }
   const size_t items = (size_t)g.M * (size_t)(g.mode == ADAPTION_MODE_RANGE ? g.N : g.y.c_stride);
   if (items == 0) return ADAPTION_OK;
-  direct_kernel<<<grid_for(items), 256, 0, g.stream>>>(p);
+  launch_after_predecessor(direct_kernel, dim3(grid_for(items)), dim3(256), g.stream, p);
   return cuda_status(cudaGetLastError());
 }
 
@@ -203,7 +205,7 @@ int launch_finalize(const int64_t* acc, int64_t ld, const GemmProblem& g) {
   const size_t items =
       (size_t)g.M * (size_t)(g.mode == ADAPTION_MODE_RANGE ? (g.N + 3) / 4 : g.y.c_stride / 4);
   if (items == 0) return ADAPTION_OK;
-  finalize_kernel<<<grid_for(items), 256, 0, g.stream>>>(p);
+  launch_after_predecessor(finalize_kernel, dim3(grid_for(items)), dim3(256), g.stream, p);
   return cuda_status(cudaGetLastError());
 }
 

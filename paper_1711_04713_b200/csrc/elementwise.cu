@@ -37,6 +37,7 @@ static inline int stream_grid(size_t work_items, int threads, int blocks_per_sm)
 __global__ void __launch_bounds__(256) range_max_abs_kernel(const float* __restrict__ x, size_t numel,
                                                             size_t head, size_t n4,
                                                             float* __restrict__ d_max_abs) {
+  pdl_prologue();
   float m = 0.0f;
   const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(256) range_max_abs_kernel(const float* __restr
 // max >= 1 with binary exponent e (max in [2^e, 2^(e+1))) that is e+1; Inf has e = 128.
 __global__ void choose_fmt_kernel(const float* __restrict__ d_max_abs, int32_t n_bits,
                                   adaption_qfmt* __restrict__ d_fmt) {
+  pdl_prologue();
   const int bits = __float_as_int(*d_max_abs) & 0x7fffffff;
   const int e = (bits >> 23) - 127;
   int m = e >= 0 ? e + 1 : 0;
@@ -171,6 +173,7 @@ __global__ void __launch_bounds__(256) quantize_flat_kernel(const float4* __rest
                                                             const adaption_qfmt* __restrict__ d_fmt,
                                                             int relu, int32_t qmin, int32_t qmax,
                                                             adaption_stats* __restrict__ stats) {
+  pdl_prologue();
   if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
   const float scale = scale_of(frac_bits);
   Counts c;
@@ -204,6 +207,7 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restr
                                                             const adaption_qfmt* __restrict__ d_fmt,
                                                             int relu, int32_t qmin, int32_t qmax,
                                                             adaption_stats* __restrict__ stats) {
+  pdl_prologue();
   if (d_fmt != nullptr) frac_bits = d_fmt->frac_bits;
   const float scale = scale_of(frac_bits);
   Counts c;
@@ -437,6 +441,7 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const uint4* __restrict
                                                          uint4* __restrict__ out_lo,
                                                          int16_t* __restrict__ out_q16, int N, int H,
                                                          int W, int kw, int64_t in_vecs64, int64_t out_vecs64) {
+  pdl_prologue();
   // in_vecs / out_vecs: 16-byte vectors per pixel (c_stride / 16).  kw = 2: 2x2 windows; kw = 1: the
   // input is already the horizontal maximum of pixel pairs (W columns), only rows are paired.
   // H is even, so output row r = n * OH + oh (counted over the batch) pairs input rows 2r, 2r + 1.
@@ -529,12 +534,12 @@ int quantize_impl(const float* d_x, size_t outer, size_t inner, const adaption_q
   if ((int64_t)inner == out.c_stride && aligned16(d_x)) {
     const size_t n4 = outer * inner / 4;
     const int grid = stream_grid((n4 + 3) / 4, 256, 8);
-    quantize_flat_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const float4*>(d_x), n4, qo,
+    launch_after_predecessor(quantize_flat_kernel, dim3(grid), dim3(256), stream, reinterpret_cast<const float4*>(d_x), n4, qo,
                                                    out.fmt.frac_bits, d_fmt, relu, qmin, qmax, d_stats);
   } else {
     const size_t groups = outer * (size_t)(out.c_stride / 16);
     const int grid = stream_grid(groups, 256, 8);
-    quantize_rows_kernel<<<grid, 256, 0, stream>>>(d_x, outer, (int64_t)inner, out.c_stride, qo,
+    launch_after_predecessor(quantize_rows_kernel, dim3(grid), dim3(256), stream, d_x, outer, (int64_t)inner, out.c_stride, qo,
                                                    out.fmt.frac_bits, d_fmt, relu, qmin, qmax, d_stats);
   }
   return cuda_status(cudaGetLastError());
@@ -567,6 +572,7 @@ struct BatchArgs {
 };
 
 __global__ void __launch_bounds__(256) quantize_batch_kernel(const __grid_constant__ BatchArgs a) {
+  pdl_prologue();
   Counts unused;
   int t = 0;                       // chunks come in increasing order: the search only moves forward
   for (unsigned long long chunk = blockIdx.x; chunk < a.total_chunks; chunk += gridDim.x) {
@@ -613,7 +619,7 @@ int quantize_batch_impl(const adaption_quantize_item* h_items, int32_t n_items, 
   auto flush = [&]() -> int {
     if (args.n == 0) return ADAPTION_OK;
     const int grid = stream_grid((size_t)args.total_chunks, 1, 8);
-    quantize_batch_kernel<<<grid, 256, 0, stream>>>(args);
+    launch_after_predecessor(quantize_batch_kernel, dim3(grid), dim3(256), stream, args);
     args.n = 0;
     args.total_chunks = 0;
     return cuda_status(cudaGetLastError());
@@ -692,11 +698,12 @@ int measure_range_impl(const float* d_x, size_t numel, int32_t n_bits, float* d_
     if (head > numel) head = numel;
     const size_t n4 = (numel - head) / 4;
     int grid = stream_grid((n4 + 3) / 4 + 4, 256, 8);
-    range_max_abs_kernel<<<grid, 256, 0, stream>>>(d_x, numel, head, n4, d_max_abs);
+    launch_after_predecessor(range_max_abs_kernel, dim3(grid), dim3(256), stream, d_x, numel, head, n4, d_max_abs);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return ADAPTION_ERR_CUDA;
   }
-  if (d_fmt_out != nullptr) choose_fmt_kernel<<<1, 1, 0, stream>>>(d_max_abs, n_bits, d_fmt_out);
+  if (d_fmt_out != nullptr)
+    launch_after_predecessor(choose_fmt_kernel, dim3(1), dim3(1), stream, (const float*)d_max_abs, n_bits, d_fmt_out);
   return cuda_status(cudaGetLastError());
 }
 
@@ -723,9 +730,10 @@ int maxpool_impl(const adaption_qtensor& x, int32_t N, int32_t H, int32_t W, int
   const unsigned long long in_total = (unsigned long long)N * H * Win * (unsigned long long)in_vecs;
   const unsigned long long limit = (1ull << 32) - (unsigned long long)grid * 256ull;
   if (in_total < limit && (unsigned long long)total < limit)
-    maxpool2x2_kernel<uint32_t><<<grid, 256, 0, stream>>>(xh, xl, yh, yl, y.q16, N, H, Win, kw, in_vecs, out_vecs);
+    launch_after_predecessor(maxpool2x2_kernel<uint32_t>, dim3(grid), dim3(256), stream, xh, xl, yh, yl, y.q16, N, H, Win, kw,
+                             in_vecs, out_vecs);
   else
-    maxpool2x2_kernel<unsigned long long><<<grid, 256, 0, stream>>>(xh, xl, yh, yl, y.q16, N, H, Win, kw, in_vecs,
+    launch_after_predecessor(maxpool2x2_kernel<unsigned long long>, dim3(grid), dim3(256), stream, xh, xl, yh, yl, y.q16, N, H, Win, kw, in_vecs,
                                                                     out_vecs);
   return cuda_status(cudaGetLastError());
 }

@@ -69,6 +69,11 @@ struct TcParams {
   int b_resident;
   uint32_t b_res_off;
   int acc_bufs;
+  // Three accumulators of 128 columns leave one quarter of TMEM free: the high accumulator then
+  // alternates between the first and the last quarter from tile to tile (the other two stay put),
+  // and the epilogue hands the low and middle accumulators back before it reads the high one, so
+  // that the next tile's MMAs start while this tile's high accumulator is still being read.
+  int split_hh;
   uint32_t tmem_cols;
   int is_conv, OH, OW, S, cblks, w_pitch, stride_h, stride_w, pad_h, pad_w;
   const int16_t* bias;
@@ -592,8 +597,8 @@ struct Acc8 {
 };
 // sixteen columns as two groups of eight, one load instruction per accumulator
 template <int NACC>
-__device__ __forceinline__ void load_acc16(uint32_t taddr, int bn, Acc8<NACC>& x, Acc8<NACC>& y) {
-  tmem_ld16(taddr, x.a[0], y.a[0]);
+__device__ __forceinline__ void load_acc16(uint32_t taddr, uint32_t first_off, int bn, Acc8<NACC>& x, Acc8<NACC>& y) {
+  tmem_ld16(taddr + first_off, x.a[0], y.a[0]);
   if (NACC >= 2) tmem_ld16(taddr + (uint32_t)bn, x.a[1], y.a[1]);
   if (NACC == 3) tmem_ld16(taddr + 2u * (uint32_t)bn, x.a[2], y.a[2]);
 }
@@ -751,6 +756,20 @@ __device__ __forceinline__ bool epi_bar_all(int group, int threads, bool pred) {
   return r != 0;
 }
 
+// An epilogue warp hands accumulator columns back to the issuing warp (of the leader CTA in a pair).
+template <bool PAIR>
+__device__ __forceinline__ void release_accumulators(unsigned long long* bar_ptr, int lane) {
+  tc_fence_before();
+  __syncwarp();
+  if (lane == 0) {
+    const uint32_t bar = smem_u32(bar_ptr);
+    if (PAIR)
+      mbar_arrive_cluster(mapa_rank(bar, 0));
+    else
+      mbar_arrive(bar);
+  }
+}
+
 // ---------------------------------------------------------------------------------- kernel
 // GROUPED: stages hold several k-blocks and / or the weights are resident in shared memory (short
 // reductions); the plain variant keeps the issue loops free of that bookkeeping.
@@ -786,7 +805,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       mbar_init(smem_u32(&ctrl.full[s]), 1);
       mbar_init(smem_u32(&ctrl.empty[s]), 1);
     }
-    for (int b = 0; b < p.acc_bufs; ++b) {
+    for (int b = 0; b < kMaxAccBufs; ++b) {
       mbar_init(smem_u32(&ctrl.tmem_full[b]), 1);
       mbar_init(smem_u32(&ctrl.tmem_empty[b]), (uint32_t)((PAIR ? 2 : 1) * (kEpiWarps / p.epi_groups)));
     }
@@ -804,6 +823,10 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   if (PAIR) cluster_sync_all();      // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = ctrl.tmem_base;
+  // Everything above touched only this block's shared and tensor memory.  From here on global memory
+  // is read (operands) and written (outputs, counters): wait for the previous kernel of the stream.
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp < kProducerWarps) {
     // ------------------------------------------------------------------ TMA producers
@@ -972,11 +995,20 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const uint32_t bph = (tile_iter / (uint32_t)p.acc_bufs) & 1u;
         if (lane == 0) TL_STAMP(1, tile_iter, 0);
         ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.tmem_empty[buf]), bph ^ 1u, &ctrl, p, false));
+        // split release: barrier 0 above covers the middle and low accumulators, barriers 1 and 2
+        // the two places of the high one
+        const uint32_t hh_sel = (NACC == 3 && p.split_hh) ? (tile_iter & 1u) : 0u;
+        if (ok && NACC == 3 && p.split_hh)
+          ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&ctrl.tmem_empty[1u + hh_sel]), ((tile_iter >> 1) & 1u) ^ 1u,
+                                                &ctrl, p, false));
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) TL_STAMP(1, tile_iter, 1);
-        const uint32_t d0 = tmem_base + buf * (uint32_t)(NACC * p.BN);
-        const uint32_t d1 = d0 + (uint32_t)p.BN, d2 = d0 + 2u * (uint32_t)p.BN;
+        // accumulator columns of this tile: the set's three (or fewer) consecutive groups of BN
+        // columns, except that with the split release the first (high) one may sit in the last quarter
+        const uint32_t dset = tmem_base + buf * (uint32_t)(NACC * p.BN);
+        const uint32_t d0 = dset + hh_sel * (uint32_t)(3 * p.BN);
+        const uint32_t d1 = dset + (uint32_t)p.BN, d2 = dset + 2u * (uint32_t)p.BN;
         uint32_t bres = bres_lo + (uint32_t)tc.kb_begin * bres_u;   // resident weights of this k-block
         for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps) {
           const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;
@@ -1120,6 +1152,12 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       const int m = tc.m0 + (int)rank * kBM + row;
       const bool row_ok = m < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * (uint32_t)(NACC * p.BN);
+      // where this tile's high accumulator lives, and the barrier that hands it back
+      const bool split = NACC == 3 && p.split_hh != 0;
+      const uint32_t hh_sel = split ? (tile_iter & 1u) : 0u;
+      const uint32_t hh_off = hh_sel * (uint32_t)(3 * p.BN);
+      unsigned long long* const bar_rest = &ctrl.tmem_empty[buf];
+      unsigned long long* const bar_hh = split ? &ctrl.tmem_empty[1u + hh_sel] : bar_rest;
       // Sixteen columns per step.  The accumulators are handed back to the issuing warp as soon as
       // the last step's values are in registers, before the arithmetic on them.
       const bool storing = FAST || (p.splits == 1 && p.mode == ADAPTION_MODE_REQUANT);
@@ -1130,15 +1168,8 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       // (the host launches the FAST kernels only where every warp owns a multiple of 32 columns)
       if (FAST) {
         if (col_begin >= col_end) {          // a warp without columns only hands the accumulators back
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
-            if (PAIR)
-              mbar_arrive_cluster(mapa_rank(bar, 0));
-            else
-              mbar_arrive(bar);
-          }
+          release_accumulators<PAIR>(bar_rest, lane);
+          if (split) release_accumulators<PAIR>(bar_hh, lane);
           released = true;
         }
         for (int c0 = col_begin; c0 < col_end; c0 += 32) {
@@ -1157,6 +1188,11 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           tmem_ld_wait();
           pin_after_wait32(t);
           if (NACC >= 2) pin_after_wait32(h);
+          // the low and middle accumulators are in registers: with the split release they go back now
+          if (split && c0 + 32 >= col_end) {
+            release_accumulators<PAIR>(bar_rest, lane);
+            if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 3);
+          }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const int4 c = cl4[j];
@@ -1170,20 +1206,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             }
           }
           if (NACC == 3) {
-            tmem_ld32(taddr + (uint32_t)c0, h);                    // hh
+            tmem_ld32(taddr + hh_off + (uint32_t)c0, h);           // hh
             tmem_ld_wait();
             pin_after_wait32(h);
           }
           if (c0 + 32 >= col_end) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-              const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
-              if (PAIR)
-                mbar_arrive_cluster(mapa_rank(bar, 0));
-              else
-                mbar_arrive(bar);
-            }
+            release_accumulators<PAIR>(bar_hh, lane);
+            if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 4);
             released = true;
           }
           if (NACC >= 2) {                                         // H = hh + Ch
@@ -1229,21 +1258,14 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const bool have = c0 < col_end;
         Acc8<NACC> xa, xb;
         if (have) {
-          load_acc16<NACC>(taddr + c0, p.BN, xa, xb);
+          load_acc16<NACC>(taddr + c0, hh_off, p.BN, xa, xb);
           tmem_ld_wait();
           pin_acc8<NACC>(xa);
           pin_acc8<NACC>(xb);
         }
         if (c0 + 16 >= col_end) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            const uint32_t bar = smem_u32(&ctrl.tmem_empty[buf]);
-            if (PAIR)
-              mbar_arrive_cluster(mapa_rank(bar, 0));
-            else
-              mbar_arrive(bar);
-          }
+          release_accumulators<PAIR>(bar_rest, lane);
+          if (split) release_accumulators<PAIR>(bar_hh, lane);
           released = true;
         }
         if (!have) break;
@@ -1379,11 +1401,11 @@ struct TcConfig {
 // from the environment, so the layer calls themselves do no string work).  Each holds its
 // default until set; the setter is the only writer.
 enum Knob { kSplits, kPair, kFast, kStaged, kStages, kBK, kBN, kKps, kBres, kWide, kEpiGroups, kTimeoutUs, kStallAt,
-            kNumKnobs };
+            kSplitHh, kPdl, kNumKnobs };
 const char* const kKnobNames[kNumKnobs] = {"splits", "pair", "fast", "staged", "stages", "bk", "bn", "kps", "bres",
-                                           "wide", "epigroups", "timeout_us", "stall_at"};
-const int kKnobDefaults[kNumKnobs] = {0, -1, 1, 1, 0, 0, 0, 0, 1, 1, 2, 0, -1};
-std::atomic<int> g_knobs[kNumKnobs] = {{0}, {-1}, {1}, {1}, {0}, {0}, {0}, {0}, {1}, {1}, {2}, {0}, {-1}};
+                                           "wide", "epigroups", "timeout_us", "stall_at", "split_hh", "pdl"};
+const int kKnobDefaults[kNumKnobs] = {0, -1, 1, 1, 0, 0, 0, 0, 1, 1, 2, 0, -1, 1, 1};
+std::atomic<int> g_knobs[kNumKnobs] = {{0}, {-1}, {1}, {1}, {0}, {0}, {0}, {0}, {1}, {1}, {2}, {0}, {-1}, {1}, {1}};
 inline int knob(Knob k) { return g_knobs[k].load(std::memory_order_relaxed); }
 
 TcConfig make_config_impl(const GemmProblem& g, bool allow_wide);
@@ -1599,15 +1621,23 @@ int launch_kernel(const CUtensorMap* maps, const TcParams& p, int grid, size_t s
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
+  unsigned n_attr = 0;
   if (PAIR) {
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+    attr[n_attr].val.clusterDim.x = 2;
+    attr[n_attr].val.clusterDim.y = 1;
+    attr[n_attr].val.clusterDim.z = 1;
+    ++n_attr;
   }
+  if (knob(kPdl) != 0) {
+    // the kernel waits for its predecessor itself (pdl_wait) before it touches global memory
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
+  }
+  cfg.attrs = n_attr ? attr : nullptr;
+  cfg.numAttrs = n_attr;
   const cudaError_t le =
       cudaLaunchKernelEx(&cfg, lp_gemm_kernel<NAX, NBW, PAIR, GROUPED, EPI>, maps[0], maps[1], maps[2], maps[3], maps[4],
                          maps[5], p);
@@ -1752,6 +1782,8 @@ extern "C" __attribute__((visibility("default"))) int adaption_debug_timeline(lo
 }
 #endif
 
+bool pdl_enabled() { return knob(kPdl) != 0; }
+
 int debug_set(const char* name, int value) {
   if (name == nullptr) return ADAPTION_ERR_INVALID_ARG;
   if (std::strcmp(name, "reset") == 0) {
@@ -1827,6 +1859,8 @@ int launch_tensor(const GemmProblem& g) {
   p.b_resident = c.b_resident ? 1 : 0;
   p.b_res_off = (uint32_t)c.stages * c.stage_bytes;
   p.acc_bufs = c.acc_bufs; p.tmem_cols = c.tmem_cols;
+  p.split_hh = (c.nacc == 3 && c.acc_bufs == 1 && 4 * c.BN <= 512 && knob(kSplitHh) != 0) ? 1 : 0;
+  if (p.split_hh) p.tmem_cols = 512;
   p.is_conv = g.is_conv ? 1 : 0;
   if (g.is_conv) {
     p.OH = g.OH; p.OW = g.OW; p.S = g.cs.S; p.cblks = c.cblks; p.w_pitch = (int)g.w.c_stride;

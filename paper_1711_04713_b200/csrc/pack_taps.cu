@@ -70,6 +70,7 @@ __device__ __forceinline__ void pack_row(const uint8_t* __restrict__ src, long l
 
 template <int C>
 __global__ void __launch_bounds__(256) pack_taps_kernel(const PackParams p) {
+  pdl_prologue();
   const int taps = p.R * p.S;
   for (long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x; m < p.rows;
        m += (long long)gridDim.x * blockDim.x) {
@@ -117,10 +118,10 @@ int launch_pack(const PackParams& p, int C, cudaStream_t stream) {
   const long long cap = (long long)num_sms() * 16;
   if (blocks > cap) blocks = cap;
   switch (C) {
-    case 1: pack_taps_kernel<1><<<(unsigned)blocks, 256, 0, stream>>>(p); break;
-    case 2: pack_taps_kernel<2><<<(unsigned)blocks, 256, 0, stream>>>(p); break;
-    case 3: pack_taps_kernel<3><<<(unsigned)blocks, 256, 0, stream>>>(p); break;
-    default: pack_taps_kernel<4><<<(unsigned)blocks, 256, 0, stream>>>(p); break;
+    case 1: launch_after_predecessor(pack_taps_kernel<1>, dim3((unsigned)blocks), dim3(256), stream, p); break;
+    case 2: launch_after_predecessor(pack_taps_kernel<2>, dim3((unsigned)blocks), dim3(256), stream, p); break;
+    case 3: launch_after_predecessor(pack_taps_kernel<3>, dim3((unsigned)blocks), dim3(256), stream, p); break;
+    default: launch_after_predecessor(pack_taps_kernel<4>, dim3((unsigned)blocks), dim3(256), stream, p); break;
   }
   return cuda_status(cudaGetLastError(), "pack_taps_kernel launch");
 }

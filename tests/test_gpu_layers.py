@@ -282,6 +282,19 @@ def test_conv_few_channels_packed_taps(case, with_q16):
     assert need >= N * OH * OW * 32 * ((nx > 8) + 1)      # the packed planes are in the workspace
 
 
+@pytest.mark.parametrize("case", [
+    (20, 56, 56, 128, 128, 3, 1, 1, 16, 16, 16, True),     # 245 pair tiles / 490 single tiles of 128 columns
+    (9, 56, 56, 128, 200, 3, 1, 1, 16, 16, 16, False),     # generic epilogue, two column tiles, ragged N
+    (40, 28, 28, 256, 128, 3, 1, 1, 16, 16, 12, True),     # 18 k-blocks, 12-bit outputs
+])
+@pytest.mark.parametrize("split_hh", [1, 0])
+def test_conv_many_tiles_per_cta(case, split_hh, cta_mode):
+    """More tiles than CTAs, so that every persistent CTA walks several tiles: the accumulator sets
+    (and, for three 128-column accumulators, the alternating place of the high one) rotate."""
+    B.adaption_debug_set("split_hh", split_hh)
+    run_conv_case(np.random.default_rng(sum(case)), *case, B.ALGO_TENSOR, with_q16=False)
+
+
 def test_conv_tensor_extreme_operands(cta_mode):
     # every operand at +-full scale: largest possible partial sums in all three accumulators
     run_conv_case(np.random.default_rng(1), 1, 32, 32, 256, 128, 3, 1, 1, 16, 16, 16, False, B.ALGO_TENSOR,
