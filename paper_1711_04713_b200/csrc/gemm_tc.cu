@@ -1379,6 +1379,7 @@ struct TcConfig {
   int nax = 1, nbw = 1, nacc = 1;
   int stages = 0;
   uint32_t a_bytes = 0, b_bytes = 0, stage_bytes = 0;
+  int a_rows = kBM;            // rows of the activation tile that are staged
   int acc_bufs = 1;
   uint32_t tmem_cols = 32;
   int num_kb = 0, splits = 1, kb_per_split = 0;
@@ -1514,7 +1515,12 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
     c.tile_m = 2 * kBM;
     c.tiles_m = (int)((g.M + c.tile_m - 1) / c.tile_m);
   }
-  c.a_bytes = (uint32_t)(kBM * c.BK);
+  // Inner products on a small batch: only the rows that exist are staged (the MMA still covers 128
+  // rows; the rest reads whatever follows in the stage and lands in accumulator rows nobody stores).
+  // Smaller stages mean a deeper ring, i.e. more weight bytes in flight per SM, which is what bounds
+  // these weight-streaming layers.
+  c.a_rows = (!g.is_conv && !c.pair && g.M <= 64) ? 64 : kBM;
+  c.a_bytes = (uint32_t)(c.a_rows * c.BK);
   c.b_bytes = (uint32_t)((c.pair ? c.BN / 2 : c.BN) * c.BK);
   // Output staging: one plane of 128 rows x BN bytes per output byte plane.  Needs a tensor map over
   // the output planes (pitch a multiple of 16 bytes and at least one tile wide) and no int16 copy.
@@ -1824,7 +1830,7 @@ int launch_tensor(const GemmProblem& g) {
       ok = encode_im2col_nhwc(&maps[i], xa[i], g.cs, g.x.c_stride, (uint32_t)c.BK, c.swizzle);
     else
       ok = encode_tiled_2d(&maps[i], xa[i], (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.x.c_stride,
-                           (uint32_t)c.BK, (uint32_t)kBM, c.swizzle);
+                           (uint32_t)c.BK, (uint32_t)c.a_rows, c.swizzle);
     if (!ok) return ADAPTION_ERR_CUDA;
     const uint64_t wk = g.is_conv ? (uint64_t)g.cs.R * g.cs.S * g.w.c_stride : (uint64_t)g.K;
     const uint64_t wpitch = g.is_conv ? wk : (uint64_t)g.w.c_stride;
