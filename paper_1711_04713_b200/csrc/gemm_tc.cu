@@ -74,6 +74,11 @@ struct TcParams {
   // and the epilogue hands the low and middle accumulators back before it reads the high one, so
   // that the next tile's MMAs start while this tile's high accumulator is still being read.
   int split_hh;
+  // With the split release: the last two k-blocks of a tile are issued product by product (all low
+  // products, then the middle ones, then the high ones) with a completion signal after each group,
+  // so that the epilogue pulls the low and the middle accumulator into registers while the
+  // remaining MMAs of the tile still run, and the next tile's MMAs can follow almost at once.
+  int tail_stagger;
   uint32_t tmem_cols;
   int is_conv, OH, OW, S, cblks, w_pitch, stride_h, stride_w, pad_h, pad_w;
   const int16_t* bias;
@@ -118,6 +123,7 @@ struct Ctrl {
   unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[kMaxAccBufs];
   unsigned long long tmem_empty[kMaxAccBufs];
+  unsigned long long part_full[2];   // staggered tail: low accumulator complete, middle accumulator complete
   unsigned long long drain;     // the issuing warp's last commit before an early exit
   unsigned long long b_ready;   // resident weights have landed
   uint32_t tmem_base;
@@ -460,6 +466,22 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctrl* ct
                                          bool relaxed = true) {
   if (mbar_try_wait(bar, parity)) return true;
   return wait_slow(bar, parity, ctrl, p, relaxed);
+}
+
+// The same bounded wait without a function call, for waits that sit between TMEM loads whose
+// results are live in registers (a call there would make the compiler save and restore them).
+__device__ __forceinline__ bool wait_bar_inline(uint32_t bar, uint32_t parity, Ctrl* ctrl, const TcParams& p) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (!mbar_try_wait_suspend(bar, parity, 1000u)) {
+    if (ctrl->abort) return false;
+    if (global_ns() - t0 > p.timeout_ns) {
+      ctrl->abort = 1;
+      atomicExch(&p.stats->status, (int)ADAPTION_ERR_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
 }
 
 struct TileCoord {
@@ -809,6 +831,8 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       mbar_init(smem_u32(&ctrl.tmem_full[b]), 1);
       mbar_init(smem_u32(&ctrl.tmem_empty[b]), (uint32_t)((PAIR ? 2 : 1) * (kEpiWarps / p.epi_groups)));
     }
+    mbar_init(smem_u32(&ctrl.part_full[0]), 1);
+    mbar_init(smem_u32(&ctrl.part_full[1]), 1);
     mbar_init(smem_u32(&ctrl.drain), 1);
     mbar_init(smem_u32(&ctrl.b_ready), 1);
     ctrl.abort = 0;
@@ -1010,7 +1034,9 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const uint32_t d0 = dset + hh_sel * (uint32_t)(3 * p.BN);
         const uint32_t d1 = dset + (uint32_t)p.BN, d2 = dset + 2u * (uint32_t)p.BN;
         uint32_t bres = bres_lo + (uint32_t)tc.kb_begin * bres_u;   // resident weights of this k-block
-        for (int kb = tc.kb_begin; kb < tc.kb_end; kb += kps) {
+        const bool stagger = !GROUPED && NAX == 2 && NBW == 2 && p.tail_stagger != 0;
+        const int kb_main_end = stagger ? tc.kb_end - 2 : tc.kb_end;
+        for (int kb = tc.kb_begin; kb < kb_main_end; kb += kps) {
           const int nkb = GROUPED ? min(kps, tc.kb_end - kb) : 1;
           {
 #ifdef ADAPTION_TIMELINE
@@ -1072,6 +1098,50 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             a0 = ring_lo;
             full_bar = full_bar0;
             empty_bar = empty_bar0;
+          }
+        }
+        if (ok && stagger) {
+          // The two last k-blocks together, product by product.  (Integer accumulation: the order of
+          // the MMAs does not matter.)  Both stages are handed back at the end.
+          uint32_t st_a[2], st_full[2], st_empty[2], st_ph[2];
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            st_a[j] = a0; st_full[j] = full_bar; st_empty[j] = empty_bar; st_ph[j] = ph;
+            a0 += stage_u;
+            full_bar += 8u;
+            empty_bar += 8u;
+            if (++s == p.stages) {
+              s = 0;
+              ph ^= 1u;
+              a0 = ring_lo;
+              full_bar = full_bar0;
+              empty_bar = empty_bar0;
+            }
+          }
+          ok = __all_sync(0xffffffffu, wait_bar(st_full[0], st_ph[0], &ctrl, p, false));
+          if (ok) ok = __all_sync(0xffffffffu, wait_bar(st_full[1], st_ph[1], &ctrl, p, false));
+          if (!ok) break;
+          tc_fence_after();
+          if (elect_one()) {
+            const uint32_t off_b1 = off_b0 + b_u;
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              for (int ks = 0; ks < ksteps; ++ks)                     // lo * lo
+                mma_i8<PAIR>(d2, st_a[j] + off_a1 + 2u * ks, st_a[j] + off_b1 + 2u * ks, dhi, id_uu, 1u);
+            tc_commit<PAIR>(smem_u32(&ctrl.part_full[0]));
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              for (int ks = 0; ks < ksteps; ++ks) {                   // hi * lo and lo * hi
+                mma_i8<PAIR>(d1, st_a[j] + 2u * ks, st_a[j] + off_b1 + 2u * ks, dhi, id_su, 1u);
+                mma_i8<PAIR>(d1, st_a[j] + off_a1 + 2u * ks, st_a[j] + off_b0 + 2u * ks, dhi, id_us, 1u);
+              }
+            tc_commit<PAIR>(smem_u32(&ctrl.part_full[1]));
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+              for (int ks = 0; ks < ksteps; ++ks)                     // hi * hi
+                mma_i8<PAIR>(d0, st_a[j] + 2u * ks, st_a[j] + off_b0 + 2u * ks, dhi, id_ss, 1u);
+            tc_commit<PAIR>(st_empty[0]);
+            tc_commit<PAIR>(st_empty[1]);
           }
         }
         if (ok && elect_one()) tc_commit<PAIR>(smem_u32(&ctrl.tmem_full[buf]));   // tile complete
@@ -1142,7 +1212,9 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       // the previous tile's bulk stores must have read the staging planes before they are reused
       if (p.staged && store_leader) bulk_wait_read_all();
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 0);
-      bool w = wait_bar(smem_u32(&ctrl.tmem_full[buf]), bph, &ctrl, p);
+      // (staggered tail: the first thing to wait for is the low accumulator)
+      const bool stagger = FAST && NACC == 3 && p.tail_stagger != 0;
+      bool w = wait_bar(smem_u32(stagger ? &ctrl.part_full[0] : &ctrl.tmem_full[buf]), bph, &ctrl, p);
       // one decision for all epilogue warps (they meet at barriers below), which also publishes the
       // constants and the free staging planes
       w = epi_bar_all(group, gthreads, w);
@@ -1162,6 +1234,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       // the last step's values are in registers, before the arithmetic on them.
       const bool storing = FAST || (p.splits == 1 && p.mode == ADAPTION_MODE_REQUANT);
       bool released = false;
+      bool tile_ok = true;        // a later wait of this tile gave up: finish the tile, then leave together
       // Fast path with thirty-two columns per warp step: one TMEM load per accumulator, the low and
       // middle accumulators first (they fold into T), the high one last; the accumulators go back
       // to the issuing warp as soon as the last load has landed.
@@ -1178,7 +1251,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           const int4* ch4 = reinterpret_cast<const int4*>(reinterpret_cast<const int*>(colconst) + p.BN + c0);
           if (NACC == 3) {
             tmem_ld32(taddr + (uint32_t)(c0 + 2 * p.BN), t);       // ll
-            tmem_ld32(taddr + (uint32_t)(c0 + p.BN), h);           // mid
+            if (!stagger) tmem_ld32(taddr + (uint32_t)(c0 + p.BN), h);   // mid
           } else if (NACC == 2) {
             tmem_ld32(taddr + (uint32_t)(c0 + p.BN), t);           // weight 1
             tmem_ld32(taddr + (uint32_t)c0, h);                    // weight 2^8
@@ -1187,7 +1260,25 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           }
           tmem_ld_wait();
           pin_after_wait32(t);
-          if (NACC >= 2) pin_after_wait32(h);
+          if (NACC >= 2 && !stagger) pin_after_wait32(h);
+          if (NACC == 3 && stagger) {
+            // fold the constant into the low accumulator while the middle one completes, then fetch it
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int4 c = cl4[j];
+              t[4 * j + 0] = (t[4 * j + 0] + c.x) >> 8;
+              t[4 * j + 1] = (t[4 * j + 1] + c.y) >> 8;
+              t[4 * j + 2] = (t[4 * j + 2] + c.z) >> 8;
+              t[4 * j + 3] = (t[4 * j + 3] + c.w) >> 8;
+            }
+            tile_ok = wait_bar_inline(smem_u32(&ctrl.part_full[1]), bph, &ctrl, p) && tile_ok;
+            tc_fence_after();
+            tmem_ld32(taddr + (uint32_t)(c0 + p.BN), h);           // mid
+            tmem_ld_wait();
+            pin_after_wait32(h);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) t[j] += h[j];             // T
+          }
           // the low and middle accumulators are in registers: with the split release they go back now
           if (split && c0 + 32 >= col_end) {
             release_accumulators<PAIR>(bar_rest, lane);
@@ -1195,6 +1286,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
           }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
+            if (NACC == 3 && stagger) break;
             const int4 c = cl4[j];
             if (NACC >= 2) {                                       // T = mid + floor((ll + Cl) / 2^8)
               t[4 * j + 0] = h[4 * j + 0] + ((t[4 * j + 0] + c.x) >> 8);
@@ -1206,6 +1298,10 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             }
           }
           if (NACC == 3) {
+            if (stagger) {
+              tile_ok = wait_bar_inline(smem_u32(&ctrl.tmem_full[buf]), bph, &ctrl, p) && tile_ok;
+              tc_fence_after();
+            }
             tmem_ld32(taddr + hh_off + (uint32_t)c0, h);           // hh
             tmem_ld_wait();
             pin_after_wait32(h);
@@ -1307,7 +1403,13 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       // the channel pitch are clipped by the tensor map); the barrier also ends this tile's reads
       // of the per-column constants
       if (p.staged) fence_async_shared();
-      epi_bar_sync(group, gthreads);
+      if (stagger) {
+        // the same barrier also carries the verdict on this tile's later waits, so that all warps
+        // of the group leave together if one of them gave up
+        if (!epi_bar_all(group, gthreads, tile_ok)) { ok = false; break; }
+      } else {
+        epi_bar_sync(group, gthreads);
+      }
       if (p.staged && store_leader) {
         const int m_first = (tc.m0 + (int)rank * kBM) >> (p.pool_w ? 1 : 0);     // row of the stored tensor
         for (int sub = 0; sub * 128 < p.BN; ++sub) {
@@ -1402,11 +1504,11 @@ struct TcConfig {
 // from the environment, so the layer calls themselves do no string work).  Each holds its
 // default until set; the setter is the only writer.
 enum Knob { kSplits, kPair, kFast, kStaged, kStages, kBK, kBN, kKps, kBres, kWide, kEpiGroups, kTimeoutUs, kStallAt,
-            kSplitHh, kPdl, kNumKnobs };
+            kSplitHh, kPdl, kStagger, kNumKnobs };
 const char* const kKnobNames[kNumKnobs] = {"splits", "pair", "fast", "staged", "stages", "bk", "bn", "kps", "bres",
-                                           "wide", "epigroups", "timeout_us", "stall_at", "split_hh", "pdl"};
-const int kKnobDefaults[kNumKnobs] = {0, -1, 1, 1, 0, 0, 0, 0, 1, 1, 2, 0, -1, 1, 1};
-std::atomic<int> g_knobs[kNumKnobs] = {{0}, {-1}, {1}, {1}, {0}, {0}, {0}, {0}, {1}, {1}, {2}, {0}, {-1}, {1}, {1}};
+                                           "wide", "epigroups", "timeout_us", "stall_at", "split_hh", "pdl", "stagger"};
+const int kKnobDefaults[kNumKnobs] = {0, -1, 1, 1, 0, 0, 0, 0, 1, 1, 2, 0, -1, 1, 1, 1};
+std::atomic<int> g_knobs[kNumKnobs] = {{0}, {-1}, {1}, {1}, {0}, {0}, {0}, {0}, {1}, {1}, {2}, {0}, {-1}, {1}, {1}, {1}};
 inline int knob(Knob k) { return g_knobs[k].load(std::memory_order_relaxed); }
 
 TcConfig make_config_impl(const GemmProblem& g, bool allow_wide);
@@ -1913,6 +2015,9 @@ int launch_tensor(const GemmProblem& g) {
     if (single) ok32 = kred * 16384 + cmax < lim;
     p.fast_relu = ok32 ? 1 : 0;
   }
+  const bool grouped_kernel = c.kps > 1 || c.b_resident;
+  p.tail_stagger = (p.split_hh && p.fast_relu && !grouped_kernel && c.kb_per_split >= 3 && c.stages >= 3 &&
+                    c.nax == 2 && c.nbw == 2 && knob(kStagger) != 0) ? 1 : 0;
   p.ws = (long long*)g.workspace; p.ws_ld = g.N;
   p.stats = g.stats;
   p.timeout_ns = knob(kTimeoutUs) > 0 ? 1000ull * (unsigned long long)knob(kTimeoutUs) : 2000000000ull;
