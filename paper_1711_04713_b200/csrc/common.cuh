@@ -199,10 +199,13 @@ __device__ __forceinline__ void pdl_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-// first statement of every kernel launched through launch_after_predecessor
+// First statement of every kernel launched through launch_after_predecessor: wait for the
+// predecessor, and only then let the successor be scheduled.  (The other order - announcing the
+// successor before this kernel has itself synchronised with its predecessor - was tried: a chain of
+// three short kernels then once let the third read what the second had only partly written.)
 __device__ __forceinline__ void pdl_prologue() {
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
 }
 
 bool pdl_enabled();      // process-wide switch (adaption_debug_set "pdl")

@@ -849,8 +849,8 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
   const uint32_t tmem_base = ctrl.tmem_base;
   // Everything above touched only this block's shared and tensor memory.  From here on global memory
   // is read (operands) and written (outputs, counters): wait for the previous kernel of the stream.
-  pdl_launch_dependents();
   pdl_wait();
+  pdl_launch_dependents();
 
   if (warp < kProducerWarps) {
     // ------------------------------------------------------------------ TMA producers
@@ -862,7 +862,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     // Planes that are streamed through the ring: all of them, or only the activation planes when
     // the weights are resident.  With fewer streamed planes than producer warps, several warps
     // share a plane and take turns stage by stage.
-    const bool b_res = GROUPED && !PAIR && p.b_resident;
+    const bool b_res = GROUPED && p.b_resident;
     const int nact = b_res ? NAX : NPLANES;
     const int kps = GROUPED ? p.kps : 1;
     const int nsub = nact >= kProducerWarps ? 1 : kProducerWarps / nact;   // warps per streamed plane
@@ -883,15 +883,18 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       if (b_res && warp == kProducerWarps - 1) {
         // the whole weight matrix of this (single) column tile, one copy per k-block and plane,
         // all reporting to one barrier
+        // (in a pair each CTA fetches its own half of the weight rows; the bytes of both are counted
+        // on the leader's barrier, which the leader arms for both)
         if (elect_one()) {
-          const uint32_t bar = smem_u32(&ctrl.b_ready);
-          mbar_expect_tx(bar, (uint32_t)p.num_kb * NBW * p.b_bytes);
+          uint32_t bar = smem_u32(&ctrl.b_ready);
+          if (rank == 0) mbar_expect_tx(bar, (PAIR ? 2u : 1u) * (uint32_t)p.num_kb * NBW * p.b_bytes);
+          if (PAIR) bar = mapa_rank(bar, 0);
           for (int kb = 0; kb < p.num_kb; ++kb) {
             const int kcol = p.is_conv ? (kb / p.cblks) * p.w_pitch + (kb % p.cblks) * p.BK : kb * p.BK;
             for (int bplane = 0; bplane < NBW; ++bplane) {
               const uint32_t dst =
                   ring + p.b_res_off + (uint32_t)kb * (NBW * p.b_bytes) + (uint32_t)bplane * p.b_bytes;
-              tma_load_2d<false>(dst, bplane == 0 ? &map_b0 : &map_b1, bar, kcol, 0);
+              tma_load_2d<PAIR>(dst, bplane == 0 ? &map_b0 : &map_b1, bar, kcol, (int)rank * b_rows);
             }
           }
         }
@@ -962,9 +965,15 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       }
       const bool is_b_loader = b_res && warp == kProducerWarps - 1;
       if (ctrl.abort && lane == 0 && is_b_loader) {
-        // another role gave up: let the resident-weight copies land before the CTA exits
+        // another role gave up: let the resident-weight copies land before the CTA exits (the
+        // follower of a pair cannot see the leader's barrier: it waits a fixed time)
         const unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(smem_u32(&ctrl.b_ready), 0) && global_ns() - t0 < 50000000ull) {
+        if (PAIR && rank != 0) {
+          while (global_ns() - t0 < 2000000ull) {
+          }
+        } else {
+          while (!mbar_try_wait(smem_u32(&ctrl.b_ready), 0) && global_ns() - t0 < 50000000ull) {
+          }
         }
       }
       if ((!ok || ctrl.abort) && lane == 0) {
@@ -1006,7 +1015,7 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
       uint32_t a0 = ring_lo, full_bar = full_bar0, empty_bar = empty_bar0;
       int s = 0;
       bool ok = true;
-      const bool b_res = GROUPED && !PAIR && p.b_resident;
+      const bool b_res = GROUPED && p.b_resident;
       const int kps = GROUPED ? p.kps : 1;
       const uint32_t bres_lo = smem_desc_lo(ring + p.b_res_off), bres_u = NBW * b_u;
       if (b_res) {
@@ -1655,7 +1664,7 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
   // stream only the activation planes (fewer bulk copies per k-block for the 64-channel and
   // 3-channel layers).  Only if at least three activation stages still fit.
   const size_t res_bytes = (size_t)c.num_kb * c.nbw * c.b_bytes;
-  if (!c.pair && c.tiles_n == 1 && c.splits == 1 && c.tiles_m >= 4 * sms &&
+  if (c.tiles_n == 1 && c.splits == 1 && c.tiles_m >= 4 * sms && (!c.pair || knob(kBres) != 2) &&
       res_bytes + 3 * (size_t)c.kps * c.nax * c.a_bytes + 1024 <= budget && knob(kBres) != 0) {
     c.b_resident = true;
     c.b_res_bytes = (uint32_t)res_bytes;
