@@ -406,6 +406,9 @@ __global__ void __launch_bounds__(256) requant_flat_kernel(const uint4* __restri
 // 2x2 / stride 2 max-pool on stored integers; 16 channels (one 16-byte vector per plane) per
 // thread.  Exact on the quantized values because the quantizer is monotone.
 // ------------------------------------------------------------------------------------------
+// Sixteen values at once, four per 32-bit word, without unpacking the byte planes: a candidate
+// 256*qh + ql beats the current 256*ph + pl iff qh > ph (signed bytes) or qh == ph and ql > pl
+// (unsigned bytes); the per-byte comparison masks then select whole bytes in both planes.
 __device__ __forceinline__ void max16(uint4& bh, uint4& bl, const uint4& h, const uint4& l, bool two) {
   uint32_t* ph = reinterpret_cast<uint32_t*>(&bh);
   uint32_t* pl = reinterpret_cast<uint32_t*>(&bl);
@@ -413,23 +416,13 @@ __device__ __forceinline__ void max16(uint4& bh, uint4& bl, const uint4& h, cons
   const uint32_t* ql = reinterpret_cast<const uint32_t*>(&l);
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    uint32_t oh = 0, ol = 0;
-#pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      int32_t cur, cand;
-      if (two) {
-        cur = ((int32_t)(int8_t)((ph[w] >> (8 * b)) & 255)) * 256 + (int32_t)((pl[w] >> (8 * b)) & 255);
-        cand = ((int32_t)(int8_t)((qh[w] >> (8 * b)) & 255)) * 256 + (int32_t)((ql[w] >> (8 * b)) & 255);
-      } else {
-        cur = (int32_t)(int8_t)((pl[w] >> (8 * b)) & 255);
-        cand = (int32_t)(int8_t)((ql[w] >> (8 * b)) & 255);
-      }
-      const int32_t m = cand > cur ? cand : cur;
-      ol |= (uint32_t)(m & 255) << (8 * b);
-      oh |= (uint32_t)((m >> 8) & 255) << (8 * b);
+    if (two) {
+      const uint32_t m = __vcmpgts4(qh[w], ph[w]) | (__vcmpeq4(qh[w], ph[w]) & __vcmpgtu4(ql[w], pl[w]));
+      ph[w] = (qh[w] & m) | (ph[w] & ~m);
+      pl[w] = (ql[w] & m) | (pl[w] & ~m);
+    } else {
+      pl[w] = __vmaxs4(pl[w], ql[w]);       // one plane of signed bytes
     }
-    ph[w] = oh;
-    pl[w] = ol;
   }
 }
 
@@ -574,27 +567,42 @@ struct BatchArgs {
 __global__ void __launch_bounds__(256) quantize_batch_kernel(const __grid_constant__ BatchArgs a) {
   pdl_prologue();
   Counts unused;
-  int t = 0;                       // chunks come in increasing order: the search only moves forward
+  // Chunks come in increasing order, so the search for a chunk's tensor only moves forward; the
+  // tensor's fields are copied to registers when it changes, not once per chunk (they sit in an
+  // array of the kernel's parameters, which a varying index can only reach through loads).
+  int t = -1;
+  const float4* x = nullptr;
+  QuantOut o{};
+  unsigned long long n4 = 0, first = 0;
+  float scale = 1.0f;
+  int32_t qmin = 0, qmax = 0;
   for (unsigned long long chunk = blockIdx.x; chunk < a.total_chunks; chunk += gridDim.x) {
-    while (t + 1 < a.n && a.item[t + 1].first_chunk <= chunk) ++t;
-    const BatchItem& it = a.item[t];
-    const int32_t f = it.d_fmt != nullptr ? it.d_fmt->frac_bits : it.frac_bits;
-    const float scale = scale_of(f);
-    QuantOut o;
-    o.hi = it.hi; o.lo = it.lo; o.q16 = it.q16; o.planes = it.planes;
-    const unsigned long long base = (chunk - it.first_chunk) * kBatchChunk4 + threadIdx.x;
+    int nt = t < 0 ? 0 : t;
+    while (nt + 1 < a.n && a.item[nt + 1].first_chunk <= chunk) ++nt;
+    if (nt != t) {
+      t = nt;
+      const BatchItem& it = a.item[t];
+      x = it.x;
+      o.hi = it.hi; o.lo = it.lo; o.q16 = it.q16; o.planes = it.planes;
+      n4 = it.n4;
+      first = it.first_chunk;
+      scale = scale_of(it.d_fmt != nullptr ? it.d_fmt->frac_bits : it.frac_bits);
+      qmin = it.qmin;
+      qmax = it.qmax;
+    }
+    const unsigned long long base = (chunk - first) * kBatchChunk4 + threadIdx.x;
     float4 v[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const unsigned long long i = base + u * 256;
-      v[u] = i < it.n4 ? __ldcs(it.x + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      v[u] = i < n4 ? __ldcs(x + i) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const unsigned long long i = base + u * 256;
-      if (i < it.n4) {
+      if (i < n4) {
         int32_t q[4];
-        quantize_f32x4(v[u], scale, 0, it.qmin, it.qmax, unused, q);
+        quantize_f32x4(v[u], scale, 0, qmin, qmax, unused, q);
         store4(o, (size_t)i, q[0], q[1], q[2], q[3]);
       }
     }
