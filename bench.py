@@ -158,6 +158,10 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        # the multi-process launcher pins every rank to one OpenMP thread; only this rank computes here,
+        # so it takes the host cores it may run on (read by the OpenMP runtime when the oracle loads)
+        os.environ["OMP_NUM_THREADS"] = str(len(os.sched_getaffinity(0)))
     from oracle import reference as orc
     from paper_1711_04713_b200 import workloads as wl
     params = wl.make_params(wl.vgg16_specs(), seed=0)
