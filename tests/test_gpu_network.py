@@ -121,6 +121,16 @@ def test_stacks_with_stochastic_rounding(algo):
                        algo, threshold=thr, rounding_seed=12)
 
 
+@pytest.mark.slow
+def test_vgg16_with_stochastic_rounding():
+    """The real VGG16 shapes (224 x 224 inputs, every tile family of the tensor-core path, the split
+    inner products) with rounding_scheme STOCHASTIC for every layer, on a batch small enough for the
+    oracle's generator: every tensor, decimal point and counter."""
+    params = wl.make_params(wl.vgg16_specs(), seed=0)
+    x = wl.vgg16_input(4, seed=7)
+    _compare_stack(params, x, None, 16, (224, 224), 3, B.ALGO_AUTO, rounding_seed=21)
+
+
 def test_giga1net_stack():
     """Giga1Net (paper Table 1): kernels of 1, 7, 5 and 3, 3 to 128 channels, four pools, two inner
     products; every tensor, decimal point and counter against the oracle on a small batch."""
