@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(LIB_DIR, "libadaption.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "--shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-cudart", "static",
+    "--threads", "0",          # the translation units compile side by side
 ]
 
 
