@@ -318,6 +318,7 @@ ADAPTION_API int adaption_probe_i8_peak(int32_t bn, int32_t pair, int32_t iters,
  *   "bk" 32|64, "bn" 32|64, "kps" 1..4, "bres" 0, "wide" 0, "epigroups" 1   narrower tiles etc.
  *   "split_hh" 0   three 128-column accumulators are handed back together            (default 1)
  *   "stagger" 0    the last k-blocks of a tile are issued like the others                 (default 1)
+ *   "stage_bufs" 1 one output staging buffer per epilogue group even where two would fit (default 2)
  *   "pdl" 0        layer kernels are launched without programmatic stream serialization (default 1)
  *   "timeout_us" t limit of every device-side wait in microseconds (default 0: two seconds)
  *   "stall_at" i   the copy-issuing warps of every block stop before their i-th stage with nothing

@@ -103,6 +103,7 @@ struct TcParams {
   int pool_w;                 // store max(row 2j, row 2j+1) of the tile: half of a 2x2 max-pool (staged only)
   int epi_groups;             // 1, or 2: the epilogue warps form two groups that take alternate tiles
   int staged;                 // outputs leave through shared memory and bulk-tensor stores
+  int stage_bufs;             // staging buffers per epilogue group: 1, or 2 used in turn (narrow tiles)
   uint32_t stage_off;         // offset of the staging planes from the ring base
   uint32_t const_off;         // offset of the per-column epilogue constants (8 bytes per column and group)
 };
@@ -749,6 +750,10 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // the bulk stores committed so far have read their shared-memory source
+// ... all but the most recent group have (two staging buffers in turn)
+__device__ __forceinline__ void bulk_wait_read_all_but_one() {
+  asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+}
 __device__ __forceinline__ void bulk_wait_read_all() {
   asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
@@ -1182,8 +1187,10 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     const int col_end = min(p.BN, col_begin + cols_per_warp);
     const int row = quarter * 32 + lane;   // row of the tile (and of this CTA's staging planes)
     const int planes_bytes = kBM * p.BN * p.rq.out_planes;
-    const uint32_t stage_lo = ring + p.stage_off + (uint32_t)(group * planes_bytes);
-    const uint32_t stage_hi = stage_lo + (uint32_t)(kBM * p.BN);
+    const uint32_t stage_group = ring + p.stage_off + (uint32_t)(group * planes_bytes * p.stage_bufs);
+    uint32_t stage_lo = stage_group;
+    uint32_t stage_hi = stage_lo + (uint32_t)(kBM * p.BN);
+    uint32_t stage_turn = 0;
     // per-column epilogue constants of the current tile, one array per group, behind the staging planes
     long long* colconst = reinterpret_cast<long long*>(smem_raw + (ring - smem_u32(smem_raw)) + p.const_off) +
                           group * p.BN;
@@ -1219,7 +1226,15 @@ lp_gemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const_n0 = tc.n0;
       }
       // the previous tile's bulk stores must have read the staging planes before they are reused
-      if (p.staged && store_leader) bulk_wait_read_all();
+      // (with two buffers in turn: the store from two tiles ago)
+      if (p.stage_bufs == 2) {
+        stage_lo = stage_group + stage_turn * (uint32_t)planes_bytes;
+        stage_hi = stage_lo + (uint32_t)(kBM * p.BN);
+        stage_turn ^= 1u;
+        if (p.staged && store_leader) bulk_wait_read_all_but_one();
+      } else if (p.staged && store_leader) {
+        bulk_wait_read_all();
+      }
       if (lane == 0 && (ew & 3) == 0) TL_STAMP(2 + (ew >> 2), tile_iter, 0);
       // (staggered tail: the first thing to wait for is the low accumulator)
       const bool stagger = FAST && NACC == 3 && p.tail_stagger != 0;
@@ -1505,6 +1520,7 @@ struct TcConfig {
   int epi_groups = 1;
   bool staged = false;         // outputs staged in shared memory and written by bulk-tensor stores
   uint32_t stage_out_bytes = 0, stage_off = 0, const_bytes = 0;
+  int stage_bufs = 1;
   size_t smem_bytes = 0;
   size_t workspace_bytes = 0;
 };
@@ -1513,11 +1529,11 @@ struct TcConfig {
 // from the environment, so the layer calls themselves do no string work).  Each holds its
 // default until set; the setter is the only writer.
 enum Knob { kSplits, kPair, kFast, kStaged, kStages, kBK, kBN, kKps, kBres, kWide, kEpiGroups, kTimeoutUs, kStallAt,
-            kSplitHh, kPdl, kStagger, kNumKnobs };
+            kSplitHh, kPdl, kStagger, kStageBufs, kNumKnobs };
 const char* const kKnobNames[kNumKnobs] = {"splits", "pair", "fast", "staged", "stages", "bk", "bn", "kps", "bres",
-                                           "wide", "epigroups", "timeout_us", "stall_at", "split_hh", "pdl", "stagger"};
-const int kKnobDefaults[kNumKnobs] = {0, -1, 1, 1, 0, 0, 0, 0, 1, 1, 2, 0, -1, 1, 1, 1};
-std::atomic<int> g_knobs[kNumKnobs] = {{0}, {-1}, {1}, {1}, {0}, {0}, {0}, {0}, {1}, {1}, {2}, {0}, {-1}, {1}, {1}, {1}};
+                                           "wide", "epigroups", "timeout_us", "stall_at", "split_hh", "pdl", "stagger", "stage_bufs"};
+const int kKnobDefaults[kNumKnobs] = {0, -1, 1, 1, 0, 0, 0, 0, 1, 1, 2, 0, -1, 1, 1, 1, 2};
+std::atomic<int> g_knobs[kNumKnobs] = {{0}, {-1}, {1}, {1}, {0}, {0}, {0}, {0}, {1}, {1}, {2}, {0}, {-1}, {1}, {1}, {1}, {2}};
 inline int knob(Knob k) { return g_knobs[k].load(std::memory_order_relaxed); }
 
 TcConfig make_config_impl(const GemmProblem& g, bool allow_wide);
@@ -1677,8 +1693,27 @@ TcConfig make_config_impl(const GemmProblem& g, bool allow_wide) {
     c.stages = (int)((budget + c.stage_out_bytes - 1024 - c.b_res_bytes) / c.stage_bytes);
     c.staged = false;
     c.stage_out_bytes = 0;
+    c.stage_bufs = 1;
   }
   if (c.stages > kMaxStages) c.stages = kMaxStages;
+  // Narrow tiles with two epilogue groups: a second staging buffer per group, so that a group does
+  // not wait for its previous tile's bulk store to have read shared memory - where the ring keeps at
+  // least four stages beside it (short reductions with small stages, e.g. a packed first layer).
+  if (c.staged && c.epi_groups == 2 && c.BN <= 64 && knob(kStageBufs) != 1) {
+    const size_t extra = c.stage_out_bytes;
+    const size_t used = (size_t)c.stages * c.stage_bytes + c.b_res_bytes + 1024;
+    size_t slack = budget > used ? budget - used : 0;
+    int stages = c.stages;
+    while (slack < extra && stages > 4) {
+      --stages;
+      slack += c.stage_bytes;
+    }
+    if (slack >= extra) {
+      c.stages = stages;
+      c.stage_bufs = 2;
+      c.stage_out_bytes = (uint32_t)(2 * extra);
+    }
+  }
   const int stage_cap = knob(kStages);   // experiment knob: shallower ring
   if (stage_cap >= 2 && stage_cap < c.stages) c.stages = stage_cap;
   if (c.stages < 2) return c;
@@ -1995,6 +2030,7 @@ int launch_tensor(const GemmProblem& g) {
   p.pool_w = g.pool_w ? 1 : 0;
   p.epi_groups = c.epi_groups;
   p.staged = c.staged ? 1 : 0;
+  p.stage_bufs = c.stage_bufs;
   p.stage_off = c.stage_off;
   p.const_off = c.stage_off + c.stage_out_bytes;
   const bool single = c.nacc == 1;
